@@ -1,0 +1,152 @@
+/*
+ * attn.h -- exact softmax attention, forward and backward, for NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  Plain pointers and sizes only.  Unless a parameter says "host", every
+ * pointer is DEVICE memory owned by the caller; the library allocates nothing and
+ * frees nothing.  All work is enqueued on the given CUDA
+ * stream (a cudaStream_t passed as void*; NULL = the legacy default stream) and the
+ * calls return without synchronising.
+ *
+ * What is computed, per (batch, head), for Q, K, V, dO of shape n x d:
+ *
+ *   S_ij  = scale * sum_c Q_ic K_jc            kept (i,j) only; masked = excluded
+ *   LSE_i = ln sum_j exp(S_ij)                  (Definitions B.3, B.4: l = exp(S) 1)
+ *   P_ij  = exp(S_ij - LSE_i)                   (Definition B.5: f = diag(l)^-1 exp(S))
+ *   O     = P V                                 (Definition B.7; Definition 3.1)
+ *   dP    = dO V^T                              (Definition B.8: q)
+ *   D_i   = sum_c dO_ic O_ic                    (Definition B.9, second matrix form)
+ *   dS    = P o (dP - D 1^T)                    (Definition B.9: p)
+ *   dQ    = scale * dS K,  dK = scale * dS^T Q  (chain rule through Definition 3.2,
+ *   dV    = P^T dO                               dL/dX = A1^T p A2, with Q = A1 X, K = A2)
+ *
+ * The paper's inputs A1 X, A2, A3 Y are the caller's Q, K, V: the projections sit
+ * in front of this boundary (Section 3.1, remark on Q, K, V), and the 1/sqrt(d)
+ * factor the paper folds into X is the explicit `scale`.
+ *
+ * Layout: Q, K, V, O, dO, dQ, dK, dV are [batch, heads, n, d] contiguous, d fastest,
+ * element type `dt`; LSE is float [batch, heads, n], natural logarithm.  Base
+ * pointers must be 16-byte aligned.  Outputs are overwritten, never accumulated into.
+ * A query row with no kept key gets O = 0, LSE = -inf and contributes no gradient.
+ *
+ * Errors: argument errors are returned synchronously, before anything is enqueued.
+ * Errors found by a kernel (a bounded wait that ran out) are written to the 4-byte
+ * status word at the start of `workspace`; read it with attn_workspace_status().
+ * A device that is not compute capability 10.x gets ATTN_ERR_ARCH: there is no
+ * fallback path of any kind.
+ */
+#ifndef ATTN_B200_H
+#define ATTN_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    ATTN_OK = 0,
+    ATTN_ERR_NULL = 1,           /* a required pointer is NULL */
+    ATTN_ERR_SHAPE = 2,          /* n, d, heads or batch out of the supported range */
+    ATTN_ERR_DTYPE = 3,          /* unknown dtype, or dtype not supported by the chosen algorithm */
+    ATTN_ERR_ALIGN = 4,          /* a base pointer is not 16-byte aligned */
+    ATTN_ERR_TILE = 5,           /* tile_q / tile_k / tile_d not in attn_supported_cfgs() */
+    ATTN_ERR_MASK = 6,           /* bad mask description */
+    ATTN_ERR_WORKSPACE = 7,      /* workspace NULL or smaller than attn_*_workspace_bytes() */
+    ATTN_ERR_ARCH = 8,           /* current device is not sm_100 */
+    ATTN_ERR_LAUNCH = 9,         /* the CUDA runtime refused a launch or a tensor-map encode */
+    ATTN_ERR_DEVICE_TIMEOUT = 10 /* a kernel gave up on a bounded wait (status word only) */
+} attn_status;
+
+typedef enum { ATTN_F32 = 0, ATTN_BF16 = 1 } attn_dtype;
+
+typedef enum { ATTN_MASK_NONE = 0, ATTN_MASK_CAUSAL = 1, ATTN_MASK_BLOCK_SPARSE = 2 } attn_mask_kind;
+
+/* Which (i, j) score entries are kept.  NULL means ATTN_MASK_NONE.
+ *   CAUSAL:       keep j <= i (one n for queries and keys).
+ *   BLOCK_SPARSE: keep (i, j) iff block_mask[h][i / block][j / block] != 0, where
+ *                 block_mask is DEVICE uint8 [mask_heads][nb][nb], nb = ceil(n / block);
+ *                 mask_heads is 1 (shared by every batch and head) or batch * heads.
+ *                 The tensor-core algorithms need block to be a multiple of 128.
+ * This is the sparse setting of Section 4.1 with Z_QK = the number of kept entries;
+ * a masked score is minus infinity, not a stored zero. */
+typedef struct {
+    int kind;                  /* attn_mask_kind */
+    int block;
+    const uint8_t *block_mask; /* device */
+    int mask_heads;
+} attn_mask;
+
+/* Which algorithm runs.  The tile sizes play the role of the paper's cache size M.
+ *   FUSED        large-cache regime (Appendix D): score tiles never leave the SM.
+ *   MATERIALIZED small-cache regime (Appendix C): P, dP and dS are written to and
+ *                re-read from device memory in tile_q x tile_k blocks, the head
+ *                dimension walked in tile_d chunks (backward only; its forward is FUSED).
+ *   SIMT         fp32 FMA kernels without tensor cores; the only choice for ATTN_F32.
+ *   AUTO         ATTN_F32 -> SIMT; ATTN_BF16 -> FUSED.                              */
+typedef enum { ATTN_ALGO_AUTO = 0, ATTN_ALGO_FUSED = 1, ATTN_ALGO_MATERIALIZED = 2, ATTN_ALGO_SIMT = 3 } attn_algo;
+
+/* NULL or all zeros = defaults.  deterministic != 0 forbids floating-point atomics
+ * (results are then bitwise repeatable run to run). */
+typedef struct {
+    int tile_q, tile_k, tile_d;
+    int algo; /* attn_algo */
+    int deterministic;
+} attn_cfg;
+
+/* Forward pass (Definition 3.1): writes O [batch,heads,n,d] and LSE [batch,heads,n].
+ * n >= 1; d a multiple of 8 up to 256 (SIMT) or one of 64, 128, 256 (tensor-core
+ * algorithms, which also need n to be a multiple of 8).  scale = 0 means 1/sqrt(d).
+ * workspace: at least attn_fwd_workspace_bytes(), 256-byte aligned, device. */
+attn_status attn_fwd(const void *Q, const void *K, const void *V, void *O, float *LSE,
+                     int n, int d, int heads, int batch, const attn_mask *mask,
+                     int dt /* attn_dtype */, float scale, const attn_cfg *cfg,
+                     void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Backward pass (Definitions B.8, B.9 and 3.2; Algorithm "large cache phase 2" with
+ * dQ, dK, dV in place of the weight gradient): reads Q, K, V, dO and the forward's
+ * O and LSE, writes dQ, dK, dV.  Same constraints as attn_fwd. */
+attn_status attn_bwd(const void *Q, const void *K, const void *V, const void *O, const void *dO,
+                     const float *LSE, void *dQ, void *dK, void *dV,
+                     int n, int d, int heads, int batch, const attn_mask *mask,
+                     int dt, float scale, const attn_cfg *cfg,
+                     void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* D_i = sum_c dO_ic O_ic for `rows` rows of length d (the vector v of Definition B.9
+ * and of the large-cache phase-2 algorithm).  D is float [rows].  attn_bwd runs this
+ * itself; it is exported because it is the memory-bound step of the path. */
+attn_status attn_bwd_preprocess(const void *O, const void *dO, float *D, size_t rows, int d, int dt,
+                                void *cuda_stream);
+
+/* Workspace sizes in bytes for the same arguments (0 on invalid arguments). */
+size_t attn_fwd_workspace_bytes(int n, int d, int heads, int batch, const attn_mask *mask, int dt,
+                                const attn_cfg *cfg);
+size_t attn_bwd_workspace_bytes(int n, int d, int heads, int batch, const attn_mask *mask, int dt,
+                                const attn_cfg *cfg);
+
+/* Synchronises `cuda_stream`, then returns the status word a kernel may have set in
+ * `workspace` (ATTN_OK if none did). */
+attn_status attn_workspace_status(const void *workspace, void *cuda_stream);
+
+/* Tile configurations that attn_fwd / attn_bwd accept for (d, dt): fills up to
+ * max_out entries of `out` (host), returns how many exist. */
+int attn_supported_cfgs(int d, int dt, attn_cfg *out /* host */, int max_out);
+
+/* On-chip elements (shared memory + tensor memory, counted in elements of the
+ * operand type) one CTA of this configuration holds: the paper's M (Section 3.3
+ * counts the cache in items).  0 on an unsupported configuration. */
+size_t attn_cfg_onchip_elems(int d, int dt, const attn_cfg *cfg, int backward);
+
+/* Closed-form I/O bounds, constant factor 1, in elements, per head.
+ * backward != 0: min{(n^2 d^2 + n d^3)/M, (n^2 d + n d^2)/sqrt(M)} (Theorem 1.1);
+ * backward == 0: min{n^2 d^2/M, n^2 d/sqrt(M)} (Table 1, forward). */
+double attn_io_bound_elems(double n, double d, double M, int backward);
+/* min{Z_input^2/M, Z_input sqrt(Z_QK)/sqrt(M)} (Theorem 1.2). */
+double attn_io_bound_sparse_elems(double z_input, double z_qk, double M);
+
+const char *attn_status_str(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ATTN_B200_H */

@@ -1,18 +1,14 @@
 """Exact softmax attention forward/backward for B200 (sm_100a) behind a C ABI.
 
-``inputs`` (seeded synthetic inputs) imports without the compiled library; the
+``inputs`` (seeded synthetic inputs) works without the compiled library; the
 binding (``attn_fwd``, ``attn_bwd`` and friends) loads ``libattn_b200.so`` on first
-use and raises if it is missing -- there is no CPU fallback.
+call and raises if it is missing -- there is no CPU fallback.
 """
 from . import inputs  # noqa: F401
-
-_BINDING_NAMES = None
-
-
-def __getattr__(name):
-    # The binding is imported lazily so that input generation works on machines
-    # where the CUDA library has not been built.
-    from . import binding
-    if hasattr(binding, name):
-        return getattr(binding, name)
-    raise AttributeError(name)
+from . import binding  # noqa: F401
+from .binding import (  # noqa: F401
+    ATTN_ALGO_AUTO, ATTN_ALGO_FUSED, ATTN_ALGO_MATERIALIZED, ATTN_ALGO_SIMT, ATTN_BF16, ATTN_F32,
+    ATTN_MASK_BLOCK_SPARSE, ATTN_MASK_CAUSAL, ATTN_MASK_NONE, AttnError, Cfg, Mask, attn_bwd, attn_bwd_preprocess,
+    attn_bwd_workspace_bytes, attn_cfg_onchip_elems, attn_fwd, attn_fwd_workspace_bytes, attn_io_bound_elems,
+    attn_io_bound_sparse_elems, attn_supported_cfgs, attn_workspace_status, status_str,
+)

@@ -1,0 +1,233 @@
+"""ctypes binding of ``libattn_b200.so`` -- same names as ``include/attn.h``.
+
+Argument marshalling only: every step of the attention path runs in the library's
+CUDA kernels.  Tensors are torch CUDA tensors (torch supplies device memory and the
+stream, nothing else); ``attn_fwd`` / ``attn_bwd`` enqueue on torch's current stream and
+do not synchronise.  If the library is missing this module raises -- there is no
+fallback of any kind.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libattn_b200.so")
+
+ATTN_OK = 0
+(ATTN_ERR_NULL, ATTN_ERR_SHAPE, ATTN_ERR_DTYPE, ATTN_ERR_ALIGN, ATTN_ERR_TILE, ATTN_ERR_MASK, ATTN_ERR_WORKSPACE,
+ ATTN_ERR_ARCH, ATTN_ERR_LAUNCH, ATTN_ERR_DEVICE_TIMEOUT) = range(1, 11)
+ATTN_F32, ATTN_BF16 = 0, 1
+ATTN_MASK_NONE, ATTN_MASK_CAUSAL, ATTN_MASK_BLOCK_SPARSE = 0, 1, 2
+ATTN_ALGO_AUTO, ATTN_ALGO_FUSED, ATTN_ALGO_MATERIALIZED, ATTN_ALGO_SIMT = 0, 1, 2, 3
+
+# every symbol include/attn.h declares
+EXPORTS = (
+    "attn_fwd", "attn_bwd", "attn_bwd_preprocess", "attn_fwd_workspace_bytes", "attn_bwd_workspace_bytes",
+    "attn_workspace_status", "attn_supported_cfgs", "attn_cfg_onchip_elems", "attn_io_bound_elems",
+    "attn_io_bound_sparse_elems", "attn_status_str",
+)
+
+
+class AttnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_str(status)} (attn_status {status})")
+
+
+class CMask(ctypes.Structure):
+    _fields_ = [("kind", ctypes.c_int), ("block", ctypes.c_int), ("block_mask", ctypes.c_void_p),
+                ("mask_heads", ctypes.c_int)]
+
+
+class CCfg(ctypes.Structure):
+    _fields_ = [("tile_q", ctypes.c_int), ("tile_k", ctypes.c_int), ("tile_d", ctypes.c_int),
+                ("algo", ctypes.c_int), ("deterministic", ctypes.c_int)]
+
+
+@dataclass
+class Mask:
+    """Which score entries are kept; ``block_mask`` is a CUDA uint8 tensor ``[mask_heads, nb, nb]``."""
+    kind: int = ATTN_MASK_NONE
+    block: int = 128
+    block_mask: object = None
+
+    def c(self) -> CMask | None:
+        if self.kind == ATTN_MASK_BLOCK_SPARSE:
+            bm = self.block_mask
+            return CMask(self.kind, self.block, bm.data_ptr() if bm is not None else None,
+                         int(bm.shape[0]) if bm is not None else 1)
+        return CMask(self.kind, 0, None, 1)
+
+
+@dataclass
+class Cfg:
+    tile_q: int = 0
+    tile_k: int = 0
+    tile_d: int = 0
+    algo: int = ATTN_ALGO_AUTO
+    deterministic: int = 0
+
+    def c(self) -> CCfg:
+        return CCfg(self.tile_q, self.tile_k, self.tile_d, self.algo, self.deterministic)
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads the library (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2410_09397_b200.build` "
+                           "(there is no fallback path)")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, ci, cf, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    L.attn_fwd.restype = ci
+    L.attn_fwd.argtypes = [vp, vp, vp, vp, vp, ci, ci, ci, ci, ctypes.POINTER(CMask), ci, cf,
+                           ctypes.POINTER(CCfg), vp, sz, vp]
+    L.attn_bwd.restype = ci
+    L.attn_bwd.argtypes = [vp] * 9 + [ci, ci, ci, ci, ctypes.POINTER(CMask), ci, cf, ctypes.POINTER(CCfg), vp, sz, vp]
+    L.attn_bwd_preprocess.restype = ci
+    L.attn_bwd_preprocess.argtypes = [vp, vp, vp, sz, ci, ci, vp]
+    for f in (L.attn_fwd_workspace_bytes, L.attn_bwd_workspace_bytes):
+        f.restype = sz
+        f.argtypes = [ci, ci, ci, ci, ctypes.POINTER(CMask), ci, ctypes.POINTER(CCfg)]
+    L.attn_workspace_status.restype = ci
+    L.attn_workspace_status.argtypes = [vp, vp]
+    L.attn_supported_cfgs.restype = ci
+    L.attn_supported_cfgs.argtypes = [ci, ci, ctypes.POINTER(CCfg), ci]
+    L.attn_cfg_onchip_elems.restype = sz
+    L.attn_cfg_onchip_elems.argtypes = [ci, ci, ctypes.POINTER(CCfg), ci]
+    L.attn_io_bound_elems.restype = ctypes.c_double
+    L.attn_io_bound_elems.argtypes = [ctypes.c_double] * 3 + [ci]
+    L.attn_io_bound_sparse_elems.restype = ctypes.c_double
+    L.attn_io_bound_sparse_elems.argtypes = [ctypes.c_double] * 3
+    L.attn_status_str.restype = ctypes.c_char_p
+    L.attn_status_str.argtypes = [ci]
+    _lib = L
+    return L
+
+
+def status_str(status: int) -> str:
+    return lib().attn_status_str(int(status)).decode()
+
+
+def _ref(x):
+    return None if x is None else ctypes.byref(x)
+
+
+def _dtype_code(t) -> int:
+    import torch
+    if t.dtype == torch.float32:
+        return ATTN_F32
+    if t.dtype == torch.bfloat16:
+        return ATTN_BF16
+    raise AttnError(ATTN_ERR_DTYPE, "binding")
+
+
+def _check_tensors(*ts):
+    for t in ts:
+        if not t.is_cuda or not t.is_contiguous():
+            raise ValueError("tensors must be contiguous CUDA tensors")
+
+
+def _stream() -> int:
+    import torch
+    return torch.cuda.current_stream().cuda_stream
+
+
+def attn_fwd_workspace_bytes(n, d, heads, batch, mask: Mask | None, dt: int, cfg: Cfg | None) -> int:
+    return int(lib().attn_fwd_workspace_bytes(n, d, heads, batch, _ref(mask.c() if mask else None), dt,
+                                              _ref(cfg.c() if cfg else None)))
+
+
+def attn_bwd_workspace_bytes(n, d, heads, batch, mask: Mask | None, dt: int, cfg: Cfg | None) -> int:
+    return int(lib().attn_bwd_workspace_bytes(n, d, heads, batch, _ref(mask.c() if mask else None), dt,
+                                              _ref(cfg.c() if cfg else None)))
+
+
+def _workspace(nbytes: int, like):
+    import torch
+    return torch.empty(max(nbytes, 256), dtype=torch.uint8, device=like.device)
+
+
+def attn_fwd(Q, K, V, O=None, LSE=None, *, mask: Mask | None = None, scale: float = 0.0, cfg: Cfg | None = None,
+             workspace=None):
+    """O, LSE = softmax(scale * Q K^T restricted to kept entries) V.  Tensors ``[batch, heads, n, d]``."""
+    import torch
+    _check_tensors(Q, K, V)
+    b, h, n, d = Q.shape
+    dt = _dtype_code(Q)
+    if O is None:
+        O = torch.empty_like(Q)
+    if LSE is None:
+        LSE = torch.empty((b, h, n), dtype=torch.float32, device=Q.device)
+    if workspace is None:
+        workspace = _workspace(attn_fwd_workspace_bytes(n, d, h, b, mask, dt, cfg), Q)
+    cm, cc = (mask.c() if mask else None), (cfg.c() if cfg else None)
+    st = lib().attn_fwd(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), LSE.data_ptr(), n, d, h, b, _ref(cm),
+                        dt, scale, _ref(cc), workspace.data_ptr(), workspace.numel(), _stream())
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_fwd")
+    return O, LSE
+
+
+def attn_bwd(Q, K, V, O, dO, LSE, dQ=None, dK=None, dV=None, *, mask: Mask | None = None, scale: float = 0.0,
+             cfg: Cfg | None = None, workspace=None):
+    """dQ, dK, dV of sum(O o G) given dO = G and the forward's O, LSE."""
+    import torch
+    _check_tensors(Q, K, V, O, dO, LSE)
+    b, h, n, d = Q.shape
+    dt = _dtype_code(Q)
+    dQ = torch.empty_like(Q) if dQ is None else dQ
+    dK = torch.empty_like(Q) if dK is None else dK
+    dV = torch.empty_like(Q) if dV is None else dV
+    if workspace is None:
+        workspace = _workspace(attn_bwd_workspace_bytes(n, d, h, b, mask, dt, cfg), Q)
+    cm, cc = (mask.c() if mask else None), (cfg.c() if cfg else None)
+    st = lib().attn_bwd(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), dO.data_ptr(), LSE.data_ptr(),
+                        dQ.data_ptr(), dK.data_ptr(), dV.data_ptr(), n, d, h, b, _ref(cm), dt, scale, _ref(cc),
+                        workspace.data_ptr(), workspace.numel(), _stream())
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_bwd")
+    return dQ, dK, dV
+
+
+def attn_bwd_preprocess(O, dO, D=None):
+    """D = rowsum(dO o O) over the last dimension; returns float32 of O.shape[:-1]."""
+    import torch
+    _check_tensors(O, dO)
+    d = O.shape[-1]
+    rows = O.numel() // d
+    if D is None:
+        D = torch.empty(O.shape[:-1], dtype=torch.float32, device=O.device)
+    st = lib().attn_bwd_preprocess(O.data_ptr(), dO.data_ptr(), D.data_ptr(), rows, d, _dtype_code(O), _stream())
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_bwd_preprocess")
+    return D
+
+
+def attn_workspace_status(workspace) -> int:
+    return int(lib().attn_workspace_status(workspace.data_ptr(), _stream()))
+
+
+def attn_supported_cfgs(d: int, dt: int) -> list[Cfg]:
+    buf = (CCfg * 64)()
+    cnt = lib().attn_supported_cfgs(d, dt, buf, 64)
+    return [Cfg(buf[i].tile_q, buf[i].tile_k, buf[i].tile_d, buf[i].algo, 0) for i in range(min(cnt, 64))]
+
+
+def attn_cfg_onchip_elems(d: int, dt: int, cfg: Cfg | None, backward: bool) -> int:
+    return int(lib().attn_cfg_onchip_elems(d, dt, _ref(cfg.c() if cfg else None), int(backward)))
+
+
+def attn_io_bound_elems(n, d, M, backward: bool) -> float:
+    return float(lib().attn_io_bound_elems(float(n), float(d), float(M), int(backward)))
+
+
+def attn_io_bound_sparse_elems(z_input, z_qk, M) -> float:
+    return float(lib().attn_io_bound_sparse_elems(float(z_input), float(z_qk), float(M)))

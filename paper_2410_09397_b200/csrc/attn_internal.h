@@ -1,0 +1,56 @@
+// Internal declarations shared by the translation units of libattn_b200.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "attn.h"
+
+namespace attn {
+
+// One fully validated problem, as handed from the C ABI to the kernel launchers.
+struct Problem {
+    const void *Q, *K, *V, *O, *dO;   // inputs (O, dO only for the backward)
+    const float *LSE;                 // backward input
+    void *Oout;                       // forward outputs
+    float *LSEout;
+    void *dQ, *dK, *dV;               // backward outputs
+    int n, d, heads, batch;
+    long BH;                          // batch * heads
+    int mask_kind, block, mask_heads, nb;
+    const uint8_t *block_mask;
+    int dt;
+    float scale;
+    attn_cfg cfg;                     // resolved: algo and tiles are final
+    // workspace sections (device)
+    uint32_t *status;                 // 4-byte status word
+    float *D;                         // [BH * n]
+    int *row_ptr, *col_idx;           // block-CSR of the mask: [mask_heads][nb+1], [mask_heads][nb*nb]
+    int *col_ptr, *row_idx;           // block-CSC
+    float *dQ_acc;                    // fp32 dQ accumulator [BH * n * d] (fused backward with atomics)
+    void *matP, *matdP, *matdS;       // materialised n x n buffers (per head chunk)
+    int mat_heads;                    // heads materialised at once
+    cudaStream_t stream;
+};
+
+struct WorkspaceLayout {
+    size_t status, D, row_ptr, col_idx, col_ptr, row_idx, dQ_acc, matP, matdP, matdS, total;
+    int mat_heads;
+};
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// SIMT fp32 path (attn_simt.cu)
+attn_status simt_fwd(const Problem &p);
+attn_status simt_bwd(const Problem &p);
+attn_status preprocess_D(const void *O, const void *dO, float *D, size_t rows, int d, int dt, cudaStream_t s);
+attn_status build_block_index(const Problem &p);
+
+// Tensor-core path (attn_tc_*.cu)
+attn_status tc_fwd(const Problem &p);
+attn_status tc_bwd(const Problem &p);
+attn_status mat_bwd(const Problem &p);
+bool tc_cfg_supported(int d, const attn_cfg &cfg, int backward);
+size_t tc_cfg_onchip_bytes(int d, const attn_cfg &cfg, int backward);
+
+}  // namespace attn

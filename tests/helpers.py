@@ -1,0 +1,88 @@
+"""Shared helpers of the GPU parity tests: seeded inputs -> oracle and CUDA library -> compare."""
+from __future__ import annotations
+
+import numpy as np
+
+from oracle import oracle as orc
+from paper_2410_09397_b200 import inputs
+
+TOL = {"f32": 1e-4, "bf16": 2e-2}   # max|err| <= TOL * max|ref| per output tensor
+
+
+def oracle_mask_kwargs(mask_kind, block, bmask):
+    if mask_kind == inputs.MASK_BLOCK_SPARSE:
+        return dict(mask_kind=orc.MASK_BLOCK, block=block, mask_bits=bmask)
+    return dict(mask_kind=mask_kind)
+
+
+def make_inputs(seed, b, h, n, d, dtype):
+    bf16 = dtype == "bf16"
+    return {name: inputs.normal_tensor(seed, tid, (b, h, n, d), bf16=bf16)
+            for name, tid in (("Q", 0), ("K", 1), ("V", 2), ("dO", 3))}
+
+
+def to_dev(x, dtype):
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(x)).cuda()
+    return t.to(torch.bfloat16) if dtype == "bf16" else t.float()
+
+
+def to_np(t):
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def rel_err(got, ref):
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    assert got.shape == ref.shape
+    assert np.all(np.isfinite(got) | ~np.isfinite(ref)), "NaN/Inf in result"
+    fin = np.isfinite(ref)
+    assert np.array_equal(got[~fin], ref[~fin]), "non-finite entries differ"
+    denom = max(np.abs(ref[fin]).max(), 1e-30) if fin.any() else 1.0
+    return float(np.abs(got[fin] - ref[fin]).max() / denom) if fin.any() else 0.0
+
+
+def run_case(b, h, n, d, dtype, mask_kind, *, seed=7, block=128, bmask=None, cfg=None, scale=0.0,
+             keep_prob=0.3, check_bwd_only=True):
+    """Runs forward + backward on the GPU and the oracle; returns dict of relative errors."""
+    import torch
+    import paper_2410_09397_b200 as attn
+    from paper_2410_09397_b200 import binding as B
+
+    x = make_inputs(seed, b, h, n, d, dtype)
+    if mask_kind == inputs.MASK_BLOCK_SPARSE and bmask is None:
+        bmask = inputs.block_mask(seed + 100, (n + block - 1) // block, keep_prob)
+    mk = oracle_mask_kwargs(mask_kind, block, bmask)
+    sc = None if scale == 0.0 else scale
+    O_ref, LSE_ref = orc.attn_fwd(x["Q"], x["K"], x["V"], scale=sc, **mk)
+    g_ref = orc.attn_bwd(x["Q"], x["K"], x["V"], O_ref, x["dO"], LSE_ref, scale=sc, **mk)
+
+    dev = {k: to_dev(v, dtype) for k, v in x.items()}
+    mask = None
+    if mask_kind != inputs.MASK_NONE:
+        mask = B.Mask(kind=mask_kind, block=block,
+                      block_mask=torch.from_numpy(bmask).cuda() if bmask is not None else None)
+    O, LSE = attn.attn_fwd(dev["Q"], dev["K"], dev["V"], mask=mask, scale=scale, cfg=cfg)
+    dQ, dK, dV = attn.attn_bwd(dev["Q"], dev["K"], dev["V"], O, dev["dO"], LSE, mask=mask, scale=scale, cfg=cfg)
+    torch.cuda.synchronize()
+    errs = {
+        "O": rel_err(to_np(O), O_ref), "LSE": rel_err(to_np(LSE), LSE_ref),
+        "dQ": rel_err(to_np(dQ), g_ref[0]), "dK": rel_err(to_np(dK), g_ref[1]), "dV": rel_err(to_np(dV), g_ref[2]),
+    }
+    if check_bwd_only:
+        # backward alone, fed the oracle's O and LSE rounded to the storage types
+        O_in = to_dev(O_ref.astype(np.float32), dtype)
+        LSE_in = torch.from_numpy(LSE_ref.astype(np.float32)).cuda()
+        g_ref2 = orc.attn_bwd(x["Q"], x["K"], x["V"], to_np(O_in), x["dO"], to_np(LSE_in), scale=sc, **mk)
+        dQ2, dK2, dV2 = attn.attn_bwd(dev["Q"], dev["K"], dev["V"], O_in, dev["dO"], LSE_in, mask=mask, scale=scale,
+                                      cfg=cfg)
+        torch.cuda.synchronize()
+        errs.update({"dQ_bwdonly": rel_err(to_np(dQ2), g_ref2[0]), "dK_bwdonly": rel_err(to_np(dK2), g_ref2[1]),
+                     "dV_bwdonly": rel_err(to_np(dV2), g_ref2[2])})
+    return errs
+
+
+def assert_within(errs, dtype):
+    tol = TOL[dtype]
+    bad = {k: v for k, v in errs.items() if not v <= tol}
+    assert not bad, f"over tolerance {tol}: {bad} (all: {errs})"
