@@ -38,7 +38,9 @@ def rel_err(got, ref):
     assert np.all(np.isfinite(got) | ~np.isfinite(ref)), "NaN/Inf in result"
     fin = np.isfinite(ref)
     assert np.array_equal(got[~fin], ref[~fin]), "non-finite entries differ"
-    denom = max(np.abs(ref[fin]).max(), 1e-30) if fin.any() else 1.0
+    # inputs are N(0,1); a reference that is identically zero (n = 1: dQ = dK = 0) is
+    # compared on an absolute floor instead of dividing by zero
+    denom = max(np.abs(ref[fin]).max(), 1e-2) if fin.any() else 1.0
     return float(np.abs(got[fin] - ref[fin]).max() / denom) if fin.any() else 0.0
 
 
