@@ -1,0 +1,442 @@
+#!/usr/bin/env python
+"""Benchmark of the attention hot path (forward saving LSE, then backward dQ/dK/dV).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload C3]
+
+One "step" is one pass of the whole hot path over one batch of the workload: forward
+(O, LSE), the D pre-pass and the backward kernels.  The metric is the backward's
+algorithmic TFLOP/s (10 * kept * d per head: the five products QK^T, dO V^T, P^T dO,
+dS^T Q, dS K; recomputation is not counted), timed with CUDA events around the backward
+call of every timed step.  Inputs are seeded synthetic N(0,1) tensors rounded to bf16.
+
+With N > 1 (launched under torch.distributed.run) every rank owns its own batch of the
+workload -- (batch, head) units are independent, so there is no data-path collective --
+and the value is the aggregate over ranks divided by the slowest rank's time.
+
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2410_09397_b200 import inputs  # noqa: E402
+
+METRIC = "attention backward TFLOP/s (bf16, n=8192, d=128)"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def kept_entries(w: inputs.Workload, bmask) -> float:
+    """Kept score entries per head used for FLOP counting (causal counted as n^2 / 2)."""
+    if w.mask == inputs.MASK_NONE:
+        return float(w.n) * w.n
+    if w.mask == inputs.MASK_CAUSAL:
+        return float(w.n) * w.n / 2
+    return float(bmask[0].sum()) * w.block * w.block
+
+
+def flops(w: inputs.Workload, bmask, heads: int | None = None):
+    bh = w.batch * w.heads if heads is None else heads
+    k = kept_entries(w, bmask)
+    return 4.0 * k * w.d * bh, 10.0 * k * w.d * bh   # forward, backward
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.thread.join(timeout=5)
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in self.rows:
+            if len(r) < 6:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def physical_gpu_index(local: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local])
+        except (ValueError, IndexError):
+            return local
+    return local
+
+
+def max_over_ranks(values, world: int):
+    """Element-wise max of a list of floats over all ranks (identity when world == 1)."""
+    if world == 1:
+        return list(values)
+    import torch
+    import torch.distributed as dist
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor(values, dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.cpu()]
+
+
+def sum_over_ranks(values, world: int):
+    if world == 1:
+        return list(values)
+    import torch
+    import torch.distributed as dist
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor(values, dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return [float(v) for v in t.cpu()]
+
+
+def cpu_baseline(w: inputs.Workload, bmask, budget_s: float = 15.0):
+    """Times the float64 oracle's backward on a bounded sample: whole (batch, head) units."""
+    from oracle import oracle as orc
+    kind = {inputs.MASK_NONE: orc.MASK_NONE, inputs.MASK_CAUSAL: orc.MASK_CAUSAL,
+            inputs.MASK_BLOCK_SPARSE: orc.MASK_BLOCK}[w.mask]
+    mk = dict(mask_kind=kind, block=w.block, mask_bits=bmask)
+
+    def run(units):
+        x = {k: v.astype(np.float64)[None] for k, v in w.tensors(head_slice=(0, units)).items()}
+        O, LSE = orc.attn_fwd(x["Q"], x["K"], x["V"], **mk)
+        t = time.perf_counter()
+        orc.attn_bwd(x["Q"], x["K"], x["V"], O, x["dO"], LSE, **mk)
+        return time.perf_counter() - t
+
+    t1 = run(1)
+    units = int(max(1, min(w.batch * w.heads, budget_s // max(t1, 1e-3))))
+    t = run(units) if units > 1 else t1
+    _, fb = flops(w, bmask, heads=units)
+    return {"value": fb / t / 1e12, "unit": "TFLOP/s", "cores": orc.threads(), "kind": "oracle",
+            "sample": f"backward of {units} of {w.batch * w.heads} (batch, head) units of {w.name} "
+                      f"(n={w.n}, d={w.d}), float64, given the oracle's own forward; {t:.2f} s",
+            "seconds": t}
+
+
+def run_reference(args, w, bmask, rank, world):
+    """--impl reference: the oracle as it stands on the host cores, a bounded sample per step."""
+    if rank != 0:
+        return
+    from oracle import oracle as orc
+    kind = {inputs.MASK_NONE: orc.MASK_NONE, inputs.MASK_CAUSAL: orc.MASK_CAUSAL,
+            inputs.MASK_BLOCK_SPARSE: orc.MASK_BLOCK}[w.mask]
+    mk = dict(mask_kind=kind, block=w.block, mask_bits=bmask)
+    x = {k: v.astype(np.float64)[None] for k, v in w.tensors(head_slice=(0, 1)).items()}
+    # sample: the leading r rows of one (batch, head) unit.  For the causal workload this
+    # is a self-contained sub-problem (rows < r only see keys < r); r is sized so that
+    # all steps end within about two minutes.
+    r = min(w.n, 1024)
+    if w.mask == inputs.MASK_BLOCK_SPARSE:
+        r = w.n
+    xs = {k: np.ascontiguousarray(v[:, :, :r]) for k, v in x.items()}
+    mks = dict(mk)
+    if w.mask == inputs.MASK_BLOCK_SPARSE:
+        mks["mask_bits"] = bmask
+    O, LSE = orc.attn_fwd(xs["Q"], xs["K"], xs["V"], **mks)
+    t = time.perf_counter()
+    orc.attn_bwd(xs["Q"], xs["K"], xs["V"], O, xs["dO"], LSE, **mks)
+    t_probe = time.perf_counter() - t
+    total_steps = args.steps + args.warmup
+    if w.mask != inputs.MASK_BLOCK_SPARSE:
+        while r * 2 <= w.n and t_probe * 4 * total_steps < 120.0:
+            r *= 2
+            t_probe *= 4
+        xs = {k: np.ascontiguousarray(v[:, :, :r]) for k, v in x.items()}
+        O, LSE = orc.attn_fwd(xs["Q"], xs["K"], xs["V"], **mks)
+    if w.mask == inputs.MASK_NONE:
+        kept = float(r) * r
+    elif w.mask == inputs.MASK_CAUSAL:
+        kept = float(r) * r / 2
+    else:
+        kept = kept_entries(w, bmask)
+    fb = 10.0 * kept * w.d
+    for _ in range(args.warmup):
+        orc.attn_bwd(xs["Q"], xs["K"], xs["V"], O, xs["dO"], LSE, **mks)
+    t = time.perf_counter()
+    for _ in range(args.steps):
+        orc.attn_bwd(xs["Q"], xs["K"], xs["V"], O, xs["dO"], LSE, **mks)
+    dt = time.perf_counter() - t
+    val = fb * args.steps / dt / 1e12
+    sample = (f"per step: backward of the leading {r} x {r} sub-problem of one (batch, head) unit of {w.name} "
+              f"(n={w.n}, d={w.d}), float64 oracle on the host")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(w), "sample": sample},
+        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": orc.threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_name(w):
+    mask = {0: "no mask", 1: "causal", 2: f"block-sparse {w.block}x{w.block} p={w.keep_prob}"}[w.mask]
+    return f"{w.name}: batch={w.batch} heads={w.heads} n={w.n} d={w.d} {w.dtype} {mask}"
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C3", choices=sorted(inputs.WORKLOADS))
+    ap.add_argument("--algo", default="auto", choices=["auto", "fused", "materialized", "simt"])
+    ap.add_argument("--tile-q", type=int, default=0)
+    ap.add_argument("--tile-k", type=int, default=0)
+    ap.add_argument("--tile-d", type=int, default=0)
+    ap.add_argument("--deterministic", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    w = inputs.WORKLOADS[args.workload]
+    bmask = w.block_mask()
+
+    if args.impl == "reference":
+        run_reference(args, w, bmask, rank, world)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_2410_09397_b200 as attn
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the attention library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    attn.binding.lib()   # fail loudly here if the library is missing
+
+    algo = {"auto": attn.ATTN_ALGO_AUTO, "fused": attn.ATTN_ALGO_FUSED, "materialized": attn.ATTN_ALGO_MATERIALIZED,
+            "simt": attn.ATTN_ALGO_SIMT}[args.algo]
+    cfg = attn.Cfg(args.tile_q, args.tile_k, args.tile_d, algo, args.deterministic)
+    dt_code = attn.ATTN_BF16 if w.bf16 else attn.ATTN_F32
+    tdtype = torch.bfloat16 if w.bf16 else torch.float32
+
+    # every rank draws its own batch: stream seed shifted by the rank (weak scaling)
+    wr = inputs.Workload(**{**w.__dict__, "seed": w.seed + 1000 * rank})
+    host = {}
+    for name, arr in wr.tensors().items():
+        t = torch.from_numpy(arr.reshape(w.batch, w.heads, w.n, w.d)).to(tdtype)
+        host[name] = t.pin_memory()
+    dev = {k: v.cuda(non_blocking=True) for k, v in host.items()}
+    mask = None
+    if w.mask != inputs.MASK_NONE:
+        mask = attn.Mask(kind=w.mask, block=w.block,
+                         block_mask=torch.from_numpy(bmask).cuda() if bmask is not None else None)
+    O = torch.empty_like(dev["Q"])
+    LSE = torch.empty((w.batch, w.heads, w.n), dtype=torch.float32, device="cuda")
+    dQ, dK, dV = (torch.empty_like(dev["Q"]) for _ in range(3))
+    ws_f = torch.empty(max(256, attn.attn_fwd_workspace_bytes(w.n, w.d, w.heads, w.batch, mask, dt_code, cfg)),
+                       dtype=torch.uint8, device="cuda")
+    ws_b = torch.empty(max(256, attn.attn_bwd_workspace_bytes(w.n, w.d, w.heads, w.batch, mask, dt_code, cfg)),
+                       dtype=torch.uint8, device="cuda")
+
+    def fwd():
+        attn.attn_fwd(dev["Q"], dev["K"], dev["V"], O, LSE, mask=mask, cfg=cfg, workspace=ws_f)
+
+    def bwd():
+        attn.attn_bwd(dev["Q"], dev["K"], dev["V"], O, dev["dO"], LSE, dQ, dK, dV, mask=mask, cfg=cfg, workspace=ws_b)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        fwd()
+        bwd()
+    barrier()
+    st = attn.attn_workspace_status(ws_b)
+    if st != attn.ATTN_OK:
+        raise SystemExit(f"kernel reported: {attn.status_str(st)}")
+
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    attn.attn_timing_enable(True)
+    attn.attn_timing_collect()
+    launches0 = attn.attn_kernel_launches()
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    kernel_ms: dict[str, list[float]] = {}
+    if rank == 0:
+        sampler.start()
+    barrier()
+    t_wall = time.perf_counter()
+    for s in range(args.steps):
+        ev[s][0].record()
+        fwd()
+        ev[s][1].record()
+        bwd()
+        ev[s][2].record()
+        if (s + 1) % 16 == 0 or s == args.steps - 1:   # the event pool holds 256 launches
+            for name, ms in attn.attn_timing_collect():
+                kernel_ms.setdefault(name, []).append(ms)
+    barrier()
+    wall_ms = (time.perf_counter() - t_wall) * 1e3
+    clocks = sampler.stop() if rank == 0 else None
+    launches = attn.attn_kernel_launches() - launches0
+    attn.attn_timing_enable(False)
+    fwd_ms = sum(ev[s][0].elapsed_time(ev[s][1]) for s in range(args.steps))
+    bwd_ms = sum(ev[s][1].elapsed_time(ev[s][2]) for s in range(args.steps))
+    step_ms = sum(ev[s][0].elapsed_time(ev[s][2]) for s in range(args.steps))
+    st = attn.attn_workspace_status(ws_b)
+    if st != attn.ATTN_OK or attn.attn_workspace_status(ws_f) != attn.ATTN_OK:
+        raise SystemExit("kernel reported a device-side timeout")
+
+    # ---- end to end through the public API with HOST buffers: H2D of Q, K, V, dO, forward,
+    # backward, D2H of dQ, dK, dV, every step
+    e2e = None
+    if not args.no_e2e:
+        out_host = [torch.empty_like(host["Q"]).pin_memory() for _ in range(3)]
+        e2e_steps = max(3, min(args.steps, 10))
+
+        def e2e_step():
+            for k in ("Q", "K", "V", "dO"):
+                dev[k].copy_(host[k], non_blocking=True)
+            fwd()
+            bwd()
+            for src, dst in zip((dQ, dK, dV), out_host):
+                dst.copy_(src, non_blocking=True)
+
+        e2e_step()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        e1.record()
+        barrier()
+        e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    ff, fb = flops(w, bmask)
+    red = max_over_ranks([fwd_ms, bwd_ms, step_ms, e2e_ms if not args.no_e2e else 0.0], world)
+    fwd_ms, bwd_ms, step_ms, e2e_ms = red
+    total = sum_over_ranks([fb, ff, float(launches)], world)
+    fb_all, ff_all, launches_all = total
+    value = fb_all * args.steps / (bwd_ms * 1e-3) / 1e12
+    peaks = load_peaks()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # dominant kernel: the one with the largest total time
+    tot = {k: sum(v) for k, v in kernel_ms.items()}
+    roofline = None
+    if tot:
+        top = max(tot, key=tot.get)
+        avg_ms = tot[top] / len(kernel_ms[top])
+        share = {k: round(v / sum(tot.values()), 4) for k, v in tot.items()}
+        if "bwd" in top and "preprocess" not in top:
+            # fraction of the backward's algorithmic FLOPs this kernel carries
+            names_bwd = [k for k in tot if "bwd" in k and "preprocess" not in k and "convert" not in k]
+            alg = fb if len(names_bwd) == 1 else fb * (0.8 if "dkdv" in top else 0.6)
+            note = ("algorithmic FLOPs of the five backward products" if len(names_bwd) == 1 else
+                    "this kernel's own products (the split backward recomputes S and dP in both kernels)")
+        else:
+            alg, note = ff, "algorithmic FLOPs of the two forward products"
+        ach = alg / (avg_ms * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "kernel": top, "achieved": ach, "peak": peaks["bf16_tflops_sustained"],
+                    "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"],
+                    "frac_of_burst_peak": ach / peaks["bf16_tflops"], "peak_source": peaks["source"] + " sustained",
+                    "avg_launch_ms": avg_ms, "launches_timed": len(kernel_ms[top]), "flops_per_launch": alg,
+                    "flops_note": note, "traffic": TRAFFIC.get((top, w.name)), "kernel_time_share": share}
+    line = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": step_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16" if w.bf16 else "f32", "data": "synthetic",
+        "config": {"workload": workload_name(w), "algo": args.algo, "tile_q": args.tile_q, "tile_k": args.tile_k,
+                   "tile_d": args.tile_d, "deterministic": args.deterministic,
+                   "step": "forward (O, LSE) + backward (D, dQ, dK, dV); value counts the backward only",
+                   "l2": "inputs (5 x %d MiB) larger than L2; no flush" % (w.batch * w.heads * w.n * w.d * 2 >> 20),
+                   "per_rank_batch": w.batch},
+        "fwd_tflops": ff_all * args.steps / (fwd_ms * 1e-3) / 1e12,
+        "fwd_ms": fwd_ms / args.steps, "bwd_ms": bwd_ms / args.steps, "wall_ms_per_step": wall_ms / args.steps,
+        "frac_of_sustained_peak": value / world / peaks["bf16_tflops_sustained"],
+        "clocks": clocks, "gpu_launches": int(launches_all),
+        "roofline": roofline,
+    }
+    if not args.no_e2e:
+        elem = 2 if w.bf16 else 4
+        per = w.batch * w.heads * w.n * w.d * elem
+        line["e2e"] = {"value": fb_all / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+                       "h2d_bytes_per_step": 4 * per, "d2h_bytes_per_step": 3 * per, "ms_per_step": e2e_ms,
+                       "note": "backward FLOPs / (H2D of Q,K,V,dO + forward + backward + D2H of dQ,dK,dV)"}
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(w, bmask)
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu
+# captures summarised under profiles/, keyed by (kernel, workload); absent = not measured
+# for the kernel as it stands.
+TRAFFIC: dict = {}
+
+
+if __name__ == "__main__":
+    main()

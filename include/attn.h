@@ -146,6 +146,20 @@ double attn_io_bound_sparse_elems(double z_input, double z_qk, double M);
 
 const char *attn_status_str(int status);
 
+/* ---- diagnostics (process-wide state; not thread-safe; off by default) ----
+ * attn_kernel_launches: kernels this library has launched since it was loaded.
+ * attn_timing_enable(1): from now on every kernel launch is bracketed by two CUDA
+ *   events recorded on the launching stream (a fixed pool of 256 launches; later
+ *   launches go untimed until collected).  attn_timing_enable(0) releases the pool.
+ * attn_timing_collect: synchronises on the recorded events, writes each launch's
+ *   device time in milliseconds to ms[] and a pointer to its static kernel name to
+ *   names[] (both host arrays of `max` entries), empties the pool and returns the
+ *   number of launches written.  This is how a caller obtains per-kernel times for
+ *   roofline arithmetic without a profiler. */
+unsigned long long attn_kernel_launches(void);
+attn_status attn_timing_enable(int on);
+int attn_timing_collect(float *ms /* host */, const char **names /* host */, int max);
+
 #ifdef __cplusplus
 }
 #endif

@@ -26,7 +26,8 @@ ATTN_ALGO_AUTO, ATTN_ALGO_FUSED, ATTN_ALGO_MATERIALIZED, ATTN_ALGO_SIMT = 0, 1, 
 EXPORTS = (
     "attn_fwd", "attn_bwd", "attn_bwd_preprocess", "attn_fwd_workspace_bytes", "attn_bwd_workspace_bytes",
     "attn_workspace_status", "attn_supported_cfgs", "attn_cfg_onchip_elems", "attn_io_bound_elems",
-    "attn_io_bound_sparse_elems", "attn_status_str",
+    "attn_io_bound_sparse_elems", "attn_status_str", "attn_kernel_launches", "attn_timing_enable",
+    "attn_timing_collect",
 )
 
 
@@ -106,6 +107,12 @@ def lib() -> ctypes.CDLL:
     L.attn_io_bound_elems.argtypes = [ctypes.c_double] * 3 + [ci]
     L.attn_io_bound_sparse_elems.restype = ctypes.c_double
     L.attn_io_bound_sparse_elems.argtypes = [ctypes.c_double] * 3
+    L.attn_kernel_launches.restype = ctypes.c_ulonglong
+    L.attn_kernel_launches.argtypes = []
+    L.attn_timing_enable.restype = ci
+    L.attn_timing_enable.argtypes = [ci]
+    L.attn_timing_collect.restype = ci
+    L.attn_timing_collect.argtypes = [ctypes.POINTER(cf), ctypes.POINTER(ctypes.c_char_p), ci]
     L.attn_status_str.restype = ctypes.c_char_p
     L.attn_status_str.argtypes = [ci]
     _lib = L
@@ -231,3 +238,21 @@ def attn_io_bound_elems(n, d, M, backward: bool) -> float:
 
 def attn_io_bound_sparse_elems(z_input, z_qk, M) -> float:
     return float(lib().attn_io_bound_sparse_elems(float(z_input), float(z_qk), float(M)))
+
+
+def attn_kernel_launches() -> int:
+    return int(lib().attn_kernel_launches())
+
+
+def attn_timing_enable(on: bool) -> None:
+    st = lib().attn_timing_enable(int(on))
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_timing_enable")
+
+
+def attn_timing_collect(max_entries: int = 256) -> list[tuple[str, float]]:
+    """[(kernel name, milliseconds), ...] for the launches since the last collect."""
+    ms = (ctypes.c_float * max_entries)()
+    names = (ctypes.c_char_p * max_entries)()
+    cnt = lib().attn_timing_collect(ms, names, max_entries)
+    return [(names[i].decode(), float(ms[i])) for i in range(cnt)]

@@ -164,6 +164,40 @@ attn_status fill_problem(Problem &p, const Args &a, int backward, float scale, v
 }  // namespace
 }  // namespace attn
 
+namespace attn {
+namespace {
+constexpr int kTimingPool = 256;
+struct Timing {
+    bool on = false;
+    int count = 0;
+    bool open = false;
+    cudaEvent_t ev[2 * kTimingPool];
+    const char *names[kTimingPool];
+} g_timing;
+unsigned long long g_launches = 0;
+}  // namespace
+
+void launch_begin(const char *name, cudaStream_t s)
+{
+    ++g_launches;
+    g_timing.open = false;
+    if (g_timing.on && g_timing.count < kTimingPool) {
+        g_timing.names[g_timing.count] = name;
+        cudaEventRecord(g_timing.ev[2 * g_timing.count], s);
+        g_timing.open = true;
+    }
+}
+
+void launch_end(cudaStream_t s)
+{
+    if (g_timing.open) {
+        cudaEventRecord(g_timing.ev[2 * g_timing.count + 1], s);
+        ++g_timing.count;
+        g_timing.open = false;
+    }
+}
+}  // namespace attn
+
 using namespace attn;
 
 extern "C" {
@@ -292,6 +326,41 @@ double attn_io_bound_sparse_elems(double z_input, double z_qk, double M)
     const double large = z_input * z_input / M;
     const double small = z_input * sqrt(z_qk) / sqrt(M);
     return large < small ? large : small;
+}
+
+unsigned long long attn_kernel_launches(void) { return g_launches; }
+
+attn_status attn_timing_enable(int on)
+{
+    if (on && !g_timing.on) {
+        for (int i = 0; i < 2 * kTimingPool; ++i)
+            if (cudaEventCreate(&g_timing.ev[i]) != cudaSuccess) return ATTN_ERR_LAUNCH;
+        g_timing.count = 0;
+        g_timing.on = true;
+    } else if (!on && g_timing.on) {
+        for (int i = 0; i < 2 * kTimingPool; ++i) cudaEventDestroy(g_timing.ev[i]);
+        g_timing.on = false;
+        g_timing.count = 0;
+    }
+    return ATTN_OK;
+}
+
+int attn_timing_collect(float *ms, const char **names, int max)
+{
+    if (!g_timing.on) return 0;
+    int out = 0;
+    for (int i = 0; i < g_timing.count; ++i) {
+        float t = 0.f;
+        if (cudaEventSynchronize(g_timing.ev[2 * i + 1]) != cudaSuccess) break;
+        if (cudaEventElapsedTime(&t, g_timing.ev[2 * i], g_timing.ev[2 * i + 1]) != cudaSuccess) break;
+        if (out < max) {
+            if (ms) ms[out] = t;
+            if (names) names[out] = g_timing.names[i];
+            ++out;
+        }
+    }
+    g_timing.count = 0;
+    return out;
 }
 
 const char *attn_status_str(int status)

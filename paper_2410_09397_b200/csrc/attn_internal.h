@@ -38,6 +38,10 @@ struct WorkspaceLayout {
     int mat_heads;
 };
 
+// Every kernel launch goes between these two calls (launch counter + optional event timing).
+void launch_begin(const char *name, cudaStream_t s);
+void launch_end(cudaStream_t s);
+
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // SIMT fp32 path (attn_simt.cu)

@@ -476,11 +476,13 @@ SimtArgs make_args(const Problem &p)
 }
 
 template <typename K>
-attn_status launch(K kernel, dim3 grid, size_t smem, cudaStream_t s, const SimtArgs &a)
+attn_status launch(const char *name, K kernel, dim3 grid, size_t smem, cudaStream_t s, const SimtArgs &a)
 {
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return ATTN_ERR_LAUNCH;
+    launch_begin(name, s);
     kernel<<<grid, NT, smem, s>>>(a);
+    launch_end(s);
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_LAUNCH;
 }
 
@@ -490,9 +492,9 @@ attn_status fwd_t(const Problem &p)
     const SimtArgs a = make_args(p);
     const dim3 grid((p.n + TS - 1) / TS, (unsigned)p.BH);
     const size_t smem = 3 * TS * LD * sizeof(float);
-    if (p.d <= 64) return launch(simt_fwd_kernel<T, 1>, grid, smem, p.stream, a);
-    if (p.d <= 128) return launch(simt_fwd_kernel<T, 2>, grid, smem, p.stream, a);
-    return launch(simt_fwd_kernel<T, 4>, grid, smem, p.stream, a);
+    if (p.d <= 64) return launch("simt_fwd", simt_fwd_kernel<T, 1>, grid, smem, p.stream, a);
+    if (p.d <= 128) return launch("simt_fwd", simt_fwd_kernel<T, 2>, grid, smem, p.stream, a);
+    return launch("simt_fwd", simt_fwd_kernel<T, 4>, grid, smem, p.stream, a);
 }
 
 template <typename T>
@@ -503,14 +505,14 @@ attn_status bwd_t(const Problem &p)
     const size_t smem3 = 3 * TS * LD * sizeof(float), smem4 = 4 * TS * LD * sizeof(float);
     attn_status st;
     if (p.d <= 64) {
-        st = launch(simt_bwd_dkdv_kernel<T, 1, 1>, grid, smem4, p.stream, a);
-        if (st == ATTN_OK) st = launch(simt_bwd_dq_kernel<T, 1>, grid, smem3, p.stream, a);
+        st = launch("simt_bwd_dkdv", simt_bwd_dkdv_kernel<T, 1, 1>, grid, smem4, p.stream, a);
+        if (st == ATTN_OK) st = launch("simt_bwd_dq", simt_bwd_dq_kernel<T, 1>, grid, smem3, p.stream, a);
     } else if (p.d <= 128) {
-        st = launch(simt_bwd_dkdv_kernel<T, 2, 2>, grid, smem4, p.stream, a);
-        if (st == ATTN_OK) st = launch(simt_bwd_dq_kernel<T, 2>, grid, smem3, p.stream, a);
+        st = launch("simt_bwd_dkdv", simt_bwd_dkdv_kernel<T, 2, 2>, grid, smem4, p.stream, a);
+        if (st == ATTN_OK) st = launch("simt_bwd_dq", simt_bwd_dq_kernel<T, 2>, grid, smem3, p.stream, a);
     } else {
-        st = launch(simt_bwd_dkdv_kernel<T, 4, 2>, dim3(grid.x, grid.y, 2), smem4, p.stream, a);
-        if (st == ATTN_OK) st = launch(simt_bwd_dq_kernel<T, 4>, grid, smem3, p.stream, a);
+        st = launch("simt_bwd_dkdv", simt_bwd_dkdv_kernel<T, 4, 2>, dim3(grid.x, grid.y, 2), smem4, p.stream, a);
+        if (st == ATTN_OK) st = launch("simt_bwd_dq", simt_bwd_dq_kernel<T, 4>, grid, smem3, p.stream, a);
     }
     return st;
 }
@@ -542,20 +544,24 @@ attn_status preprocess_D(const void *O, const void *dO, float *D, size_t rows, i
     size_t blocks = (warps + 7) / 8;
     const size_t cap = 148 * 8 * 4;  // a few resident CTAs per SM, grid-stride beyond that
     if (blocks > cap) blocks = cap;
+    launch_begin("bwd_preprocess_D", s);
     if (dt == ATTN_F32)
         preprocess_kernel<float><<<(unsigned)blocks, 256, 0, s>>>((const float *)O, (const float *)dO, D, rows, d,
                                                                 lanes);
     else
         preprocess_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, s>>>((const __nv_bfloat16 *)O,
                                                                          (const __nv_bfloat16 *)dO, D, rows, d, lanes);
+    launch_end(s);
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_LAUNCH;
 }
 
 attn_status build_block_index(const Problem &p)
 {
     if (p.mask_kind != ATTN_MASK_BLOCK_SPARSE || !p.row_ptr) return ATTN_OK;
+    launch_begin("block_index", p.stream);
     block_index_kernel<<<dim3(p.nb, p.mask_heads), 64, 0, p.stream>>>(p.block_mask, p.nb, p.row_ptr, p.col_idx,
                                                                       p.col_ptr, p.row_idx);
+    launch_end(p.stream);
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_LAUNCH;
 }
 
