@@ -56,5 +56,9 @@ attn_status tc_bwd(const Problem &p);
 attn_status mat_bwd(const Problem &p);
 bool tc_cfg_supported(int d, const attn_cfg &cfg, int backward);
 size_t tc_cfg_onchip_bytes(int d, const attn_cfg &cfg, int backward);
+size_t fwd_smem_bytes(int d);
+size_t bwd_smem_bytes(int d);
+bool mat_cfg_supported(int d, const attn_cfg &cfg);
+size_t mat_onchip_bytes(int d, const attn_cfg &cfg);
 
 }  // namespace attn

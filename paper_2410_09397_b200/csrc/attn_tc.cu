@@ -1,10 +1,37 @@
-// Tensor-core (tcgen05 / TMEM / TMA) path -- placeholder until the kernels land.
+// Which tile configurations the tensor-core algorithms accept, and how much on-chip
+// memory (shared memory + tensor memory) a CTA of each holds.
 #include "attn_internal.h"
 
 namespace attn {
-bool tc_cfg_supported(int, const attn_cfg &, int) { return false; }
-size_t tc_cfg_onchip_bytes(int, const attn_cfg &, int) { return 0; }
-attn_status tc_fwd(const Problem &) { return ATTN_ERR_TILE; }
-attn_status tc_bwd(const Problem &) { return ATTN_ERR_TILE; }
-attn_status mat_bwd(const Problem &) { return ATTN_ERR_TILE; }
+
+// Fused forward: 128 queries x (128 keys for d <= 128, 64 keys for d = 256).
+// Fused backward: 128 x 128 for d = 64, 128 (at d = 256 the dK and dV accumulators alone
+// would fill tensor memory; that case belongs to the materialised algorithm).
+bool tc_cfg_supported(int d, const attn_cfg &c, int backward)
+{
+    if (d != 64 && d != 128 && d != 256) return false;
+    if (c.algo == ATTN_ALGO_FUSED) {
+        if (c.tile_d != 0 && c.tile_d != d) return false;
+        if (c.tile_q != 0 && c.tile_q != 128) return false;
+        if (backward) {
+            if (d == 256) return false;
+            if (c.deterministic) return false;   // the fused backward reduces dQ with floating-point atomics
+            return c.tile_k == 0 || c.tile_k == 128;
+        }
+        const int tk = d == 256 ? 64 : 128;
+        return c.tile_k == 0 || c.tile_k == tk;
+    }
+    if (c.algo == ATTN_ALGO_MATERIALIZED) return backward && mat_cfg_supported(d, c);
+    return false;
+}
+
+size_t tc_cfg_onchip_bytes(int d, const attn_cfg &c, int backward)
+{
+    if (!tc_cfg_supported(d, c, backward)) return 0;
+    if (c.algo == ATTN_ALGO_MATERIALIZED) return mat_onchip_bytes(d, c);
+    // tensor memory: 128 lanes x 4 bytes per column
+    if (backward) return bwd_smem_bytes(d) + (size_t)(256 + 2 * d) * 128 * 4;
+    return fwd_smem_bytes(d) + (size_t)(256 + d) * 128 * 4;
+}
+
 }  // namespace attn

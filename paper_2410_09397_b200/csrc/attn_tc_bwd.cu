@@ -1,0 +1,440 @@
+// Fused backward for bf16 on the 5th-generation tensor cores (large-cache regime of
+// Appendix D: no n x n matrix ever leaves the SM).
+//
+// The loops of the paper's phase-2 algorithm are swapped: a CTA owns one tile of 128
+// KEYS j (K_j, V_j stay in shared memory, dK_j and dV_j stay in tensor memory) and walks
+// the kept QUERY tiles i.  Per (i, j) pair, with everything transposed so that the
+// tensor-memory lane is the key index:
+//
+//   S^T  = K_j Q_i^T                         (tcgen05.mma, both operands K-major smem)
+//   dP^T = V_j dO_i^T                        (same)
+//   P^T  = exp2(S^T * scale*log2e - LSE_i*log2e)        (256 threads, fp32)
+//   dS^T = P^T o (dP^T - D_i)                           (Definition B.9, p = f o q - diag(v) f)
+//   dV_j += P^T  dO_i      A = P^T  in tensor memory (bf16), B = dO_i MN-major smem
+//   dK_j += dS^T Q_i       A = dS^T K-major smem,            B = Q_i  MN-major smem
+//   dQ_i += dS K_j         computed as dQ^T = K_j^T dS^T for d = 128 (so that the fp32
+//                          reductions into global memory are coalesced), as dS K_j for d = 64
+//
+// dQ partial tiles are added into an fp32 accumulator in the workspace with
+// red.global.add (the one place where summation order is not fixed); a small kernel
+// converts it to bf16 at the end.  Tensor memory (512 columns): S^T / P^T 128,
+// dP^T then dQ 128, dV d, dK d.
+//
+// Roles: warps 0-7 = two warpgroups that split the 128 query columns of each tile
+// between them (softmax, dS, dQ reduction, epilogue); warp 8 lane 0 = TMA producer and
+// MMA issuer.  All waits are bounded (tc_common.cuh).
+#include "attn_internal.h"
+#include "tc_common.cuh"
+
+namespace attn {
+namespace {
+
+using namespace tc;
+
+constexpr int TQ = 128, TK = 128;
+constexpr int kSoftmaxThreads = 256;
+constexpr int kThreads = kSoftmaxThreads + 32;
+constexpr uint32_t SLAB = 128 * 128;   // bytes of one [128 rows][64 bf16] slab
+
+struct BwdArgs {
+    const float *LSE, *D;
+    float *dQ_acc;
+    __nv_bfloat16 *dK, *dV;
+    int n, BH;
+    int mask_kind, block, nb, mask_heads;
+    const int *col_ptr, *row_idx;   // block-CSC of the mask
+    float scale;
+    uint32_t *status;
+};
+
+template <int HD>
+struct BwdSmem {
+    static constexpr uint32_t kSlabs = HD / 64;
+    static constexpr uint32_t kTile = kSlabs * SLAB;      // one [128][HD] bf16 tile
+    static constexpr uint32_t oK = 0;
+    static constexpr uint32_t oV = oK + kTile;
+    static constexpr uint32_t oQ = oV + kTile;            // 2 stages
+    static constexpr uint32_t odO = oQ + 2 * kTile;       // 2 stages
+    static constexpr uint32_t odS = odO + 2 * kTile;      // [128 keys][128 queries] bf16, 2 slabs
+    static constexpr uint32_t oLSE = odS + 2 * SLAB;      // 2 stages x 128 floats
+    static constexpr uint32_t oD = oLSE + 2 * 128 * 4;
+    static constexpr uint32_t oBar = oD + 2 * 128 * 4;    // mbarriers (8 bytes each)
+    static constexpr uint32_t oMisc = oBar + 16 * 8;      // tmem base, abort flag
+    static constexpr uint32_t kBytes = oMisc + 64;
+    static_assert(kBytes <= 227 * 1024, "shared memory budget");
+};
+
+enum { BAR_KV = 0, BAR_QFULL = 1, BAR_QEMPTY = 3, BAR_S = 5, BAR_P = 6, BAR_DQ = 7, BAR_DQDONE = 8 };
+
+struct TileIter {
+    // Enumerates the query tiles a key tile jt has to visit.
+    int kind, n, jt, sub, raw;
+    const int *rows;   // block rows kept in this block column
+    __device__ TileIter(const BwdArgs &a, int jt_, long bh) : kind(a.mask_kind), n(a.n), jt(jt_), sub(1), raw(0), rows(nullptr)
+    {
+        const int nt = (n + TQ - 1) / TQ;
+        if (kind == ATTN_MASK_NONE) raw = nt;
+        else if (kind == ATTN_MASK_CAUSAL) raw = nt - jt;
+        else {
+            sub = a.block / TQ;
+            const int J = jt / sub;
+            const long mh = a.mask_heads == 1 ? 0 : bh;
+            const int *cp = a.col_ptr + mh * 2 * a.nb + 2 * J;
+            rows = a.row_idx + mh * (long)a.nb * a.nb + cp[0];
+            raw = (cp[1] - cp[0]) * sub;
+        }
+    }
+    // query tile of raw index idx, or -1 if that tile lies beyond n
+    __device__ int tile(int idx) const
+    {
+        int it;
+        if (kind == ATTN_MASK_NONE) it = idx;
+        else if (kind == ATTN_MASK_CAUSAL) it = jt + idx;
+        else it = rows[idx / sub] * sub + idx % sub;
+        return it * TQ < n ? it : -1;
+    }
+};
+
+__device__ __forceinline__ void bulk_load_1d(void *dst, const void *src, uint32_t bytes, uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void named_bar_sync(int id, int count)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+__device__ __forceinline__ void red_add_f32(float *p, float v)
+{
+    asm volatile("red.global.add.f32 [%0], %1;" ::"l"(p), "f"(v) : "memory");
+}
+__device__ __forceinline__ void red_add_v4(float *p, float a, float b, float c, float d)
+{
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+
+template <int HD>
+__global__ void __launch_bounds__(kThreads, 1)
+tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mK,
+              const __grid_constant__ CUtensorMap mV, const __grid_constant__ CUtensorMap mdO, const BwdArgs a)
+{
+    using L = BwdSmem<HD>;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::oBar);
+    uint32_t *tmem_base_s = reinterpret_cast<uint32_t *>(smem + L::oMisc);
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(smem + L::oMisc + 4);
+    const Abort ab{abort_flag, a.status};
+
+    const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
+    const int jt = blockIdx.x;
+    const long bh = blockIdx.y;
+    const int j0 = jt * TK, n = a.n;
+
+    if ((smem_u32(smem) & 1023u) != 0) {   // operand tiles need 1024-byte alignment
+        if (tid == 0) atomicExch(a.status, 9u);
+        return;
+    }
+    if (tid == 0) {
+        *abort_flag = 0;
+        mbar_init(&bars[BAR_KV], 1);
+        mbar_init(&bars[BAR_QFULL], 1); mbar_init(&bars[BAR_QFULL + 1], 1);
+        mbar_init(&bars[BAR_QEMPTY], 1); mbar_init(&bars[BAR_QEMPTY + 1], 1);
+        mbar_init(&bars[BAR_S], 1);
+        mbar_init(&bars[BAR_P], kSoftmaxThreads);
+        mbar_init(&bars[BAR_DQ], 1);
+        mbar_init(&bars[BAR_DQDONE], kSoftmaxThreads);
+        fence_barrier_init();
+        prefetch_tensormap(&mQ); prefetch_tensormap(&mK); prefetch_tensormap(&mV); prefetch_tensormap(&mdO);
+    }
+    if (warp == 0) tmem_alloc(tmem_base_s, 512);
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tm = *tmem_base_s;
+    const uint32_t T_S = tm, T_dP = tm + 128, T_dV = tm + 256, T_dK = tm + 256 + HD;
+
+    const TileIter iter(a, jt, bh);
+    const float sl2 = a.scale * 1.4426950408889634f;
+
+    if (warp == 8) {
+        // ------------------------------------------------------------ producer + MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = idesc_bf16(128, 128, 0, 0);       // S^T, dP^T
+            constexpr uint32_t idesc_dv = idesc_bf16(128, HD, 0, 1);       // dV (A tmem), dK (A K-major smem)
+            constexpr uint32_t idesc_dq = HD == 128 ? idesc_bf16(128, 128, 1, 1) : idesc_bf16(128, HD, 1, 1);
+            const uint32_t sK = smem_u32(smem + L::oK), sV = smem_u32(smem + L::oV), sdS = smem_u32(smem + L::odS);
+            auto issue_load = [&](int it, int s) {
+                const int i0 = it * TQ;
+                const uint32_t rows = min(TQ, n - i0);
+                uint64_t *bar = &bars[BAR_QFULL + s];
+                mbar_expect_tx(bar, 2 * L::kTile + 2 * rows * 4);
+#pragma unroll
+                for (uint32_t sl = 0; sl < L::kSlabs; ++sl) {
+                    tma_load_3d(smem + L::oQ + s * L::kTile + sl * SLAB, &mQ, bar, sl * 64, i0, (int)bh);
+                    tma_load_3d(smem + L::odO + s * L::kTile + sl * SLAB, &mdO, bar, sl * 64, i0, (int)bh);
+                }
+                bulk_load_1d(smem + L::oLSE + s * 512, a.LSE + bh * n + i0, rows * 4, bar);
+                bulk_load_1d(smem + L::oD + s * 512, a.D + bh * n + i0, rows * 4, bar);
+            };
+            mbar_expect_tx(&bars[BAR_KV], 2 * L::kTile);
+#pragma unroll
+            for (uint32_t sl = 0; sl < L::kSlabs; ++sl) {
+                tma_load_3d(smem + L::oK + sl * SLAB, &mK, &bars[BAR_KV], sl * 64, j0, (int)bh);
+                tma_load_3d(smem + L::oV + sl * SLAB, &mV, &bars[BAR_KV], sl * 64, j0, (int)bh);
+            }
+            // first valid tile
+            int idx = 0, it = -1;
+            while (idx < iter.raw && (it = iter.tile(idx)) < 0) ++idx;
+            if (it >= 0) issue_load(it, 0);
+            int k = 0;   // count of processed tiles
+            while (idx < iter.raw) {
+                const int s = k & 1;
+                // look ahead for the next valid tile and prefetch it
+                int nidx = idx + 1, nit = -1;
+                while (nidx < iter.raw && (nit = iter.tile(nidx)) < 0) ++nidx;
+                if (nit >= 0) {
+                    if (k >= 1) mbar_wait(&bars[BAR_QEMPTY + (s ^ 1)], ((k - 1) >> 1) & 1, ab);
+                    issue_load(nit, s ^ 1);
+                }
+                mbar_wait(&bars[BAR_QFULL + s], (k >> 1) & 1, ab);
+                if (k == 0) mbar_wait(&bars[BAR_KV], 0, ab);
+                tcgen05_fence_after();
+                const uint32_t sQ = smem_u32(smem + L::oQ + s * L::kTile), sdO = smem_u32(smem + L::odO + s * L::kTile);
+                // S^T = K_j Q_i^T
+#pragma unroll
+                for (int kk = 0; kk < HD / 16; ++kk) {
+                    const uint32_t off = (kk / 4) * SLAB + (kk % 4) * 32;
+                    mma_ss(T_S, smem_desc_kmajor(sK + off), smem_desc_kmajor(sQ + off), idesc_s, kk > 0);
+                }
+                if (k > 0) {
+                    mbar_wait(&bars[BAR_DQDONE], (k - 1) & 1, ab);
+                    tcgen05_fence_after();
+                }
+                // dP^T = V_j dO_i^T
+#pragma unroll
+                for (int kk = 0; kk < HD / 16; ++kk) {
+                    const uint32_t off = (kk / 4) * SLAB + (kk % 4) * 32;
+                    mma_ss(T_dP, smem_desc_kmajor(sV + off), smem_desc_kmajor(sdO + off), idesc_s, kk > 0);
+                }
+                mma_commit(&bars[BAR_S]);
+                mbar_wait(&bars[BAR_P], k & 1, ab);
+                tcgen05_fence_after();
+                // dV += P^T dO_i ; dK += dS^T Q_i   (contraction over the 128 queries of the tile)
+#pragma unroll
+                for (int kk = 0; kk < TQ / 16; ++kk)
+                    mma_ts(T_dV, T_S + kk * 8, smem_desc_mnmajor(sdO + kk * 2048, SLAB), idesc_dv, (k > 0) || (kk > 0));
+#pragma unroll
+                for (int kk = 0; kk < TQ / 16; ++kk) {
+                    const uint32_t offa = (kk / 4) * SLAB + (kk % 4) * 32;
+                    mma_ss(T_dK, smem_desc_kmajor(sdS + offa), smem_desc_mnmajor(sQ + kk * 2048, SLAB), idesc_dv,
+                           (k > 0) || (kk > 0));
+                }
+                // dQ tile (contraction over the 128 keys of this CTA)
+#pragma unroll
+                for (int kk = 0; kk < TK / 16; ++kk) {
+                    if (HD == 128)   // dQ^T = K_j^T dS^T : A = K_j MN-major, B = dS^T MN-major
+                        mma_ss(T_dP, smem_desc_mnmajor(sK + kk * 2048, SLAB), smem_desc_mnmajor(sdS + kk * 2048, SLAB),
+                               idesc_dq, kk > 0);
+                    else             // dQ = dS K_j : A = dS^T read MN-major, B = K_j MN-major
+                        mma_ss(T_dP, smem_desc_mnmajor(sdS + kk * 2048, SLAB), smem_desc_mnmajor(sK + kk * 2048, SLAB),
+                               idesc_dq, kk > 0);
+                }
+                mma_commit(&bars[BAR_DQ]);
+                mma_commit(&bars[BAR_QEMPTY + s]);
+                ++k;
+                idx = nidx;
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ softmax / dS / dQ reduction warpgroups
+        const int wg = warp / 4;                       // which half of the query columns
+        const int row = (warp % 4) * 32 + lane;        // tensor-memory lane = key row inside the tile
+        const uint32_t lane_addr = (uint32_t)((warp % 4) * 32) << 16;
+        const int jg = j0 + row;
+        int k = 0;
+        for (int idx = 0; idx < iter.raw; ++idx) {
+            const int it = iter.tile(idx);
+            if (it < 0) continue;
+            const int s = k & 1, i0 = it * TQ;
+            const float *sLSE = reinterpret_cast<const float *>(smem + L::oLSE + s * 512);
+            const float *sD = reinterpret_cast<const float *>(smem + L::oD + s * 512);
+            mbar_wait(&bars[BAR_QFULL + s], (k >> 1) & 1, ab);   // LSE_i, D_i visible
+            mbar_wait(&bars[BAR_S], k & 1, ab);
+            tcgen05_fence_after();
+            const bool diag = a.mask_kind == ATTN_MASK_CAUSAL && it == jt;
+            uint32_t ppack[32];
+#pragma unroll
+            for (int ch = 0; ch < 2; ++ch) {
+                const int c0 = wg * 64 + ch * 32;
+                uint32_t sv[32], pv[32];
+                tmem_ld32(T_S + lane_addr + c0, sv);
+                tmem_ld32(T_dP + lane_addr + c0, pv);
+                tmem_wait_ld();
+                uint32_t dsp[16];
+#pragma unroll
+                for (int e = 0; e < 32; e += 2) {
+                    float p[2], ds[2];
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        const int il = c0 + e + u, ig = i0 + il;
+                        const float lse = sLSE[il];
+                        const bool ok = ig < n && jg < n && lse != -INFINITY && (!diag || jg <= ig);
+                        const float x = exp2f(__uint_as_float(sv[e + u]) * sl2 - lse * 1.4426950408889634f);
+                        p[u] = ok ? x : 0.f;
+                        ds[u] = ok ? p[u] * (__uint_as_float(pv[e + u]) - sD[il]) : 0.f;
+                    }
+                    ppack[ch * 16 + e / 2] = pack_bf16(p[0], p[1]);
+                    dsp[e / 2] = pack_bf16(ds[0], ds[1]);
+                }
+                // dS^T[j][i] into shared memory, 128-byte-swizzled slab wg (queries 64 wg .. 64 wg + 63)
+                uint8_t *slab = smem + L::odS + wg * SLAB;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const uint32_t col = ch * 32 + q * 8;
+                    *reinterpret_cast<uint4 *>(slab + sw128_offset(row, col)) =
+                        make_uint4(dsp[q * 4], dsp[q * 4 + 1], dsp[q * 4 + 2], dsp[q * 4 + 3]);
+                }
+            }
+            // every thread has finished reading S^T before anyone overwrites it with P^T
+            named_bar_sync(1, kSoftmaxThreads);
+            tmem_st32(T_S + lane_addr + wg * 32, ppack);
+            tmem_wait_st();
+            fence_proxy_async_smem();
+            tcgen05_fence_before();
+            mbar_arrive(&bars[BAR_P]);
+
+            // dQ tile: read out of tensor memory and reduce into the fp32 accumulator
+            mbar_wait(&bars[BAR_DQ], k & 1, ab);
+            tcgen05_fence_after();
+            if (HD == 128) {
+                // lanes = head-dimension index c, columns = queries
+                float *base = a.dQ_acc + ((size_t)bh * n + i0) * HD + row;
+#pragma unroll
+                for (int ch = 0; ch < 2; ++ch) {
+                    const int c0 = wg * 64 + ch * 32;
+                    uint32_t v[32];
+                    tmem_ld32(T_dP + lane_addr + c0, v);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        if (i0 + c0 + e < n) red_add_f32(base + (size_t)(c0 + e) * HD, __uint_as_float(v[e]) * a.scale);
+                }
+            } else {
+                // lanes = queries, columns = head-dimension index
+                const int c0 = wg * (HD / 2);
+                uint32_t v[32];
+                tmem_ld32(T_dP + lane_addr + c0, v);
+                tmem_wait_ld();
+                if (i0 + row < n) {
+                    float *base = a.dQ_acc + ((size_t)bh * n + i0 + row) * HD + c0;
+#pragma unroll
+                    for (int e = 0; e < HD / 2; e += 4)
+                        red_add_v4(base + e, __uint_as_float(v[e]) * a.scale, __uint_as_float(v[e + 1]) * a.scale,
+                                   __uint_as_float(v[e + 2]) * a.scale, __uint_as_float(v[e + 3]) * a.scale);
+                }
+            }
+            tcgen05_fence_before();
+            mbar_arrive(&bars[BAR_DQDONE]);
+            ++k;
+        }
+        // ------------------------------------------------------------ epilogue: dV_j, dK_j
+        // (the last BAR_DQ phase also covers the last dV / dK accumulation)
+        {
+            constexpr int HALF = HD / 2;
+            const int jc = jg < n ? jg : 0;   // rows past n take part in the warp-wide loads but store nothing
+            __nv_bfloat16 *pv = a.dV + ((size_t)bh * n + jc) * HD + wg * HALF;
+            __nv_bfloat16 *pk = a.dK + ((size_t)bh * n + jc) * HD + wg * HALF;
+#pragma unroll
+            for (int c = 0; c < HALF; c += 32) {
+                uint32_t v[32], w[32];
+                if (k > 0) {
+                    tmem_ld32(T_dV + lane_addr + wg * HALF + c, v);
+                    tmem_ld32(T_dK + lane_addr + wg * HALF + c, w);
+                    tmem_wait_ld();
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) v[e] = w[e] = 0u;
+                }
+                if (jg < n) {
+#pragma unroll
+                    for (int e = 0; e < 32; e += 8) {
+                        uint4 ov, ok;
+                        ov.x = pack_bf16(__uint_as_float(v[e]), __uint_as_float(v[e + 1]));
+                        ov.y = pack_bf16(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
+                        ov.z = pack_bf16(__uint_as_float(v[e + 4]), __uint_as_float(v[e + 5]));
+                        ov.w = pack_bf16(__uint_as_float(v[e + 6]), __uint_as_float(v[e + 7]));
+                        ok.x = pack_bf16(__uint_as_float(w[e]) * a.scale, __uint_as_float(w[e + 1]) * a.scale);
+                        ok.y = pack_bf16(__uint_as_float(w[e + 2]) * a.scale, __uint_as_float(w[e + 3]) * a.scale);
+                        ok.z = pack_bf16(__uint_as_float(w[e + 4]) * a.scale, __uint_as_float(w[e + 5]) * a.scale);
+                        ok.w = pack_bf16(__uint_as_float(w[e + 6]) * a.scale, __uint_as_float(w[e + 7]) * a.scale);
+                        *reinterpret_cast<uint4 *>(pv + c + e) = ov;
+                        *reinterpret_cast<uint4 *>(pk + c + e) = ok;
+                    }
+                }
+            }
+        }
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tm, 512);
+}
+
+// fp32 accumulator -> bf16 dQ
+__global__ void __launch_bounds__(256) dq_convert_kernel(const float4 *__restrict__ acc, uint2 *__restrict__ out, size_t n4)
+{
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x) {
+        const float4 v = acc[i];
+        out[i] = make_uint2(pack_bf16(v.x, v.y), pack_bf16(v.z, v.w));
+    }
+}
+
+template <int HD>
+attn_status launch_bwd(const Problem &p)
+{
+    using L = BwdSmem<HD>;
+    CUtensorMap mQ, mK, mV, mdO;
+    const uint64_t BH = (uint64_t)p.BH;
+    if (!make_tmap_bf16_3d(&mQ, p.Q, HD, p.n, BH, 128) || !make_tmap_bf16_3d(&mK, p.K, HD, p.n, BH, 128) ||
+        !make_tmap_bf16_3d(&mV, p.V, HD, p.n, BH, 128) || !make_tmap_bf16_3d(&mdO, p.dO, HD, p.n, BH, 128))
+        return ATTN_ERR_LAUNCH;
+    BwdArgs a{};
+    a.LSE = p.LSE; a.D = p.D; a.dQ_acc = p.dQ_acc;
+    a.dK = (__nv_bfloat16 *)p.dK; a.dV = (__nv_bfloat16 *)p.dV;
+    a.n = p.n; a.BH = (int)p.BH;
+    a.mask_kind = p.mask_kind; a.block = p.block; a.nb = p.nb; a.mask_heads = p.mask_heads;
+    a.col_ptr = p.col_ptr; a.row_idx = p.row_idx;
+    a.scale = p.scale;
+    a.status = p.status;
+    auto kernel = tc_bwd_kernel<HD>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::kBytes) != cudaSuccess)
+        return ATTN_ERR_LAUNCH;
+    const size_t acc_elems = (size_t)p.BH * p.n * HD;
+    if (cudaMemsetAsync(p.dQ_acc, 0, acc_elems * sizeof(float), p.stream) != cudaSuccess) return ATTN_ERR_LAUNCH;
+    const dim3 grid((p.n + TK - 1) / TK, (unsigned)p.BH);
+    launch_begin("tc_bwd_fused", p.stream);
+    kernel<<<grid, kThreads, L::kBytes, p.stream>>>(mQ, mK, mV, mdO, a);
+    launch_end(p.stream);
+    if (cudaGetLastError() != cudaSuccess) return ATTN_ERR_LAUNCH;
+    const size_t n4 = acc_elems / 4;
+    const unsigned blocks = (unsigned)((n4 + 255) / 256 < 148 * 16 ? (n4 + 255) / 256 : 148 * 16);
+    launch_begin("bwd_dq_convert", p.stream);
+    dq_convert_kernel<<<blocks, 256, 0, p.stream>>>((const float4 *)p.dQ_acc, (uint2 *)p.dQ, n4);
+    launch_end(p.stream);
+    return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_LAUNCH;
+}
+
+}  // namespace
+
+size_t bwd_smem_bytes(int d) { return d == 64 ? BwdSmem<64>::kBytes : d == 128 ? BwdSmem<128>::kBytes : 0; }
+
+attn_status tc_bwd(const Problem &p)
+{
+    attn_status st = preprocess_D(p.O, p.dO, p.D, (size_t)p.BH * p.n, p.d, p.dt, p.stream);
+    if (st != ATTN_OK) return st;
+    if (p.d == 64) return launch_bwd<64>(p);
+    if (p.d == 128) return launch_bwd<128>(p);
+    return ATTN_ERR_TILE;
+}
+
+}  // namespace attn

@@ -1,0 +1,372 @@
+// Fused forward for bf16 on the 5th-generation tensor cores: O = softmax(scale Q K^T) V
+// and LSE, never writing a score tile to device memory (Definition 3.1; large-cache
+// tiling: row block of 128 queries stays on chip, key/value blocks stream through).
+//
+// A CTA owns one tile of 128 queries (tensor-memory lane = query row) and walks the
+// kept key tiles j of TKF keys (128 for d <= 128, 64 for d = 256):
+//
+//   S   = Q_i K_j^T                 tcgen05.mma, operands K-major in shared memory,
+//                                   two S buffers in tensor memory so that S(j+1) is
+//                                   computed while the softmax of S(j) runs
+//   m, l running row maximum / row sum in the exp2 domain; the reference maximum is
+//       only moved (and O rescaled in tensor memory) when the tile maximum exceeds it
+//       by more than 2^8 -- the final LSE does not depend on which reference was used
+//   P   = exp2(S * scale*log2e - m)  -> bf16, written over S in tensor memory
+//   O  += P V_j                      A = P from tensor memory, B = V_j MN-major
+//
+// Roles: warps 0-7 = two warpgroups that split the key columns of every tile (row
+// maxima are exchanged through shared memory), warp 8 lane 0 = MMA issuer, warp 9
+// lane 0 = TMA producer.  Tensor memory: S0 128, S1 128, O d columns.
+#include "attn_internal.h"
+#include "tc_common.cuh"
+
+namespace attn {
+namespace {
+
+using namespace tc;
+
+constexpr int TQ = 128;
+constexpr int kSoftmaxThreads = 256;
+constexpr int kThreads = kSoftmaxThreads + 64;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kRescaleThreshold = 8.f;   // log2 units
+
+struct FwdArgs {
+    __nv_bfloat16 *O;
+    float *LSE;
+    int n, BH;
+    int mask_kind, block, nb, mask_heads;
+    const int *row_ptr, *col_idx;   // block-CSR of the mask
+    float scale;
+    uint32_t *status;
+};
+
+template <int HD>
+struct FwdCfg {
+    static constexpr int TKF = HD == 256 ? 64 : 128;
+    static constexpr int NST = HD == 256 ? 2 : 3;
+    static constexpr uint32_t kQSlab = 128 * 128;              // [128 queries][64 bf16]
+    static constexpr uint32_t kKSlab = TKF * 128;              // [TKF keys][64 bf16]
+    static constexpr uint32_t kSlabs = HD / 64;
+    static constexpr uint32_t kQTile = kSlabs * kQSlab;
+    static constexpr uint32_t kKTile = kSlabs * kKSlab;
+    static constexpr uint32_t oQ = 0;
+    static constexpr uint32_t oK = oQ + kQTile;                // NST stages
+    static constexpr uint32_t oV = oK + NST * kKTile;          // NST stages
+    static constexpr uint32_t oX = oV + NST * kKTile;          // row-max exchange [2 buffers][2 wg][128]; row sums reuse buffer 0
+    static constexpr uint32_t oBar = oX + 4 * 128 * 4;
+    static constexpr uint32_t oMisc = oBar + 16 * 8;
+    static constexpr uint32_t kUsed = oMisc + 64;
+    static_assert(kUsed <= 227 * 1024, "shared memory budget");
+    // at least 117 KB so that only one CTA (which allocates all 512 tensor-memory columns) fits per SM
+    static constexpr uint32_t kBytes = kUsed < 117 * 1024 ? 117 * 1024 : kUsed;
+};
+
+enum { FB_Q = 0, FB_KVFULL = 1, FB_KVEMPTY = 4, FB_S = 7, FB_P = 9, FB_O = 11 };
+
+template <int TKF>
+struct KeyIter {
+    // Enumerates the key tiles (of TKF keys) a query tile `it` (128 queries) has to visit.
+    int kind, n, sub, raw;
+    const int *cols;
+    __device__ KeyIter(const FwdArgs &a, int it, long bh) : kind(a.mask_kind), n(a.n), sub(1), raw(0), cols(nullptr)
+    {
+        const int ntk = (n + TKF - 1) / TKF;
+        if (kind == ATTN_MASK_NONE) raw = ntk;
+        else if (kind == ATTN_MASK_CAUSAL) {
+            const int last_i = min(it * TQ + TQ, n) - 1;
+            raw = last_i / TKF + 1;
+        } else {
+            sub = a.block / TKF;
+            const int I = it * TQ / a.block;
+            const long mh = a.mask_heads == 1 ? 0 : bh;
+            const int *rp = a.row_ptr + mh * 2 * a.nb + 2 * I;
+            cols = a.col_idx + mh * (long)a.nb * a.nb + rp[0];
+            raw = (rp[1] - rp[0]) * sub;
+        }
+    }
+    __device__ int tile(int idx) const
+    {
+        int jt;
+        if (kind == ATTN_MASK_BLOCK_SPARSE) jt = cols[idx / sub] * sub + idx % sub;
+        else jt = idx;
+        return jt * TKF < n ? jt : -1;
+    }
+};
+
+__device__ __forceinline__ void named_bar_sync_f(int id, int count)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+
+template <int HD>
+__global__ void __launch_bounds__(kThreads, 1)
+tc_fwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mK,
+              const __grid_constant__ CUtensorMap mV, const FwdArgs a)
+{
+    using C = FwdCfg<HD>;
+    constexpr int TKF = C::TKF, NST = C::NST;
+    constexpr int CW = TKF / 2;      // key columns per warpgroup
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + C::oBar);
+    uint32_t *tmem_base_s = reinterpret_cast<uint32_t *>(smem + C::oMisc);
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(smem + C::oMisc + 4);
+    float *xmax = reinterpret_cast<float *>(smem + C::oX);            // [2][2][128]
+    float *xsum = xmax;                                               // [2][128], reuses exchange buffer 0 in the epilogue
+    const Abort ab{abort_flag, a.status};
+
+    const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
+    const int nt = (a.n + TQ - 1) / TQ;
+    const int it = nt - 1 - (int)blockIdx.x;    // heaviest causal tiles first
+    const long bh = blockIdx.y;
+    const int i0 = it * TQ, n = a.n;
+
+    if ((smem_u32(smem) & 1023u) != 0) {
+        if (tid == 0) atomicExch(a.status, 9u);
+        return;
+    }
+    if (tid == 0) {
+        *abort_flag = 0;
+        mbar_init(&bars[FB_Q], 1);
+        for (int s = 0; s < NST; ++s) { mbar_init(&bars[FB_KVFULL + s], 1); mbar_init(&bars[FB_KVEMPTY + s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&bars[FB_S + b], 1); mbar_init(&bars[FB_P + b], kSoftmaxThreads); }
+        mbar_init(&bars[FB_O], 1);
+        fence_barrier_init();
+        prefetch_tensormap(&mQ); prefetch_tensormap(&mK); prefetch_tensormap(&mV);
+    }
+    if (warp == 0) tmem_alloc(tmem_base_s, 512);
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tm = *tmem_base_s;
+    const uint32_t T_O = tm + 256;
+    const KeyIter<TKF> iter(a, it, bh);
+
+    // number of valid key tiles (same in every role)
+    int niter = 0;
+    for (int idx = 0; idx < iter.raw; ++idx) niter += iter.tile(idx) >= 0;
+
+    if (warp == 9) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            mbar_expect_tx(&bars[FB_Q], C::kQTile);
+#pragma unroll
+            for (uint32_t sl = 0; sl < C::kSlabs; ++sl)
+                tma_load_3d(smem + C::oQ + sl * C::kQSlab, &mQ, &bars[FB_Q], sl * 64, i0, (int)bh);
+            int k = 0;
+            for (int idx = 0; idx < iter.raw; ++idx) {
+                const int jt = iter.tile(idx);
+                if (jt < 0) continue;
+                const int s = k % NST;
+                if (k >= NST) mbar_wait(&bars[FB_KVEMPTY + s], ((k / NST) - 1) & 1, ab);
+                uint64_t *bar = &bars[FB_KVFULL + s];
+                mbar_expect_tx(bar, 2 * C::kKTile);
+#pragma unroll
+                for (uint32_t sl = 0; sl < C::kSlabs; ++sl) {
+                    tma_load_3d(smem + C::oK + s * C::kKTile + sl * C::kKSlab, &mK, bar, sl * 64, jt * TKF, (int)bh);
+                    tma_load_3d(smem + C::oV + s * C::kKTile + sl * C::kKSlab, &mV, bar, sl * 64, jt * TKF, (int)bh);
+                }
+                ++k;
+            }
+        }
+    } else if (warp == 8) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0 && niter == 0) mbar_wait(&bars[FB_Q], 0, ab);   // let the Q load land before exit
+        if (lane == 0 && niter > 0) {
+            constexpr uint32_t idesc_s = idesc_bf16(128, TKF, 0, 0);
+            constexpr uint32_t idesc_o = idesc_bf16(128, HD, 0, 1);
+            const uint32_t sQ = smem_u32(smem + C::oQ);
+            auto issue_S = [&](int k) {
+                const int s = k % NST;
+                mbar_wait(&bars[FB_KVFULL + s], (k / NST) & 1, ab);
+                tcgen05_fence_after();
+                const uint32_t sK = smem_u32(smem + C::oK + s * C::kKTile);
+#pragma unroll
+                for (int kk = 0; kk < HD / 16; ++kk)
+                    mma_ss(tm + (k & 1) * 128, smem_desc_kmajor(sQ + (kk / 4) * C::kQSlab + (kk % 4) * 32),
+                           smem_desc_kmajor(sK + (kk / 4) * C::kKSlab + (kk % 4) * 32), idesc_s, kk > 0);
+                mma_commit(&bars[FB_S + (k & 1)]);
+            };
+            mbar_wait(&bars[FB_Q], 0, ab);
+            issue_S(0);
+            for (int k = 0; k < niter; ++k) {
+                if (k + 1 < niter) issue_S(k + 1);
+                const int s = k % NST, b = k & 1;
+                mbar_wait(&bars[FB_P + b], (k >> 1) & 1, ab);
+                tcgen05_fence_after();
+                const uint32_t sV = smem_u32(smem + C::oV + s * C::kKTile);
+#pragma unroll
+                for (int kk = 0; kk < TKF / 16; ++kk)
+                    mma_ts(T_O, tm + b * 128 + kk * 8, smem_desc_mnmajor(sV + kk * 2048, C::kKSlab), idesc_o,
+                           (k > 0) || (kk > 0));
+                mma_commit(&bars[FB_KVEMPTY + s]);
+                mma_commit(&bars[FB_O]);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ softmax warpgroups
+        const int wg = warp / 4;
+        const int row = (warp % 4) * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)((warp % 4) * 32) << 16;
+        const int ig = i0 + row;
+        const float sl2 = a.scale * kLog2e;
+        float m_ref = -INFINITY, l_part = 0.f;
+        int k = 0;
+        for (int idx = 0; idx < iter.raw; ++idx) {
+            const int jt = iter.tile(idx);
+            if (jt < 0) continue;
+            const int b = k & 1, j0 = jt * TKF;
+            mbar_wait(&bars[FB_S + b], (k >> 1) & 1, ab);
+            tcgen05_fence_after();
+            const uint32_t T_S = tm + b * 128;
+            float sv[CW];
+#pragma unroll
+            for (int c = 0; c < CW; c += 32) {
+                uint32_t v[32];
+                tmem_ld32(T_S + lane_addr + wg * CW + c, v);
+                tmem_wait_ld();
+#pragma unroll
+                for (int e = 0; e < 32; ++e) sv[c + e] = __uint_as_float(v[e]) * sl2;
+            }
+            const bool need_mask = (a.mask_kind == ATTN_MASK_CAUSAL && j0 + TKF - 1 > i0) || j0 + TKF > n;
+            float mx = -INFINITY;
+            if (need_mask) {
+                const bool causal = a.mask_kind == ATTN_MASK_CAUSAL;
+#pragma unroll
+                for (int e = 0; e < CW; ++e) {
+                    const int jg = j0 + wg * CW + e;
+                    if (jg >= n || (causal && jg > ig)) sv[e] = -INFINITY;
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < CW; ++e) mx = fmaxf(mx, sv[e]);
+            float *xm = xmax + b * 256;
+            xm[wg * 128 + row] = mx;
+            named_bar_sync_f(1, kSoftmaxThreads);   // also: every S read of this tile is done
+            const float m_tile = fmaxf(xm[row], xm[128 + row]);
+            const bool need = m_tile > m_ref + kRescaleThreshold || (m_ref == -INFINITY && m_tile != -INFINITY);
+            if (__any_sync(0xffffffffu, need)) {
+                const float m_new = need ? fmaxf(m_ref, m_tile) : m_ref;
+                const float alpha = (need && m_ref != -INFINITY) ? exp2f(m_ref - m_new) : 1.f;
+                if (k > 0) {
+                    mbar_wait(&bars[FB_O], (k - 1) & 1, ab);   // O += P V of the previous tile has landed
+                    tcgen05_fence_after();
+#pragma unroll
+                    for (int c = 0; c < HD / 2; c += 32) {
+                        uint32_t v[32];
+                        tmem_ld32(T_O + lane_addr + wg * (HD / 2) + c, v);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * alpha);
+                        tmem_st32(T_O + lane_addr + wg * (HD / 2) + c, v);
+                    }
+                }
+                l_part *= alpha;
+                m_ref = m_new;
+            }
+            const float off = m_ref == -INFINITY ? 0.f : m_ref;
+            uint32_t pp[CW / 2];
+            float rs = 0.f;
+#pragma unroll
+            for (int e = 0; e < CW; e += 2) {
+                const float p0 = exp2f(sv[e] - off), p1 = exp2f(sv[e + 1] - off);
+                rs += p0 + p1;
+                pp[e / 2] = pack_bf16(p0, p1);
+            }
+            l_part += rs;
+            if (CW == 64) {
+                uint32_t(&pp32)[32] = *reinterpret_cast<uint32_t(*)[32]>(pp);
+                tmem_st32(T_S + lane_addr + wg * (CW / 2), pp32);
+            } else {
+                uint32_t(&pp16)[16] = *reinterpret_cast<uint32_t(*)[16]>(pp);
+                tmem_st16(T_S + lane_addr + wg * (CW / 2), pp16);
+            }
+            tmem_wait_st();
+            tcgen05_fence_before();
+            mbar_arrive(&bars[FB_P + b]);
+            ++k;
+        }
+        // ------------------------------------------------------------ epilogue
+        named_bar_sync_f(1, kSoftmaxThreads);   // everyone is done with the row-max exchange buffers
+        xsum[wg * 128 + row] = l_part;
+        named_bar_sync_f(1, kSoftmaxThreads);
+        const float l_tot = xsum[row] + xsum[128 + row];
+        if (k > 0) {
+            mbar_wait(&bars[FB_O], (k - 1) & 1, ab);
+            tcgen05_fence_after();
+        }
+        const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
+        const int ic = ig < n ? ig : 0;
+        __nv_bfloat16 *po = a.O + ((size_t)bh * n + ic) * HD + wg * (HD / 2);
+#pragma unroll
+        for (int c = 0; c < HD / 2; c += 32) {
+            uint32_t v[32];
+            if (k > 0) {
+                tmem_ld32(T_O + lane_addr + wg * (HD / 2) + c, v);
+                tmem_wait_ld();
+            } else {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) v[e] = 0u;
+            }
+            if (ig < n) {
+#pragma unroll
+                for (int e = 0; e < 32; e += 8) {
+                    uint4 o;
+                    o.x = pack_bf16(__uint_as_float(v[e]) * inv, __uint_as_float(v[e + 1]) * inv);
+                    o.y = pack_bf16(__uint_as_float(v[e + 2]) * inv, __uint_as_float(v[e + 3]) * inv);
+                    o.z = pack_bf16(__uint_as_float(v[e + 4]) * inv, __uint_as_float(v[e + 5]) * inv);
+                    o.w = pack_bf16(__uint_as_float(v[e + 6]) * inv, __uint_as_float(v[e + 7]) * inv);
+                    *reinterpret_cast<uint4 *>(po + c + e) = o;
+                }
+            }
+        }
+        if (wg == 0 && ig < n) a.LSE[(size_t)bh * n + ig] = l_tot > 0.f ? m_ref * kLn2 + logf(l_tot) : -INFINITY;
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tm, 512);
+}
+
+template <int HD>
+attn_status launch_fwd(const Problem &p)
+{
+    using C = FwdCfg<HD>;
+    CUtensorMap mQ, mK, mV;
+    const uint64_t BH = (uint64_t)p.BH;
+    if (!make_tmap_bf16_3d(&mQ, p.Q, HD, p.n, BH, 128) || !make_tmap_bf16_3d(&mK, p.K, HD, p.n, BH, C::TKF) ||
+        !make_tmap_bf16_3d(&mV, p.V, HD, p.n, BH, C::TKF))
+        return ATTN_ERR_LAUNCH;
+    FwdArgs a{};
+    a.O = (__nv_bfloat16 *)p.Oout; a.LSE = p.LSEout;
+    a.n = p.n; a.BH = (int)p.BH;
+    a.mask_kind = p.mask_kind; a.block = p.block; a.nb = p.nb; a.mask_heads = p.mask_heads;
+    a.row_ptr = p.row_ptr; a.col_idx = p.col_idx;
+    a.scale = p.scale;
+    a.status = p.status;
+    auto kernel = tc_fwd_kernel<HD>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kBytes) != cudaSuccess)
+        return ATTN_ERR_LAUNCH;
+    const dim3 grid((p.n + TQ - 1) / TQ, (unsigned)p.BH);
+    launch_begin("tc_fwd", p.stream);
+    kernel<<<grid, kThreads, C::kBytes, p.stream>>>(mQ, mK, mV, a);
+    launch_end(p.stream);
+    return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_LAUNCH;
+}
+
+}  // namespace
+
+size_t fwd_smem_bytes(int d)
+{
+    return d == 64 ? FwdCfg<64>::kUsed : d == 128 ? FwdCfg<128>::kUsed : d == 256 ? FwdCfg<256>::kUsed : 0;
+}
+
+attn_status tc_fwd(const Problem &p)
+{
+    if (p.d == 64) return launch_fwd<64>(p);
+    if (p.d == 128) return launch_fwd<128>(p);
+    if (p.d == 256) return launch_fwd<256>(p);
+    return ATTN_ERR_TILE;
+}
+
+}  // namespace attn

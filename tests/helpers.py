@@ -64,8 +64,14 @@ def run_case(b, h, n, d, dtype, mask_kind, *, seed=7, block=128, bmask=None, cfg
     if mask_kind != inputs.MASK_NONE:
         mask = B.Mask(kind=mask_kind, block=block,
                       block_mask=torch.from_numpy(bmask).cuda() if bmask is not None else None)
-    O, LSE = attn.attn_fwd(dev["Q"], dev["K"], dev["V"], mask=mask, scale=scale, cfg=cfg)
-    dQ, dK, dV = attn.attn_bwd(dev["Q"], dev["K"], dev["V"], O, dev["dO"], LSE, mask=mask, scale=scale, cfg=cfg)
+    dt = B.ATTN_BF16 if dtype == "bf16" else B.ATTN_F32
+    ws_f = torch.zeros(max(256, B.attn_fwd_workspace_bytes(n, d, h, b, mask, dt, cfg)), dtype=torch.uint8, device="cuda")
+    ws_b = torch.zeros(max(256, B.attn_bwd_workspace_bytes(n, d, h, b, mask, dt, cfg)), dtype=torch.uint8, device="cuda")
+    O, LSE = attn.attn_fwd(dev["Q"], dev["K"], dev["V"], mask=mask, scale=scale, cfg=cfg, workspace=ws_f)
+    assert attn.attn_workspace_status(ws_f) == B.ATTN_OK, "forward kernel reported an error"
+    dQ, dK, dV = attn.attn_bwd(dev["Q"], dev["K"], dev["V"], O, dev["dO"], LSE, mask=mask, scale=scale, cfg=cfg,
+                               workspace=ws_b)
+    assert attn.attn_workspace_status(ws_b) == B.ATTN_OK, "backward kernel reported an error"
     torch.cuda.synchronize()
     errs = {
         "O": rel_err(to_np(O), O_ref), "LSE": rel_err(to_np(LSE), LSE_ref),
@@ -77,7 +83,8 @@ def run_case(b, h, n, d, dtype, mask_kind, *, seed=7, block=128, bmask=None, cfg
         LSE_in = torch.from_numpy(LSE_ref.astype(np.float32)).cuda()
         g_ref2 = orc.attn_bwd(x["Q"], x["K"], x["V"], to_np(O_in), x["dO"], to_np(LSE_in), scale=sc, **mk)
         dQ2, dK2, dV2 = attn.attn_bwd(dev["Q"], dev["K"], dev["V"], O_in, dev["dO"], LSE_in, mask=mask, scale=scale,
-                                      cfg=cfg)
+                                      cfg=cfg, workspace=ws_b)
+        assert attn.attn_workspace_status(ws_b) == B.ATTN_OK, "backward kernel reported an error"
         torch.cuda.synchronize()
         errs.update({"dQ_bwdonly": rel_err(to_np(dQ2), g_ref2[0]), "dK_bwdonly": rel_err(to_np(dK2), g_ref2[1]),
                      "dV_bwdonly": rel_err(to_np(dV2), g_ref2[2])})

@@ -1,0 +1,97 @@
+"""GPU parity of the tensor-core (tcgen05 / TMEM / TMA) kernels against the float64 oracle.
+
+Tolerance for bf16 inputs with fp32 accumulation: max|err| <= 2e-2 * max|ref| per tensor.
+"""
+import numpy as np
+import pytest
+
+from paper_2410_09397_b200 import inputs
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+def fused():
+    from paper_2410_09397_b200 import binding as B
+    return B.Cfg(algo=B.ATTN_ALGO_FUSED)
+
+
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("n", [128, 256, 640])
+@pytest.mark.parametrize("mask_kind", [inputs.MASK_NONE, inputs.MASK_CAUSAL])
+def test_fused_small(n, d, mask_kind):
+    errs = H.run_case(1, 2, n, d, "bf16", mask_kind, seed=31, cfg=fused())
+    H.assert_within(errs, "bf16")
+
+
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("n", [8, 136, 200, 1000])
+@pytest.mark.parametrize("mask_kind", [inputs.MASK_NONE, inputs.MASK_CAUSAL])
+def test_fused_ragged_tails(n, d, mask_kind):
+    """n not a multiple of the 128-row tile: TMA zero fill + masked tail columns."""
+    errs = H.run_case(2, 1, n, d, "bf16", mask_kind, seed=32, cfg=fused())
+    H.assert_within(errs, "bf16")
+
+
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("n,block", [(512, 128), (1024, 256), (896, 128), (600, 128)])
+def test_fused_block_sparse(n, d, block):
+    errs = H.run_case(1, 3, n, d, "bf16", inputs.MASK_BLOCK_SPARSE, seed=33, block=block, keep_prob=0.3, cfg=fused())
+    H.assert_within(errs, "bf16")
+
+
+def test_fused_block_sparse_per_head_masks_and_empty_columns():
+    b, h, n, d, block = 1, 2, 512, 64, 128
+    bm = inputs.block_mask(34, n // block, 0.4, heads=b * h)
+    bm[1, :, 2] = 0          # no query attends to key block 2 of head 1: dK = dV = 0 there
+    bm[1, 2, 2] = 0
+    bm[1, 2, 0] = 1          # row 2 still has a kept block
+    errs = H.run_case(b, h, n, d, "bf16", inputs.MASK_BLOCK_SPARSE, seed=34, block=block, bmask=bm, cfg=fused())
+    H.assert_within(errs, "bf16")
+
+
+@pytest.mark.parametrize("n", [128, 320, 1024])
+@pytest.mark.parametrize("mask_kind", [inputs.MASK_NONE, inputs.MASK_CAUSAL])
+def test_forward_d256(n, mask_kind):
+    """d = 256 forward runs fused (64-key tiles); its backward is not the fused kernel."""
+    import torch
+    import paper_2410_09397_b200 as attn
+    from oracle import oracle as orc
+    x = H.make_inputs(35, 1, 2, n, 256, "bf16")
+    O_ref, LSE_ref = orc.attn_fwd(x["Q"], x["K"], x["V"], mask_kind=mask_kind)
+    dev = {k: H.to_dev(v, "bf16") for k, v in x.items()}
+    mask = attn.Mask(kind=mask_kind) if mask_kind else None
+    O, LSE = attn.attn_fwd(dev["Q"], dev["K"], dev["V"], mask=mask, cfg=fused())
+    torch.cuda.synchronize()
+    assert H.rel_err(H.to_np(O), O_ref) <= 2e-2
+    assert H.rel_err(H.to_np(LSE), LSE_ref) <= 2e-2
+
+
+def test_auto_selects_tensor_cores_for_bf16():
+    errs = H.run_case(2, 2, 512, 128, "bf16", inputs.MASK_CAUSAL, seed=36)
+    H.assert_within(errs, "bf16")
+    import paper_2410_09397_b200 as attn
+    attn.attn_timing_enable(True)
+    attn.attn_timing_collect()
+    H.run_case(1, 1, 256, 128, "bf16", inputs.MASK_NONE, seed=36, check_bwd_only=False)
+    names = [k for k, _ in attn.attn_timing_collect()]
+    attn.attn_timing_enable(False)
+    assert "tc_fwd" in names and "tc_bwd_fused" in names, names
+
+
+def test_large_scores_trigger_rescale():
+    """Scores that grow along the key axis force the running maximum to move (O rescale path)."""
+    import torch
+    import paper_2410_09397_b200 as attn
+    from oracle import oracle as orc
+    n, d = 512, 64
+    x = H.make_inputs(37, 1, 1, n, d, "bf16")
+    ramp = np.linspace(0.0, 6.0, n, dtype=np.float32)[None, None, :, None]
+    x["K"] = inputs.round_to_bf16((x["K"] * 0.2 + ramp * np.sign(x["Q"].mean())).astype(np.float32))
+    x["Q"] = inputs.round_to_bf16(np.abs(x["Q"]).astype(np.float32))
+    O_ref, LSE_ref = orc.attn_fwd(x["Q"], x["K"], x["V"])
+    dev = {k: H.to_dev(v, "bf16") for k, v in x.items()}
+    O, LSE = attn.attn_fwd(dev["Q"], dev["K"], dev["V"], cfg=fused())
+    torch.cuda.synchronize()
+    assert H.rel_err(H.to_np(O), O_ref) <= 2e-2
+    assert H.rel_err(H.to_np(LSE), LSE_ref) <= 2e-2
