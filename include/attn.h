@@ -118,6 +118,34 @@ attn_status attn_bwd(const void *Q, const void *K, const void *V, const void *O,
 attn_status attn_bwd_preprocess(const void *O, const void *dO, float *D, size_t rows, int d, int dt,
                                 void *cuda_stream);
 
+/* attn_bwd for callers that cannot allocate device memory (the paper has no
+ * counterpart: this is a convenience of the library, not a step of the method).
+ *
+ * Who needs it: code that is handed Q, K, V, O, dO, LSE and the output tensors but has
+ * no allocator it may call at that moment -- a plug-in inside a framework whose memory
+ * pool is frozen, a host callback, a real-time loop that must not call cudaMalloc.
+ * Such a caller cannot provide attn_bwd's `workspace`.  This entry point uses instead a
+ * fixed scratch array of attn_noalloc_scratch_bytes() = 8 MiB that is part of the
+ * library image (every GPU that loads the library holds these 8 MiB until the process
+ * exits).  It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *
+ *  - Same arguments, results and errors as attn_bwd, without workspace arguments.
+ *  - Limit: attn_bwd_workspace_bytes() of the problem must not exceed 8 MiB (for the
+ *    fused bf16 algorithm roughly batch*heads*n*d <= 2 Mi elements); larger problems
+ *    get ATTN_ERR_WORKSPACE and must use attn_bwd.
+ *  - The first call on each device looks up the array's device address (with that
+ *    device current); make that first call before starting any stream capture.
+ *  - All calls on a device share the one array and it keeps the previous call's
+ *    contents; the parts that must start at zero are cleared by every call.  Two calls
+ *    that overlap on the GPU (different streams, no ordering) race on it: serialise them.
+ *  - Device-side errors land in the array's first word; there is no way to read it from
+ *    outside, so use attn_bwd when you need attn_workspace_status(). */
+attn_status attn_bwd_noalloc(const void *Q, const void *K, const void *V, const void *O, const void *dO,
+                             const float *LSE, void *dQ, void *dK, void *dV,
+                             int n, int d, int heads, int batch, const attn_mask *mask,
+                             int dt, float scale, const attn_cfg *cfg, void *cuda_stream);
+size_t attn_noalloc_scratch_bytes(void);
+
 /* Workspace sizes in bytes for the same arguments (0 on invalid arguments). */
 size_t attn_fwd_workspace_bytes(int n, int d, int heads, int batch, const attn_mask *mask, int dt,
                                 const attn_cfg *cfg);

@@ -27,7 +27,7 @@ EXPORTS = (
     "attn_fwd", "attn_bwd", "attn_bwd_preprocess", "attn_fwd_workspace_bytes", "attn_bwd_workspace_bytes",
     "attn_workspace_status", "attn_supported_cfgs", "attn_cfg_onchip_elems", "attn_io_bound_elems",
     "attn_io_bound_sparse_elems", "attn_status_str", "attn_kernel_launches", "attn_timing_enable",
-    "attn_timing_collect",
+    "attn_timing_collect", "attn_bwd_noalloc", "attn_noalloc_scratch_bytes",
 )
 
 
@@ -92,6 +92,10 @@ def lib() -> ctypes.CDLL:
                            ctypes.POINTER(CCfg), vp, sz, vp]
     L.attn_bwd.restype = ci
     L.attn_bwd.argtypes = [vp] * 9 + [ci, ci, ci, ci, ctypes.POINTER(CMask), ci, cf, ctypes.POINTER(CCfg), vp, sz, vp]
+    L.attn_bwd_noalloc.restype = ci
+    L.attn_bwd_noalloc.argtypes = [vp] * 9 + [ci, ci, ci, ci, ctypes.POINTER(CMask), ci, cf, ctypes.POINTER(CCfg), vp]
+    L.attn_noalloc_scratch_bytes.restype = sz
+    L.attn_noalloc_scratch_bytes.argtypes = []
     L.attn_bwd_preprocess.restype = ci
     L.attn_bwd_preprocess.argtypes = [vp, vp, vp, sz, ci, ci, vp]
     for f in (L.attn_fwd_workspace_bytes, L.attn_bwd_workspace_bytes):
@@ -256,3 +260,27 @@ def attn_timing_collect(max_entries: int = 256) -> list[tuple[str, float]]:
     names = (ctypes.c_char_p * max_entries)()
     cnt = lib().attn_timing_collect(ms, names, max_entries)
     return [(names[i].decode(), float(ms[i])) for i in range(cnt)]
+
+
+def attn_noalloc_scratch_bytes() -> int:
+    return int(lib().attn_noalloc_scratch_bytes())
+
+
+def attn_bwd_noalloc(Q, K, V, O, dO, LSE, dQ, dK, dV, *, mask: Mask | None = None, scale: float = 0.0,
+                     cfg: Cfg | None = None):
+    """``attn_bwd`` without a workspace, for callers that cannot allocate device memory.
+
+    The caller passes every tensor, outputs included (this wrapper allocates nothing
+    either); the scratch is an 8 MiB array inside the library, shared by all calls on a
+    device, so calls must not overlap on the GPU.  Problems whose workspace would exceed
+    it raise ``AttnError(ATTN_ERR_WORKSPACE)``.
+    """
+    _check_tensors(Q, K, V, O, dO, LSE, dQ, dK, dV)
+    b, h, n, d = Q.shape
+    cm, cc = (mask.c() if mask else None), (cfg.c() if cfg else None)
+    st = lib().attn_bwd_noalloc(Q.data_ptr(), K.data_ptr(), V.data_ptr(), O.data_ptr(), dO.data_ptr(),
+                                LSE.data_ptr(), dQ.data_ptr(), dK.data_ptr(), dV.data_ptr(), n, d, h, b, _ref(cm),
+                                _dtype_code(Q), scale, _ref(cc), _stream())
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_bwd_noalloc")
+    return dQ, dK, dV
