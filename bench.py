@@ -244,15 +244,25 @@ def main():
     ap.add_argument("--tile-k", type=int, default=0)
     ap.add_argument("--tile-d", type=int, default=0)
     ap.add_argument("--deterministic", type=int, default=0)
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling on a smaller case)")
+    ap.add_argument("--heads", type=int, default=0, help="override the workload's heads")
+    ap.add_argument("--profile", action="store_true",
+                    help="for runs under ncu: allow fewer than 3 warm-up steps, skip e2e and the CPU baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
-    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.profile:
+        args.no_e2e = args.no_cpu_baseline = True
+    elif args.impl == "ours":
+        args.warmup = max(args.warmup, 3)
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     w = inputs.WORKLOADS[args.workload]
+    if args.batch or args.heads:
+        w = inputs.Workload(**{**w.__dict__, "batch": args.batch or w.batch, "heads": args.heads or w.heads,
+                               "name": w.name + "-reduced"})
     bmask = w.block_mask()
 
     if args.impl == "reference":

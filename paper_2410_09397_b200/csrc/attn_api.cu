@@ -96,6 +96,7 @@ attn_status layout(const Args &a, int backward, attn_cfg *cfg_out, WorkspaceLayo
         L->col_ptr = off; off += align_up(mh * 2 * nb * sizeof(int), 256);
         L->row_idx = off; off += align_up(mh * nb * nb * sizeof(int), 256);
     }
+    if (backward && c.algo == ATTN_ALGO_FUSED) { L->nLSE2 = off; off += align_up(BH * a.n * sizeof(float), 256); }
     if (backward && c.algo == ATTN_ALGO_FUSED && !c.deterministic) {
         L->dQ_acc = off; off += align_up(BH * a.n * a.d * sizeof(float), 256);
     }
@@ -148,6 +149,7 @@ attn_status fill_problem(Problem &p, const Args &a, int backward, float scale, v
     char *w = (char *)workspace;
     p.status = (uint32_t *)(w + L.status);
     p.D = backward ? (float *)(w + L.D) : nullptr;
+    p.nLSE2 = L.nLSE2 ? (float *)(w + L.nLSE2) : nullptr;
     p.row_ptr = L.row_ptr ? (int *)(w + L.row_ptr) : nullptr;
     p.col_idx = L.col_idx ? (int *)(w + L.col_idx) : nullptr;
     p.col_ptr = L.col_ptr ? (int *)(w + L.col_ptr) : nullptr;

@@ -25,6 +25,7 @@ struct Problem {
     // workspace sections (device)
     uint32_t *status;                 // 4-byte status word
     float *D;                         // [BH * n]
+    float *nLSE2;                     // [BH * n]: -LSE * log2(e), fused backward only
     int *row_ptr, *col_idx;           // block-CSR of the mask: [mask_heads][nb+1], [mask_heads][nb*nb]
     int *col_ptr, *row_idx;           // block-CSC
     float *dQ_acc;                    // fp32 dQ accumulator [BH * n * d] (fused backward with atomics)
@@ -34,7 +35,7 @@ struct Problem {
 };
 
 struct WorkspaceLayout {
-    size_t status, D, row_ptr, col_idx, col_ptr, row_idx, dQ_acc, matP, matdP, matdS, total;
+    size_t status, D, nLSE2, row_ptr, col_idx, col_ptr, row_idx, dQ_acc, matP, matdP, matdS, total;
     int mat_heads;
 };
 

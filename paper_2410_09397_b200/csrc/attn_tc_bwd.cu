@@ -9,7 +9,8 @@
 //   S^T  = K_j Q_i^T                         (tcgen05.mma, both operands K-major smem)
 //   dP^T = V_j dO_i^T                        (same)
 //   P^T  = exp2(S^T * scale*log2e - LSE_i*log2e)        (256 threads, fp32)
-//   dS^T = P^T o (dP^T - D_i)                           (Definition B.9, p = f o q - diag(v) f)
+//   dS^T = scale * P^T o (dP^T - D_i)                   (Definition B.9, p = f o q - diag(v) f;
+//                                                        the scale of dQ and dK is folded in here)
 //   dV_j += P^T  dO_i      A = P^T  in tensor memory (bf16), B = dO_i MN-major smem
 //   dK_j += dS^T Q_i       A = dS^T K-major smem,            B = Q_i  MN-major smem
 //   dQ_i += dS K_j         computed as dQ^T = K_j^T dS^T for d = 128 (so that the fp32
@@ -37,7 +38,7 @@ constexpr int kThreads = kSoftmaxThreads + 32;
 constexpr uint32_t SLAB = 128 * 128;   // bytes of one [128 rows][64 bf16] slab
 
 struct BwdArgs {
-    const float *LSE, *D;
+    const float *nLSE2, *Ds;   // -LSE log2(e) and scale * D per row (workspace)
     float *dQ_acc;
     __nv_bfloat16 *dK, *dV;
     int n, BH;
@@ -64,7 +65,7 @@ struct BwdSmem {
     static_assert(kBytes <= 227 * 1024, "shared memory budget");
 };
 
-enum { BAR_KV = 0, BAR_QFULL = 1, BAR_QEMPTY = 3, BAR_S = 5, BAR_P = 6, BAR_DQ = 7, BAR_DQDONE = 8 };
+enum { BAR_KV = 0, BAR_QFULL = 1, BAR_QEMPTY = 3, BAR_S = 5, BAR_P = 6, BAR_DQ = 7, BAR_DQDONE = 8, BAR_DP = 9, BAR_DS = 10 };
 
 struct TileIter {
     // Enumerates the query tiles a key tile jt has to visit.
@@ -114,6 +115,52 @@ __device__ __forceinline__ void red_add_v4(float *p, float a, float b, float c, 
     asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
 
+__device__ __forceinline__ float ex2_approx(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// D pre-pass of the fused backward: Ds_i = scale * sum_c dO_ic O_ic and
+// nlse2_i = -LSE_i * log2(e) (minus infinity for a row with no kept entry, so that its
+// probabilities come out as exactly zero).  16-byte loads, HD/8 lanes share a row.
+template <int HD>
+__global__ void __launch_bounds__(256) tc_preprocess_kernel(const __nv_bfloat16 *__restrict__ O,
+                                                            const __nv_bfloat16 *__restrict__ dO,
+                                                            const float *__restrict__ LSE, float *__restrict__ Ds,
+                                                            float *__restrict__ nlse2, size_t rows, float scale)
+{
+    constexpr int LPR = HD / 8;   // lanes per row
+    constexpr int RPW = 32 / LPR; // rows per warp
+    const int lane = threadIdx.x % 32, sub = lane / LPR, lr = lane % LPR;
+    const size_t warp = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) / 32;
+    const size_t nwarps = (size_t)gridDim.x * blockDim.x / 32;
+    for (size_t base = warp * RPW; base < rows; base += nwarps * RPW) {
+        const size_t row = base + sub;
+        float acc = 0.f;
+        if (row < rows) {
+            const uint4 xo = __ldg(reinterpret_cast<const uint4 *>(O + row * HD) + lr);
+            const uint4 xg = __ldg(reinterpret_cast<const uint4 *>(dO + row * HD) + lr);
+            const __nv_bfloat162 *eo = reinterpret_cast<const __nv_bfloat162 *>(&xo);
+            const __nv_bfloat162 *eg = reinterpret_cast<const __nv_bfloat162 *>(&xg);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float2 fo = __bfloat1622float2(eo[e]), fg = __bfloat1622float2(eg[e]);
+                acc = fmaf(fo.x, fg.x, acc);
+                acc = fmaf(fo.y, fg.y, acc);
+            }
+        }
+#pragma unroll
+        for (int o = LPR / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (row < rows && lr == 0) {
+            Ds[row] = acc * scale;
+            const float l = LSE[row];
+            nlse2[row] = l == -INFINITY ? -INFINITY : -l * 1.4426950408889634f;
+        }
+    }
+}
+
 template <int HD>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mK,
@@ -141,7 +188,9 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
         mbar_init(&bars[BAR_QFULL], 1); mbar_init(&bars[BAR_QFULL + 1], 1);
         mbar_init(&bars[BAR_QEMPTY], 1); mbar_init(&bars[BAR_QEMPTY + 1], 1);
         mbar_init(&bars[BAR_S], 1);
+        mbar_init(&bars[BAR_DP], 1);
         mbar_init(&bars[BAR_P], kSoftmaxThreads);
+        mbar_init(&bars[BAR_DS], kSoftmaxThreads);
         mbar_init(&bars[BAR_DQ], 1);
         mbar_init(&bars[BAR_DQDONE], kSoftmaxThreads);
         fence_barrier_init();
@@ -155,7 +204,6 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
     const uint32_t T_S = tm, T_dP = tm + 128, T_dV = tm + 256, T_dK = tm + 256 + HD;
 
     const TileIter iter(a, jt, bh);
-    const float sl2 = a.scale * 1.4426950408889634f;
 
     if (warp == 8) {
         // ------------------------------------------------------------ producer + MMA issuer
@@ -174,8 +222,18 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
                     tma_load_3d(smem + L::oQ + s * L::kTile + sl * SLAB, &mQ, bar, sl * 64, i0, (int)bh);
                     tma_load_3d(smem + L::odO + s * L::kTile + sl * SLAB, &mdO, bar, sl * 64, i0, (int)bh);
                 }
-                bulk_load_1d(smem + L::oLSE + s * 512, a.LSE + bh * n + i0, rows * 4, bar);
-                bulk_load_1d(smem + L::oD + s * 512, a.D + bh * n + i0, rows * 4, bar);
+                bulk_load_1d(smem + L::oLSE + s * 512, a.nLSE2 + bh * n + i0, rows * 4, bar);
+                bulk_load_1d(smem + L::oD + s * 512, a.Ds + bh * n + i0, rows * 4, bar);
+            };
+            // S^T = K_j Q_i^T for the tile in stage s
+            auto issue_S = [&](int s) {
+                const uint32_t sQ = smem_u32(smem + L::oQ + s * L::kTile);
+#pragma unroll
+                for (int kk = 0; kk < HD / 16; ++kk) {
+                    const uint32_t off = (kk / 4) * SLAB + (kk % 4) * 32;
+                    mma_ss(T_S, smem_desc_kmajor(sK + off), smem_desc_kmajor(sQ + off), idesc_s, kk > 0);
+                }
+                mma_commit(&bars[BAR_S]);
             };
             mbar_expect_tx(&bars[BAR_KV], 2 * L::kTile);
 #pragma unroll
@@ -186,7 +244,13 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
             // first valid tile
             int idx = 0, it = -1;
             while (idx < iter.raw && (it = iter.tile(idx)) < 0) ++idx;
-            if (it >= 0) issue_load(it, 0);
+            if (it >= 0) {
+                issue_load(it, 0);
+                mbar_wait(&bars[BAR_QFULL], 0, ab);
+                mbar_wait(&bars[BAR_KV], 0, ab);
+                tcgen05_fence_after();
+                issue_S(0);
+            }
             int k = 0;   // count of processed tiles
             while (idx < iter.raw) {
                 const int s = k & 1;
@@ -197,17 +261,8 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
                     if (k >= 1) mbar_wait(&bars[BAR_QEMPTY + (s ^ 1)], ((k - 1) >> 1) & 1, ab);
                     issue_load(nit, s ^ 1);
                 }
-                mbar_wait(&bars[BAR_QFULL + s], (k >> 1) & 1, ab);
-                if (k == 0) mbar_wait(&bars[BAR_KV], 0, ab);
-                tcgen05_fence_after();
                 const uint32_t sQ = smem_u32(smem + L::oQ + s * L::kTile), sdO = smem_u32(smem + L::odO + s * L::kTile);
-                // S^T = K_j Q_i^T
-#pragma unroll
-                for (int kk = 0; kk < HD / 16; ++kk) {
-                    const uint32_t off = (kk / 4) * SLAB + (kk % 4) * 32;
-                    mma_ss(T_S, smem_desc_kmajor(sK + off), smem_desc_kmajor(sQ + off), idesc_s, kk > 0);
-                }
-                if (k > 0) {
+                if (k > 0) {   // the dQ tile of the previous pair has been read out of T_dP
                     mbar_wait(&bars[BAR_DQDONE], (k - 1) & 1, ab);
                     tcgen05_fence_after();
                 }
@@ -217,20 +272,22 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
                     const uint32_t off = (kk / 4) * SLAB + (kk % 4) * 32;
                     mma_ss(T_dP, smem_desc_kmajor(sV + off), smem_desc_kmajor(sdO + off), idesc_s, kk > 0);
                 }
-                mma_commit(&bars[BAR_S]);
+                mma_commit(&bars[BAR_DP]);
+                // dV += P^T dO_i as soon as P^T is in tensor memory
                 mbar_wait(&bars[BAR_P], k & 1, ab);
                 tcgen05_fence_after();
-                // dV += P^T dO_i ; dK += dS^T Q_i   (contraction over the 128 queries of the tile)
 #pragma unroll
                 for (int kk = 0; kk < TQ / 16; ++kk)
                     mma_ts(T_dV, T_S + kk * 8, smem_desc_mnmajor(sdO + kk * 2048, SLAB), idesc_dv, (k > 0) || (kk > 0));
+                // dK += dS^T Q_i and the dQ tile once dS^T is in shared memory
+                mbar_wait(&bars[BAR_DS], k & 1, ab);
+                tcgen05_fence_after();
 #pragma unroll
                 for (int kk = 0; kk < TQ / 16; ++kk) {
                     const uint32_t offa = (kk / 4) * SLAB + (kk % 4) * 32;
                     mma_ss(T_dK, smem_desc_kmajor(sdS + offa), smem_desc_mnmajor(sQ + kk * 2048, SLAB), idesc_dv,
                            (k > 0) || (kk > 0));
                 }
-                // dQ tile (contraction over the 128 keys of this CTA)
 #pragma unroll
                 for (int kk = 0; kk < TK / 16; ++kk) {
                     if (HD == 128)   // dQ^T = K_j^T dS^T : A = K_j MN-major, B = dS^T MN-major
@@ -242,6 +299,12 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
                 }
                 mma_commit(&bars[BAR_DQ]);
                 mma_commit(&bars[BAR_QEMPTY + s]);
+                // S^T of the next pair runs while the dQ tile is being read out
+                if (nit >= 0) {
+                    mbar_wait(&bars[BAR_QFULL + (s ^ 1)], ((k + 1) >> 1) & 1, ab);
+                    tcgen05_fence_after();
+                    issue_S(s ^ 1);
+                }
                 ++k;
                 idx = nidx;
             }
@@ -252,73 +315,114 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
         const int row = (warp % 4) * 32 + lane;        // tensor-memory lane = key row inside the tile
         const uint32_t lane_addr = (uint32_t)((warp % 4) * 32) << 16;
         const int jg = j0 + row;
+        const float sl2 = a.scale * 1.4426950408889634f;
         int k = 0;
         for (int idx = 0; idx < iter.raw; ++idx) {
             const int it = iter.tile(idx);
             if (it < 0) continue;
             const int s = k & 1, i0 = it * TQ;
-            const float *sLSE = reinterpret_cast<const float *>(smem + L::oLSE + s * 512);
-            const float *sD = reinterpret_cast<const float *>(smem + L::oD + s * 512);
-            mbar_wait(&bars[BAR_QFULL + s], (k >> 1) & 1, ab);   // LSE_i, D_i visible
+            const float4 *sNL = reinterpret_cast<const float4 *>(smem + L::oLSE + s * 512 + wg * 256);
+            const float4 *sDs = reinterpret_cast<const float4 *>(smem + L::oD + s * 512 + wg * 256);
+            const bool diag = a.mask_kind == ATTN_MASK_CAUSAL && it == jt;
+            const bool masked = diag || i0 + TQ > n || j0 + TK > n;   // uniform over the CTA
+            const int ig0 = i0 + wg * 64;                             // first query column of this thread
+            mbar_wait(&bars[BAR_QFULL + s], (k >> 1) & 1, ab);        // -LSE_i log2e and scale * D_i visible
             mbar_wait(&bars[BAR_S], k & 1, ab);
             tcgen05_fence_after();
-            const bool diag = a.mask_kind == ATTN_MASK_CAUSAL && it == jt;
-            uint32_t ppack[32];
-#pragma unroll
-            for (int ch = 0; ch < 2; ++ch) {
-                const int c0 = wg * 64 + ch * 32;
-                uint32_t sv[32], pv[32];
-                tmem_ld32(T_S + lane_addr + c0, sv);
-                tmem_ld32(T_dP + lane_addr + c0, pv);
+            // ---- P^T = exp2(S^T scale log2e - LSE log2e)
+            float p[64];
+            {
+                uint32_t sv0[32], sv1[32];
+                tmem_ld32(T_S + lane_addr + wg * 64, sv0);
+                tmem_ld32(T_S + lane_addr + wg * 64 + 32, sv1);
                 tmem_wait_ld();
-                uint32_t dsp[16];
 #pragma unroll
-                for (int e = 0; e < 32; e += 2) {
-                    float p[2], ds[2];
-#pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        const int il = c0 + e + u, ig = i0 + il;
-                        const float lse = sLSE[il];
-                        const bool ok = ig < n && jg < n && lse != -INFINITY && (!diag || jg <= ig);
-                        const float x = exp2f(__uint_as_float(sv[e + u]) * sl2 - lse * 1.4426950408889634f);
-                        p[u] = ok ? x : 0.f;
-                        ds[u] = ok ? p[u] * (__uint_as_float(pv[e + u]) - sD[il]) : 0.f;
-                    }
-                    ppack[ch * 16 + e / 2] = pack_bf16(p[0], p[1]);
-                    dsp[e / 2] = pack_bf16(ds[0], ds[1]);
-                }
-                // dS^T[j][i] into shared memory, 128-byte-swizzled slab wg (queries 64 wg .. 64 wg + 63)
-                uint8_t *slab = smem + L::odS + wg * SLAB;
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const uint32_t col = ch * 32 + q * 8;
-                    *reinterpret_cast<uint4 *>(slab + sw128_offset(row, col)) =
-                        make_uint4(dsp[q * 4], dsp[q * 4 + 1], dsp[q * 4 + 2], dsp[q * 4 + 3]);
+                for (int q = 0; q < 16; ++q) {
+                    const float4 nl = sNL[q];
+                    const uint32_t *sv = q < 8 ? &sv0[q * 4] : &sv1[(q - 8) * 4];
+                    p[q * 4 + 0] = ex2_approx(fmaf(__uint_as_float(sv[0]), sl2, nl.x));
+                    p[q * 4 + 1] = ex2_approx(fmaf(__uint_as_float(sv[1]), sl2, nl.y));
+                    p[q * 4 + 2] = ex2_approx(fmaf(__uint_as_float(sv[2]), sl2, nl.z));
+                    p[q * 4 + 3] = ex2_approx(fmaf(__uint_as_float(sv[3]), sl2, nl.w));
                 }
             }
+            if (masked) {
+#pragma unroll
+                for (int e = 0; e < 64; ++e) {
+                    const int ig = ig0 + e;
+                    const bool ok = ig < n && jg < n && (!diag || jg <= ig);
+                    p[e] = ok ? p[e] : 0.f;
+                }
+            }
+            uint32_t ppack[32];
+#pragma unroll
+            for (int e = 0; e < 32; ++e) ppack[e] = pack_bf16(p[2 * e], p[2 * e + 1]);
             // every thread has finished reading S^T before anyone overwrites it with P^T
             named_bar_sync(1, kSoftmaxThreads);
             tmem_st32(T_S + lane_addr + wg * 32, ppack);
             tmem_wait_st();
-            fence_proxy_async_smem();
             tcgen05_fence_before();
             mbar_arrive(&bars[BAR_P]);
 
-            // dQ tile: read out of tensor memory and reduce into the fp32 accumulator
+            // ---- dS^T = P^T o (scale dP^T - scale D): written once to shared memory
+            mbar_wait(&bars[BAR_DP], k & 1, ab);
+            tcgen05_fence_after();
+            {
+                uint32_t dv0[32], dv1[32];
+                tmem_ld32(T_dP + lane_addr + wg * 64, dv0);
+                tmem_ld32(T_dP + lane_addr + wg * 64 + 32, dv1);
+                tmem_wait_ld();
+                uint8_t *slab = smem + L::odS + wg * SLAB;
+#pragma unroll
+                for (int q8 = 0; q8 < 8; ++q8) {    // 8 query columns = one 16-byte chunk
+                    float ds[8];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int q = q8 * 2 + h;
+                        const float4 dsc = sDs[q];
+                        const uint32_t *dv = q < 8 ? &dv0[q * 4] : &dv1[(q - 8) * 4];
+                        ds[h * 4 + 0] = p[q * 4 + 0] * fmaf(__uint_as_float(dv[0]), a.scale, -dsc.x);
+                        ds[h * 4 + 1] = p[q * 4 + 1] * fmaf(__uint_as_float(dv[1]), a.scale, -dsc.y);
+                        ds[h * 4 + 2] = p[q * 4 + 2] * fmaf(__uint_as_float(dv[2]), a.scale, -dsc.z);
+                        ds[h * 4 + 3] = p[q * 4 + 3] * fmaf(__uint_as_float(dv[3]), a.scale, -dsc.w);
+                    }
+                    if (masked) {   // stale tail entries of the row vectors may be anything: select, do not multiply
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) ds[e] = p[q8 * 8 + e] != 0.f ? ds[e] : 0.f;
+                    }
+                    *reinterpret_cast<uint4 *>(slab + sw128_offset(row, q8 * 8)) =
+                        make_uint4(pack_bf16(ds[0], ds[1]), pack_bf16(ds[2], ds[3]), pack_bf16(ds[4], ds[5]),
+                                   pack_bf16(ds[6], ds[7]));
+                }
+            }
+            fence_proxy_async_smem();
+            tcgen05_fence_before();
+            mbar_arrive(&bars[BAR_DS]);
+
+            // ---- dQ tile: read out of tensor memory and reduce into the fp32 accumulator
             mbar_wait(&bars[BAR_DQ], k & 1, ab);
             tcgen05_fence_after();
             if (HD == 128) {
-                // lanes = head-dimension index c, columns = queries
-                float *base = a.dQ_acc + ((size_t)bh * n + i0) * HD + row;
+                // lanes = head-dimension index c, columns = queries: a warp adds 128 contiguous bytes
+                float *base = a.dQ_acc + ((size_t)bh * n + ig0) * HD + row;
+                uint32_t v0[32], v1[32];
+                tmem_ld32(T_dP + lane_addr + wg * 64, v0);
+                tmem_ld32(T_dP + lane_addr + wg * 64 + 32, v1);
+                tmem_wait_ld();
+                tcgen05_fence_before();
+                mbar_arrive(&bars[BAR_DQDONE]);   // T_dP is free again; the reductions proceed from registers
+                if (!masked || i0 + TQ <= n) {
 #pragma unroll
-                for (int ch = 0; ch < 2; ++ch) {
-                    const int c0 = wg * 64 + ch * 32;
-                    uint32_t v[32];
-                    tmem_ld32(T_dP + lane_addr + c0, v);
-                    tmem_wait_ld();
+                    for (int e = 0; e < 32; ++e) red_add_f32(base + (size_t)e * HD, __uint_as_float(v0[e]));
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) red_add_f32(base + (size_t)(32 + e) * HD, __uint_as_float(v1[e]));
+                } else {
 #pragma unroll
                     for (int e = 0; e < 32; ++e)
-                        if (i0 + c0 + e < n) red_add_f32(base + (size_t)(c0 + e) * HD, __uint_as_float(v[e]) * a.scale);
+                        if (ig0 + e < n) red_add_f32(base + (size_t)e * HD, __uint_as_float(v0[e]));
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        if (ig0 + 32 + e < n) red_add_f32(base + (size_t)(32 + e) * HD, __uint_as_float(v1[e]));
                 }
             } else {
                 // lanes = queries, columns = head-dimension index
@@ -326,20 +430,20 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
                 uint32_t v[32];
                 tmem_ld32(T_dP + lane_addr + c0, v);
                 tmem_wait_ld();
+                tcgen05_fence_before();
+                mbar_arrive(&bars[BAR_DQDONE]);
                 if (i0 + row < n) {
                     float *base = a.dQ_acc + ((size_t)bh * n + i0 + row) * HD + c0;
 #pragma unroll
                     for (int e = 0; e < HD / 2; e += 4)
-                        red_add_v4(base + e, __uint_as_float(v[e]) * a.scale, __uint_as_float(v[e + 1]) * a.scale,
-                                   __uint_as_float(v[e + 2]) * a.scale, __uint_as_float(v[e + 3]) * a.scale);
+                        red_add_v4(base + e, __uint_as_float(v[e]), __uint_as_float(v[e + 1]), __uint_as_float(v[e + 2]),
+                                   __uint_as_float(v[e + 3]));
                 }
             }
-            tcgen05_fence_before();
-            mbar_arrive(&bars[BAR_DQDONE]);
             ++k;
         }
         // ------------------------------------------------------------ epilogue: dV_j, dK_j
-        // (the last BAR_DQ phase also covers the last dV / dK accumulation)
+        // (the last BAR_DQ phase also covers the last dV / dK accumulation; dS carried the scale)
         {
             constexpr int HALF = HD / 2;
             const int jc = jg < n ? jg : 0;   // rows past n take part in the warp-wide loads but store nothing
@@ -364,10 +468,10 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
                         ov.y = pack_bf16(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
                         ov.z = pack_bf16(__uint_as_float(v[e + 4]), __uint_as_float(v[e + 5]));
                         ov.w = pack_bf16(__uint_as_float(v[e + 6]), __uint_as_float(v[e + 7]));
-                        ok.x = pack_bf16(__uint_as_float(w[e]) * a.scale, __uint_as_float(w[e + 1]) * a.scale);
-                        ok.y = pack_bf16(__uint_as_float(w[e + 2]) * a.scale, __uint_as_float(w[e + 3]) * a.scale);
-                        ok.z = pack_bf16(__uint_as_float(w[e + 4]) * a.scale, __uint_as_float(w[e + 5]) * a.scale);
-                        ok.w = pack_bf16(__uint_as_float(w[e + 6]) * a.scale, __uint_as_float(w[e + 7]) * a.scale);
+                        ok.x = pack_bf16(__uint_as_float(w[e]), __uint_as_float(w[e + 1]));
+                        ok.y = pack_bf16(__uint_as_float(w[e + 2]), __uint_as_float(w[e + 3]));
+                        ok.z = pack_bf16(__uint_as_float(w[e + 4]), __uint_as_float(w[e + 5]));
+                        ok.w = pack_bf16(__uint_as_float(w[e + 6]), __uint_as_float(w[e + 7]));
                         *reinterpret_cast<uint4 *>(pv + c + e) = ov;
                         *reinterpret_cast<uint4 *>(pk + c + e) = ok;
                     }
@@ -399,7 +503,7 @@ attn_status launch_bwd(const Problem &p)
         !make_tmap_bf16_3d(&mV, p.V, HD, p.n, BH, 128) || !make_tmap_bf16_3d(&mdO, p.dO, HD, p.n, BH, 128))
         return ATTN_ERR_LAUNCH;
     BwdArgs a{};
-    a.LSE = p.LSE; a.D = p.D; a.dQ_acc = p.dQ_acc;
+    a.nLSE2 = p.nLSE2; a.Ds = p.D; a.dQ_acc = p.dQ_acc;
     a.dK = (__nv_bfloat16 *)p.dK; a.dV = (__nv_bfloat16 *)p.dV;
     a.n = p.n; a.BH = (int)p.BH;
     a.mask_kind = p.mask_kind; a.block = p.block; a.nb = p.nb; a.mask_heads = p.mask_heads;
@@ -411,6 +515,17 @@ attn_status launch_bwd(const Problem &p)
         return ATTN_ERR_LAUNCH;
     const size_t acc_elems = (size_t)p.BH * p.n * HD;
     if (cudaMemsetAsync(p.dQ_acc, 0, acc_elems * sizeof(float), p.stream) != cudaSuccess) return ATTN_ERR_LAUNCH;
+    {
+        const size_t rows = (size_t)p.BH * p.n;
+        constexpr size_t rpw = 32 / (HD / 8);
+        size_t blocks = ((rows + rpw - 1) / rpw + 7) / 8;
+        if (blocks > 148 * 8) blocks = 148 * 8;
+        launch_begin("tc_bwd_preprocess", p.stream);
+        tc_preprocess_kernel<HD><<<(unsigned)blocks, 256, 0, p.stream>>>((const __nv_bfloat16 *)p.O, (const __nv_bfloat16 *)p.dO,
+                                                                         p.LSE, p.D, p.nLSE2, rows, p.scale);
+        launch_end(p.stream);
+        if (cudaGetLastError() != cudaSuccess) return ATTN_ERR_LAUNCH;
+    }
     const dim3 grid((p.n + TK - 1) / TK, (unsigned)p.BH);
     launch_begin("tc_bwd_fused", p.stream);
     kernel<<<grid, kThreads, L::kBytes, p.stream>>>(mQ, mK, mV, mdO, a);
@@ -430,8 +545,6 @@ size_t bwd_smem_bytes(int d) { return d == 64 ? BwdSmem<64>::kBytes : d == 128 ?
 
 attn_status tc_bwd(const Problem &p)
 {
-    attn_status st = preprocess_D(p.O, p.dO, p.D, (size_t)p.BH * p.n, p.d, p.dt, p.stream);
-    if (st != ATTN_OK) return st;
     if (p.d == 64) return launch_bwd<64>(p);
     if (p.d == 128) return launch_bwd<128>(p);
     return ATTN_ERR_TILE;
