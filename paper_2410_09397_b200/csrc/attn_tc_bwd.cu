@@ -36,6 +36,9 @@ constexpr int TQ = 128, TK = 128;
 constexpr int kSoftmaxThreads = 256;
 constexpr int kThreads = kSoftmaxThreads + 32;
 constexpr uint32_t SLAB = 128 * 128;   // bytes of one [128 rows][64 bf16] slab
+// dQ tile orientation at d = 128: transposed (lane = head-dimension index, coalesced scalar
+// reductions) or plain (lane = query, 16-byte vector reductions)
+constexpr bool kDqTransposed128 = true;
 
 struct BwdArgs {
     const float *nLSE2, *Ds;   // -LSE log2(e) and scale * D per row (workspace)
@@ -204,13 +207,14 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
     const uint32_t T_S = tm, T_dP = tm + 128, T_dV = tm + 256, T_dK = tm + 256 + HD;
 
     const TileIter iter(a, jt, bh);
+    constexpr bool kDqT = HD == 128 && kDqTransposed128;
 
     if (warp == 8) {
         // ------------------------------------------------------------ producer + MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc_s = idesc_bf16(128, 128, 0, 0);       // S^T, dP^T
             constexpr uint32_t idesc_dv = idesc_bf16(128, HD, 0, 1);       // dV (A tmem), dK (A K-major smem)
-            constexpr uint32_t idesc_dq = HD == 128 ? idesc_bf16(128, 128, 1, 1) : idesc_bf16(128, HD, 1, 1);
+            constexpr uint32_t idesc_dq = kDqT ? idesc_bf16(128, 128, 1, 1) : idesc_bf16(128, HD, 1, 1);
             const uint32_t sK = smem_u32(smem + L::oK), sV = smem_u32(smem + L::oV), sdS = smem_u32(smem + L::odS);
             auto issue_load = [&](int it, int s) {
                 const int i0 = it * TQ;
@@ -290,7 +294,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
                 }
 #pragma unroll
                 for (int kk = 0; kk < TK / 16; ++kk) {
-                    if (HD == 128)   // dQ^T = K_j^T dS^T : A = K_j MN-major, B = dS^T MN-major
+                    if (kDqT)        // dQ^T = K_j^T dS^T : A = K_j MN-major, B = dS^T MN-major
                         mma_ss(T_dP, smem_desc_mnmajor(sK + kk * 2048, SLAB), smem_desc_mnmajor(sdS + kk * 2048, SLAB),
                                idesc_dq, kk > 0);
                     else             // dQ = dS K_j : A = dS^T read MN-major, B = K_j MN-major
@@ -402,7 +406,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
             // ---- dQ tile: read out of tensor memory and reduce into the fp32 accumulator
             mbar_wait(&bars[BAR_DQ], k & 1, ab);
             tcgen05_fence_after();
-            if (HD == 128) {
+            if (kDqT) {
                 // lanes = head-dimension index c, columns = queries: a warp adds 128 contiguous bytes
                 float *base = a.dQ_acc + ((size_t)bh * n + ig0) * HD + row;
                 uint32_t v0[32], v1[32];
@@ -425,17 +429,19 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
                         if (ig0 + 32 + e < n) red_add_f32(base + (size_t)(32 + e) * HD, __uint_as_float(v1[e]));
                 }
             } else {
-                // lanes = queries, columns = head-dimension index
-                const int c0 = wg * (HD / 2);
-                uint32_t v[32];
-                tmem_ld32(T_dP + lane_addr + c0, v);
+                // lanes = queries, columns = head-dimension index: 16-byte vector reductions
+                constexpr int HALF = HD / 2;
+                uint32_t v[HALF];
+#pragma unroll
+                for (int c = 0; c < HALF; c += 32)
+                    tmem_ld32(T_dP + lane_addr + wg * HALF + c, *reinterpret_cast<uint32_t(*)[32]>(&v[c]));
                 tmem_wait_ld();
                 tcgen05_fence_before();
                 mbar_arrive(&bars[BAR_DQDONE]);
                 if (i0 + row < n) {
-                    float *base = a.dQ_acc + ((size_t)bh * n + i0 + row) * HD + c0;
+                    float *base = a.dQ_acc + ((size_t)bh * n + i0 + row) * HD + wg * HALF;
 #pragma unroll
-                    for (int e = 0; e < HD / 2; e += 4)
+                    for (int e = 0; e < HALF; e += 4)
                         red_add_v4(base + e, __uint_as_float(v[e]), __uint_as_float(v[e + 1]), __uint_as_float(v[e + 2]),
                                    __uint_as_float(v[e + 3]));
                 }

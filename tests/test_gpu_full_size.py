@@ -1,0 +1,73 @@
+"""Parity at the full benchmark sizes, in the launch configuration bench.py times.
+
+The whole workload runs on the GPU; the float64 oracle recomputes a sample of
+(batch, head) units -- heads are independent, so a sampled head is checked on every one
+of its outputs (O, LSE, dQ, dK, dV).  Sampled heads carry the repository generator's
+data; the other heads are filled with seeded device noise of the same distribution
+(they are computed but not compared).
+"""
+import numpy as np
+import pytest
+
+from oracle import oracle as orc
+from paper_2410_09397_b200 import inputs
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+def run_full(name, sample_heads, cfg=None, backward=True):
+    import torch
+    import paper_2410_09397_b200 as attn
+    w = inputs.WORKLOADS[name]
+    BH = w.batch * w.heads
+    tdt = torch.bfloat16 if w.bf16 else torch.float32
+    gen = torch.Generator(device="cuda").manual_seed(1234 + w.seed)
+    dev = {}
+    for k in ("Q", "K", "V", "dO"):
+        t = torch.randn((BH, w.n, w.d), generator=gen, device="cuda", dtype=torch.float32).to(tdt)
+        dev[k] = t
+    host = {}
+    for h in sample_heads:
+        host[h] = w.tensors(head_slice=(h, h + 1))
+        for k in dev:
+            dev[k][h].copy_(torch.from_numpy(host[h][k][0]).to(tdt))
+    bmask = w.block_mask()
+    mask = None
+    if w.mask != inputs.MASK_NONE:
+        mask = attn.Mask(kind=w.mask, block=w.block, block_mask=torch.from_numpy(bmask).cuda() if bmask is not None else None)
+    view = {k: v.view(w.batch, w.heads, w.n, w.d) for k, v in dev.items()}
+    O, LSE = attn.attn_fwd(view["Q"], view["K"], view["V"], mask=mask, cfg=cfg)
+    if backward:
+        dQ, dK, dV = attn.attn_bwd(view["Q"], view["K"], view["V"], O, view["dO"], LSE, mask=mask, cfg=cfg)
+    torch.cuda.synchronize()
+    assert torch.isfinite(O.float()).all()
+    mk = H.oracle_mask_kwargs(w.mask, w.block, bmask)
+    tol = H.TOL[w.dtype]
+    for h in sample_heads:
+        x = {k: v.astype(np.float64)[None] for k, v in host[h].items()}
+        O_ref, LSE_ref = orc.attn_fwd(x["Q"], x["K"], x["V"], **mk)
+        b, hh = divmod(h, w.heads)
+        errs = {"O": H.rel_err(H.to_np(O[b, hh]), O_ref[0, 0]), "LSE": H.rel_err(H.to_np(LSE[b, hh]), LSE_ref[0, 0])}
+        if backward:
+            g = orc.attn_bwd(x["Q"], x["K"], x["V"], O_ref, x["dO"], LSE_ref, **mk)
+            for nm, got, ref in zip(("dQ", "dK", "dV"), (dQ, dK, dV), g):
+                errs[nm] = H.rel_err(H.to_np(got[b, hh]), ref[0, 0])
+        bad = {k: v for k, v in errs.items() if not v <= tol}
+        assert not bad, f"{name} head {h}: over tolerance {tol}: {bad} (all {errs})"
+
+
+def test_config2_full():
+    run_full("C2", [0, 21, 63])
+
+
+def test_config3_full_headline():
+    run_full("C3", [0, 31])
+
+
+def test_config5_full_block_sparse():
+    run_full("C5", [17])
+
+
+def test_config4_forward_full():
+    run_full("C4", [0, 7], backward=False)
