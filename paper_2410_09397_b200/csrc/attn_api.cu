@@ -29,8 +29,16 @@ attn_status resolve_cfg(const Args &a, int backward, attn_cfg *out)
         const bool tc_ok = a.dt == ATTN_BF16 && (a.n % 8) == 0 && tc_cfg_supported(a.d, probe, backward) &&
                            !(a.mask && a.mask->kind == ATTN_MASK_BLOCK_SPARSE && a.mask->block % 128 != 0);
         c.algo = tc_ok ? ATTN_ALGO_FUSED : ATTN_ALGO_SIMT;
+        // d = 256 backward: the fused tile set does not fit on chip; the small-cache algorithm takes it
+        probe.algo = ATTN_ALGO_MATERIALIZED;
+        if (!tc_ok && backward && a.dt == ATTN_BF16 && a.d == 256 && (a.n % 8) == 0 &&
+            !(a.mask && a.mask->kind == ATTN_MASK_BLOCK_SPARSE) && tc_cfg_supported(a.d, probe, backward))
+            c.algo = ATTN_ALGO_MATERIALIZED;
     }
-    if (c.algo == ATTN_ALGO_MATERIALIZED && !backward) c.algo = ATTN_ALGO_FUSED;  // its forward is the fused one
+    if (c.algo == ATTN_ALGO_MATERIALIZED && !backward) {   // its forward is the fused one, with that kernel's own tiles
+        c.algo = ATTN_ALGO_FUSED;
+        c.tile_q = c.tile_k = c.tile_d = 0;
+    }
     if (c.algo == ATTN_ALGO_SIMT) {
         if ((c.tile_q && c.tile_q != 64) || (c.tile_k && c.tile_k != 64) || (c.tile_d && c.tile_d != 64))
             return ATTN_ERR_TILE;
@@ -40,6 +48,7 @@ attn_status resolve_cfg(const Args &a, int backward, attn_cfg *out)
         if (a.d != 64 && a.d != 128 && a.d != 256) return ATTN_ERR_SHAPE;
         if (a.n % 8 != 0) return ATTN_ERR_SHAPE;
         if (a.mask && a.mask->kind == ATTN_MASK_BLOCK_SPARSE && a.mask->block % 128 != 0) return ATTN_ERR_MASK;
+        if (c.algo == ATTN_ALGO_MATERIALIZED && a.mask && a.mask->kind == ATTN_MASK_BLOCK_SPARSE) return ATTN_ERR_MASK;
         if (!tc_cfg_supported(a.d, c, backward)) return ATTN_ERR_TILE;
         // fill defaults the way the kernels resolve them
         attn_cfg list[32];
@@ -96,7 +105,7 @@ attn_status layout(const Args &a, int backward, attn_cfg *cfg_out, WorkspaceLayo
         L->col_ptr = off; off += align_up(mh * 2 * nb * sizeof(int), 256);
         L->row_idx = off; off += align_up(mh * nb * nb * sizeof(int), 256);
     }
-    if (backward && c.algo == ATTN_ALGO_FUSED) { L->nLSE2 = off; off += align_up(BH * a.n * sizeof(float), 256); }
+    if (backward && (c.algo == ATTN_ALGO_FUSED || c.algo == ATTN_ALGO_MATERIALIZED)) { L->nLSE2 = off; off += align_up(BH * a.n * sizeof(float), 256); }
     if (backward && c.algo == ATTN_ALGO_FUSED && !c.deterministic) {
         L->dQ_acc = off; off += align_up(BH * a.n * a.d * sizeof(float), 256);
     }

@@ -69,5 +69,12 @@ def test_config5_full_block_sparse():
     run_full("C5", [17])
 
 
-def test_config4_forward_full():
-    run_full("C4", [0, 7], backward=False)
+@pytest.mark.parametrize("tile_k", [128, 64, 32])
+def test_config4_full_small_cache_regime_tile_sweep(tile_k):
+    """d = 256: fused forward, materialised (small-cache) backward, block edge swept over three values."""
+    import paper_2410_09397_b200 as attn
+    run_full("C4", [0, 7] if tile_k == 128 else [5], cfg=attn.Cfg(tile_k=tile_k, algo=attn.ATTN_ALGO_MATERIALIZED))
+
+
+def test_config4_full_default_cfg():
+    run_full("C4", [3])

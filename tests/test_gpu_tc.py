@@ -95,3 +95,33 @@ def test_large_scores_trigger_rescale():
     torch.cuda.synchronize()
     assert H.rel_err(H.to_np(O), O_ref) <= 2e-2
     assert H.rel_err(H.to_np(LSE), LSE_ref) <= 2e-2
+
+
+def materialized(tile_k=0):
+    from paper_2410_09397_b200 import binding as B
+    return B.Cfg(tile_k=tile_k, algo=B.ATTN_ALGO_MATERIALIZED)
+
+
+@pytest.mark.parametrize("tile_k", [128, 64, 32])
+@pytest.mark.parametrize("n,d", [(256, 256), (1000, 256), (384, 128), (200, 64)])
+@pytest.mark.parametrize("mask_kind", [inputs.MASK_NONE, inputs.MASK_CAUSAL])
+def test_materialized_backward(n, d, tile_k, mask_kind):
+    """Small-cache algorithm: P, dP, dS go through device memory; three tile sizes."""
+    errs = H.run_case(1, 2, n, d, "bf16", mask_kind, seed=38, cfg=materialized(tile_k))
+    H.assert_within(errs, "bf16")
+
+
+def test_materialized_rejects_block_sparse_and_auto_picks_it_for_d256():
+    import torch
+    import paper_2410_09397_b200 as attn
+    from paper_2410_09397_b200 import binding as B
+    bm = torch.ones(1, 2, 2, dtype=torch.uint8, device="cuda")
+    mask = attn.Mask(kind=attn.ATTN_MASK_BLOCK_SPARSE, block=128, block_mask=bm)
+    assert attn.attn_bwd_workspace_bytes(256, 256, 1, 1, mask, attn.ATTN_BF16, materialized()) == 0
+    attn.attn_timing_enable(True)
+    attn.attn_timing_collect()
+    errs = H.run_case(1, 1, 256, 256, "bf16", inputs.MASK_NONE, seed=39, check_bwd_only=False)
+    names = [k for k, _ in attn.attn_timing_collect()]
+    attn.attn_timing_enable(False)
+    H.assert_within(errs, "bf16")
+    assert "mat_phase1_P" in names and "mat_phase4_dQ" in names, names
