@@ -35,6 +35,7 @@ using namespace tc;
 constexpr int TQ = 128, TK = 128;
 constexpr int kSoftmaxThreads = 256;
 constexpr int kThreads = kSoftmaxThreads + 32;
+constexpr int kThreadsV2 = 512 + 32;   // pipelined d = 128 kernel: 16 softmax warps + issuer warp
 constexpr uint32_t SLAB = 128 * 128;   // bytes of one [128 rows][64 bf16] slab
 // dQ tile orientation at d = 128: transposed (lane = head-dimension index, coalesced scalar
 // reductions) or plain (lane = query, 16-byte vector reductions)
@@ -48,6 +49,7 @@ struct BwdArgs {
     int mask_kind, block, nb, mask_heads;
     const int *col_ptr, *row_idx;   // block-CSC of the mask
     float scale;
+    int group;                 // heads per launch group (divides BH)
     uint32_t *status;
 };
 
@@ -63,7 +65,7 @@ struct BwdSmem {
     static constexpr uint32_t oLSE = odS + 2 * SLAB;      // 2 stages x 128 floats
     static constexpr uint32_t oD = oLSE + 2 * 128 * 4;
     static constexpr uint32_t oBar = oD + 2 * 128 * 4;    // mbarriers (8 bytes each)
-    static constexpr uint32_t oMisc = oBar + 16 * 8;      // tmem base, abort flag
+    static constexpr uint32_t oMisc = oBar + 20 * 8;      // tmem base, abort flag
     static constexpr uint32_t kBytes = oMisc + 64;
     static_assert(kBytes <= 227 * 1024, "shared memory budget");
 };
@@ -177,8 +179,10 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
     const Abort ab{abort_flag, a.status};
 
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
-    const int jt = blockIdx.x;
-    const long bh = blockIdx.y;
+    // launch order: heads in groups of `a.group`, inside a group key tile major -- with a causal
+    // mask the CTAs of a group then start longest first, which evens out the tail of the grid
+    const int jt = blockIdx.x / a.group;
+    const long bh = (long)blockIdx.y * a.group + blockIdx.x % a.group;
     const int j0 = jt * TK, n = a.n;
 
     if ((smem_u32(smem) & 1023u) != 0) {   // operand tiles need 1024-byte alignment
@@ -490,6 +494,332 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
     if (warp == 0) tmem_dealloc(tm, 512);
 }
 
+// ---------------------------------------------------------------------------------------
+// d = 128, pipelined variant.  Same tiles, same shared-memory and tensor-memory layout as
+// tc_bwd_kernel, but every 128-query tile is handled as two independent halves of 64
+// queries (every barrier exists once per half) and sixteen warps share the exp / dS /
+// reduction work: warpgroups 2h and 2h+1 own the two 32-query quarters of half h, so
+// each scheduler has four warps to hide tensor-memory and MUFU latency.  The MMA issuer interleaves the two halves and issues
+// S^T of the next tile as soon as a half's dQ product is queued, so the tensor pipe keeps
+// running while the other half is in its exp / dS / reduction phase.
+enum { V2_KV = 0, V2_QFULL = 1, V2_QEMPTY = 3, V2_S = 5, V2_DP = 7, V2_P = 9, V2_DS = 11, V2_DQ = 13, V2_DQDONE = 15 };
+
+__global__ void __launch_bounds__(kThreadsV2, 1)
+tc_bwd_kernel_v2(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mK_,
+                 const __grid_constant__ CUtensorMap mV, const __grid_constant__ CUtensorMap mdO, const BwdArgs a)
+{
+    constexpr int HD = 128;
+    constexpr int kHalfThreads = 256;
+    using L = BwdSmem<HD>;
+    static_assert(L::oMisc - L::oBar >= 17 * 8, "barrier area");
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::oBar);
+    uint32_t *tmem_base_s = reinterpret_cast<uint32_t *>(smem + L::oMisc);
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(smem + L::oMisc + 4);
+    const Abort ab{abort_flag, a.status};
+
+    const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
+    // launch order: heads in groups of `a.group`, inside a group key tile major -- with a causal
+    // mask the CTAs of a group then start longest first, which evens out the tail of the grid
+    const int jt = blockIdx.x / a.group;
+    const long bh = (long)blockIdx.y * a.group + blockIdx.x % a.group;
+    const int j0 = jt * TK, n = a.n;
+
+    if ((smem_u32(smem) & 1023u) != 0) {
+        if (tid == 0) atomicExch(a.status, 9u);
+        return;
+    }
+    if (tid == 0) {
+        *abort_flag = 0;
+        mbar_init(&bars[V2_KV], 1);
+        for (int h = 0; h < 2; ++h) {
+            mbar_init(&bars[V2_QFULL + h], 1);
+            mbar_init(&bars[V2_QEMPTY + h], 1);
+            mbar_init(&bars[V2_S + h], 1);
+            mbar_init(&bars[V2_DP + h], 1);
+            mbar_init(&bars[V2_P + h], kHalfThreads);
+            mbar_init(&bars[V2_DS + h], kHalfThreads);
+            mbar_init(&bars[V2_DQ + h], 1);
+            mbar_init(&bars[V2_DQDONE + h], kHalfThreads);
+        }
+        fence_barrier_init();
+        prefetch_tensormap(&mQ); prefetch_tensormap(&mK_); prefetch_tensormap(&mV); prefetch_tensormap(&mdO);
+    }
+    if (warp == 0) tmem_alloc(tmem_base_s, 512);
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tm = *tmem_base_s;
+    const uint32_t T_S = tm, T_dP = tm + 128, T_dV = tm + 256, T_dK = tm + 256 + HD;
+    constexpr uint32_t HALF_ROWS = 64 * 128;   // byte offset of rows 64.. inside a [128][64] slab
+
+    const TileIter iter(a, jt, bh);
+
+    if (warp == 16) {
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = idesc_bf16(128, 128, 0, 0);       // S^T, dP^T (both halves at once)
+            constexpr uint32_t idesc_dv = idesc_bf16(128, HD, 0, 1);       // dV (A tmem), dK (A K-major smem)
+            constexpr uint32_t idesc_dq = idesc_bf16(128, 64, 1, 1);       // dQ^T half
+            // low descriptor words (tc_common.cuh): per-step offsets are added as (bytes >> 4)
+            const uint32_t kK = desc_lo_kmajor(smem_u32(smem + L::oK)), kV = desc_lo_kmajor(smem_u32(smem + L::oV));
+            const uint32_t mK = desc_lo_mnmajor(smem_u32(smem + L::oK), SLAB);
+            const uint32_t kdS = desc_lo_kmajor(smem_u32(smem + L::odS)), mdS = desc_lo_mnmajor(smem_u32(smem + L::odS), SLAB);
+            constexpr uint32_t kHalf = HALF_ROWS >> 4, kSlab = SLAB >> 4;
+            auto issue_load = [&](int it, int s) {
+                const int i0 = it * TQ;
+                const uint32_t rows = min(TQ, n - i0);
+                uint64_t *bar = &bars[V2_QFULL + s];
+                mbar_expect_tx(bar, 2 * L::kTile + 2 * rows * 4);
+#pragma unroll
+                for (uint32_t sl = 0; sl < L::kSlabs; ++sl) {
+                    tma_load_3d(smem + L::oQ + s * L::kTile + sl * SLAB, &mQ, bar, sl * 64, i0, (int)bh);
+                    tma_load_3d(smem + L::odO + s * L::kTile + sl * SLAB, &mdO, bar, sl * 64, i0, (int)bh);
+                }
+                bulk_load_1d(smem + L::oLSE + s * 512, a.nLSE2 + bh * n + i0, rows * 4, bar);
+                bulk_load_1d(smem + L::oD + s * 512, a.Ds + bh * n + i0, rows * 4, bar);
+            };
+            // S^T = K_j Q_i^T for the whole tile in stage s; one commit per half's barrier
+            auto issue_S = [&](int s) {
+                const uint32_t kQ = desc_lo_kmajor(smem_u32(smem + L::oQ + s * L::kTile));
+#pragma unroll
+                for (int kk = 0; kk < HD / 16; ++kk) {
+                    const uint32_t off = (kk / 4) * kSlab + (kk % 4) * 2;
+                    mma_ss_lo(T_S, kK + off, kQ + off, idesc_s, kk > 0);
+                }
+                mma_commit(&bars[V2_S]);
+                mma_commit(&bars[V2_S + 1]);
+            };
+            mbar_expect_tx(&bars[V2_KV], 2 * L::kTile);
+#pragma unroll
+            for (uint32_t sl = 0; sl < L::kSlabs; ++sl) {
+                tma_load_3d(smem + L::oK + sl * SLAB, &mK_, &bars[V2_KV], sl * 64, j0, (int)bh);
+                tma_load_3d(smem + L::oV + sl * SLAB, &mV, &bars[V2_KV], sl * 64, j0, (int)bh);
+            }
+            int idx = 0, it = -1;
+            while (idx < iter.raw && (it = iter.tile(idx)) < 0) ++idx;
+            if (it >= 0) {
+                issue_load(it, 0);
+                mbar_wait(&bars[V2_QFULL], 0, ab);
+                mbar_wait(&bars[V2_KV], 0, ab);
+                tcgen05_fence_after();
+                issue_S(0);
+            }
+            int k = 0;
+            while (idx < iter.raw) {
+                const int s = k & 1;
+                int nidx = idx + 1, nit = -1;
+                while (nidx < iter.raw && (nit = iter.tile(nidx)) < 0) ++nidx;
+                if (nit >= 0) {
+                    if (k >= 1) mbar_wait(&bars[V2_QEMPTY + (s ^ 1)], ((k - 1) >> 1) & 1, ab);
+                    issue_load(nit, s ^ 1);
+                }
+                const uint32_t sQa = smem_u32(smem + L::oQ + s * L::kTile), sdOa = smem_u32(smem + L::odO + s * L::kTile);
+                const uint32_t kdO = desc_lo_kmajor(sdOa), mdO_ = desc_lo_mnmajor(sdOa, SLAB), mQ_ = desc_lo_mnmajor(sQa, SLAB);
+                // dP^T = V_j dO_i^T once both halves of the previous dQ^T have left T_dP
+                if (k > 0) {
+                    mbar_wait(&bars[V2_DQDONE], (k - 1) & 1, ab);
+                    mbar_wait(&bars[V2_DQDONE + 1], (k - 1) & 1, ab);
+                    tcgen05_fence_after();
+                }
+#pragma unroll
+                for (int kk = 0; kk < HD / 16; ++kk) {
+                    const uint32_t off = (kk / 4) * kSlab + (kk % 4) * 2;
+                    mma_ss_lo(T_dP, kV + off, kdO + off, idesc_s, kk > 0);
+                }
+                mma_commit(&bars[V2_DP]);
+                mma_commit(&bars[V2_DP + 1]);
+                // dV += P_h^T dO_h
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    mbar_wait(&bars[V2_P + h], k & 1, ab);
+                    tcgen05_fence_after();
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        mma_ts_lo(T_dV, T_S + 64 * h + (kk < 2 ? kk * 8 : 48 + (kk - 2) * 8), mdO_ + h * kHalf + kk * 128,
+                                  idesc_dv, (k > 0) || (h > 0) || (kk > 0));
+                }
+                // T_S is free again: S^T of the next tile runs while this tile's dS is being formed
+                if (nit >= 0) {
+                    mbar_wait(&bars[V2_QFULL + (s ^ 1)], ((k + 1) >> 1) & 1, ab);
+                    tcgen05_fence_after();
+                    issue_S(s ^ 1);
+                }
+                // dK += dS_h^T Q_h ; dQ_h^T = K_j^T dS_h^T
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    mbar_wait(&bars[V2_DS + h], k & 1, ab);
+                    tcgen05_fence_after();
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        mma_ss_lo(T_dK, kdS + h * kSlab + kk * 2, mQ_ + h * kHalf + kk * 128, idesc_dv,
+                                  (k > 0) || (h > 0) || (kk > 0));
+#pragma unroll
+                    for (int kk = 0; kk < TK / 16; ++kk)
+                        mma_ss_lo(T_dP + 64 * h, mK + kk * 128, mdS + h * kSlab + kk * 128, idesc_dq, kk > 0);
+                    mma_commit(&bars[V2_DQ + h]);
+                }
+                mma_commit(&bars[V2_QEMPTY + s]);
+                ++k;
+                idx = nidx;
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ warpgroup 2h + qq owns queries 64 h + 32 qq .. + 31
+        const int h = warp / 8, qq = (warp / 4) & 1;
+        const int row = (warp % 4) * 32 + lane;        // tensor-memory lane = key row inside the tile
+        const uint32_t lane_addr = (uint32_t)((warp % 4) * 32) << 16;
+        const int jg = j0 + row;
+        const float sl2 = a.scale * 1.4426950408889634f;
+        int k = 0;
+        for (int idx = 0; idx < iter.raw; ++idx) {
+            const int it = iter.tile(idx);
+            if (it < 0) continue;
+            const int s = k & 1, i0 = it * TQ;
+            const float4 *sNL = reinterpret_cast<const float4 *>(smem + L::oLSE + s * 512 + h * 256 + qq * 128);
+            const float4 *sDs = reinterpret_cast<const float4 *>(smem + L::oD + s * 512 + h * 256 + qq * 128);
+            const bool diag = a.mask_kind == ATTN_MASK_CAUSAL && it == jt;
+            const bool masked = diag || i0 + TQ > n || j0 + TK > n;
+            const int ig0 = i0 + h * 64 + qq * 32;
+            const uint32_t c0 = h * 64 + qq * 32;      // this thread's first column in T_S / T_dP
+            mbar_wait(&bars[V2_QFULL + s], (k >> 1) & 1, ab);
+            mbar_wait(&bars[V2_S + h], k & 1, ab);
+            tcgen05_fence_after();
+            float p[32];
+            {
+                uint32_t sv0[32];
+                tmem_ld32(T_S + lane_addr + c0, sv0);
+                tmem_wait_ld();
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const float4 nl = sNL[q];
+                    const uint32_t *sv = &sv0[q * 4];
+                    p[q * 4 + 0] = ex2_approx(fmaf(__uint_as_float(sv[0]), sl2, nl.x));
+                    p[q * 4 + 1] = ex2_approx(fmaf(__uint_as_float(sv[1]), sl2, nl.y));
+                    p[q * 4 + 2] = ex2_approx(fmaf(__uint_as_float(sv[2]), sl2, nl.z));
+                    p[q * 4 + 3] = ex2_approx(fmaf(__uint_as_float(sv[3]), sl2, nl.w));
+                }
+            }
+            if (masked) {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                    const int ig = ig0 + e;
+                    const bool ok = ig < n && jg < n && (!diag || jg <= ig);
+                    p[e] = ok ? p[e] : 0.f;
+                }
+            }
+            {
+                // P^T (bf16 pairs) goes over columns this very thread has just read -- quarter 0
+                // to columns 0..15 of the half, quarter 1 to columns 48..63 -- so no thread
+                // overwrites S^T entries another thread still has to read
+                uint32_t ppack[16];
+#pragma unroll
+                for (int e = 0; e < 16; ++e) ppack[e] = pack_bf16(p[2 * e], p[2 * e + 1]);
+                tmem_st16(T_S + lane_addr + h * 64 + qq * 48, ppack);
+                tmem_wait_st();
+            }
+            tcgen05_fence_before();
+            mbar_arrive(&bars[V2_P + h]);
+
+            mbar_wait(&bars[V2_DP + h], k & 1, ab);
+            tcgen05_fence_after();
+            {
+                uint32_t dv0[32];
+                tmem_ld32(T_dP + lane_addr + c0, dv0);
+                tmem_wait_ld();
+                uint8_t *slab = smem + L::odS + h * SLAB;
+#pragma unroll
+                for (int q8 = 0; q8 < 4; ++q8) {
+                    float ds[8];
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        const int q = q8 * 2 + u;
+                        const float4 dsc = sDs[q];
+                        const uint32_t *dv = &dv0[q * 4];
+                        ds[u * 4 + 0] = p[q * 4 + 0] * fmaf(__uint_as_float(dv[0]), a.scale, -dsc.x);
+                        ds[u * 4 + 1] = p[q * 4 + 1] * fmaf(__uint_as_float(dv[1]), a.scale, -dsc.y);
+                        ds[u * 4 + 2] = p[q * 4 + 2] * fmaf(__uint_as_float(dv[2]), a.scale, -dsc.z);
+                        ds[u * 4 + 3] = p[q * 4 + 3] * fmaf(__uint_as_float(dv[3]), a.scale, -dsc.w);
+                    }
+                    if (masked) {
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) ds[e] = p[q8 * 8 + e] != 0.f ? ds[e] : 0.f;
+                    }
+                    *reinterpret_cast<uint4 *>(slab + sw128_offset(row, qq * 32 + q8 * 8)) =
+                        make_uint4(pack_bf16(ds[0], ds[1]), pack_bf16(ds[2], ds[3]), pack_bf16(ds[4], ds[5]),
+                                   pack_bf16(ds[6], ds[7]));
+                }
+            }
+            fence_proxy_async_smem();
+            tcgen05_fence_before();
+            mbar_arrive(&bars[V2_DS + h]);
+
+            mbar_wait(&bars[V2_DQ + h], k & 1, ab);
+            tcgen05_fence_after();
+            {
+                float *base = a.dQ_acc + ((size_t)bh * n + ig0) * HD + row;
+                uint32_t v0[32];
+                tmem_ld32(T_dP + lane_addr + c0, v0);
+                tmem_wait_ld();
+                tcgen05_fence_before();
+                mbar_arrive(&bars[V2_DQDONE + h]);
+                if (!masked || i0 + TQ <= n) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) red_add_f32(base + (size_t)e * HD, __uint_as_float(v0[e]));
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        if (ig0 + e < n) red_add_f32(base + (size_t)e * HD, __uint_as_float(v0[e]));
+                }
+            }
+            ++k;
+        }
+        // ------------------------------------------------------------ epilogue: dV_j, dK_j (32 columns per warpgroup)
+        if (k > 0) {
+            // both halves' last products must have landed, not only this warpgroup's own
+            mbar_wait(&bars[V2_DQ + (h ^ 1)], (k - 1) & 1, ab);
+            tcgen05_fence_after();
+        }
+        {
+            constexpr int HALF = 32;
+            const int cq = (warp / 4) * 32;
+            const int jc = jg < n ? jg : 0;
+            __nv_bfloat16 *pv = a.dV + ((size_t)bh * n + jc) * HD + cq;
+            __nv_bfloat16 *pk = a.dK + ((size_t)bh * n + jc) * HD + cq;
+#pragma unroll
+            for (int c = 0; c < HALF; c += 32) {
+                uint32_t v[32], w[32];
+                if (k > 0) {
+                    tmem_ld32(T_dV + lane_addr + cq + c, v);
+                    tmem_ld32(T_dK + lane_addr + cq + c, w);
+                    tmem_wait_ld();
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) v[e] = w[e] = 0u;
+                }
+                if (jg < n) {
+#pragma unroll
+                    for (int e = 0; e < 32; e += 8) {
+                        uint4 ov, ok;
+                        ov.x = pack_bf16(__uint_as_float(v[e]), __uint_as_float(v[e + 1]));
+                        ov.y = pack_bf16(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
+                        ov.z = pack_bf16(__uint_as_float(v[e + 4]), __uint_as_float(v[e + 5]));
+                        ov.w = pack_bf16(__uint_as_float(v[e + 6]), __uint_as_float(v[e + 7]));
+                        ok.x = pack_bf16(__uint_as_float(w[e]), __uint_as_float(w[e + 1]));
+                        ok.y = pack_bf16(__uint_as_float(w[e + 2]), __uint_as_float(w[e + 3]));
+                        ok.z = pack_bf16(__uint_as_float(w[e + 4]), __uint_as_float(w[e + 5]));
+                        ok.w = pack_bf16(__uint_as_float(w[e + 6]), __uint_as_float(w[e + 7]));
+                        *reinterpret_cast<uint4 *>(pv + c + e) = ov;
+                        *reinterpret_cast<uint4 *>(pk + c + e) = ok;
+                    }
+                }
+            }
+        }
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tm, 512);
+}
+
 // fp32 accumulator -> bf16 dQ
 __global__ void __launch_bounds__(256) dq_convert_kernel(const float4 *__restrict__ acc, uint2 *__restrict__ out, size_t n4)
 {
@@ -516,6 +846,7 @@ attn_status launch_bwd(const Problem &p)
     a.col_ptr = p.col_ptr; a.row_idx = p.row_idx;
     a.scale = p.scale;
     a.status = p.status;
+    a.group = p.BH % 8 == 0 ? 8 : p.BH % 4 == 0 ? 4 : p.BH % 2 == 0 ? 2 : 1;
     auto kernel = tc_bwd_kernel<HD>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::kBytes) != cudaSuccess)
         return ATTN_ERR_LAUNCH;
@@ -532,9 +863,15 @@ attn_status launch_bwd(const Problem &p)
         launch_end(p.stream);
         if (cudaGetLastError() != cudaSuccess) return ATTN_ERR_LAUNCH;
     }
-    const dim3 grid((p.n + TK - 1) / TK, (unsigned)p.BH);
+    const dim3 grid((unsigned)((p.n + TK - 1) / TK * a.group), (unsigned)(p.BH / a.group));
     launch_begin("tc_bwd_fused", p.stream);
-    kernel<<<grid, kThreads, L::kBytes, p.stream>>>(mQ, mK, mV, mdO, a);
+    if (HD == 128) {
+        if (cudaFuncSetAttribute(tc_bwd_kernel_v2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::kBytes) != cudaSuccess)
+            return ATTN_ERR_LAUNCH;
+        tc_bwd_kernel_v2<<<grid, kThreadsV2, L::kBytes, p.stream>>>(mQ, mK, mV, mdO, a);
+    } else {
+        kernel<<<grid, kThreads, L::kBytes, p.stream>>>(mQ, mK, mV, mdO, a);
+    }
     launch_end(p.stream);
     if (cudaGetLastError() != cudaSuccess) return ATTN_ERR_LAUNCH;
     const size_t n4 = acc_elems / 4;
