@@ -235,8 +235,8 @@ def workload_name(w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C3", choices=sorted(inputs.WORKLOADS))
     ap.add_argument("--algo", default="auto", choices=["auto", "fused", "materialized", "simt"])
@@ -317,6 +317,9 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    if rank == 0:
+        sampler.start()   # nvidia-smi needs a moment to come up: start it before the warm-up
     for _ in range(args.warmup):
         fwd()
         bwd()
@@ -329,10 +332,7 @@ def main():
     attn.attn_timing_enable(True)
     attn.attn_timing_collect()
     launches0 = attn.attn_kernel_launches()
-    sampler = ClockSampler(physical_gpu_index(local_rank))
     kernel_ms: dict[str, list[float]] = {}
-    if rank == 0:
-        sampler.start()
     barrier()
     t_wall = time.perf_counter()
     for s in range(args.steps):
