@@ -54,6 +54,7 @@ attn_status build_block_index(const Problem &p);
 // Tensor-core path (attn_tc_*.cu)
 attn_status tc_fwd(const Problem &p);
 attn_status tc_bwd(const Problem &p);
+attn_status tc_bwd_dq(const Problem &p);   // query-stationary dQ without atomics (needs p.D = scale*D, p.nLSE2)
 attn_status mat_bwd(const Problem &p);
 bool tc_cfg_supported(int d, const attn_cfg &cfg, int backward);
 size_t tc_cfg_onchip_bytes(int d, const attn_cfg &cfg, int backward);

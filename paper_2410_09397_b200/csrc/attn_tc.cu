@@ -15,7 +15,6 @@ bool tc_cfg_supported(int d, const attn_cfg &c, int backward)
         if (c.tile_q != 0 && c.tile_q != 128) return false;
         if (backward) {
             if (d == 256) return false;
-            if (c.deterministic) return false;   // the fused backward reduces dQ with floating-point atomics
             return c.tile_k == 0 || c.tile_k == 128;
         }
         const int tk = d == 256 ? 64 : 128;

@@ -166,7 +166,9 @@ __global__ void __launch_bounds__(256) tc_preprocess_kernel(const __nv_bfloat16 
     }
 }
 
-template <int HD>
+// WITH_DQ = false leaves the dQ product and its reductions out (dK and dV only): the
+// deterministic path computes dQ in a kernel of its own (attn_tc_bwd_dq.cu).
+template <int HD, bool WITH_DQ>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mK,
               const __grid_constant__ CUtensorMap mV, const __grid_constant__ CUtensorMap mdO, const BwdArgs a)
@@ -270,7 +272,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
                     issue_load(nit, s ^ 1);
                 }
                 const uint32_t sQ = smem_u32(smem + L::oQ + s * L::kTile), sdO = smem_u32(smem + L::odO + s * L::kTile);
-                if (k > 0) {   // the dQ tile of the previous pair has been read out of T_dP
+                if (WITH_DQ && k > 0) {   // the dQ tile of the previous pair has been read out of T_dP
                     mbar_wait(&bars[BAR_DQDONE], (k - 1) & 1, ab);
                     tcgen05_fence_after();
                 }
@@ -297,7 +299,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
                            (k > 0) || (kk > 0));
                 }
 #pragma unroll
-                for (int kk = 0; kk < TK / 16; ++kk) {
+                for (int kk = 0; WITH_DQ && kk < TK / 16; ++kk) {
                     if (kDqT)        // dQ^T = K_j^T dS^T : A = K_j MN-major, B = dS^T MN-major
                         mma_ss(T_dP, smem_desc_mnmajor(sK + kk * 2048, SLAB), smem_desc_mnmajor(sdS + kk * 2048, SLAB),
                                idesc_dq, kk > 0);
@@ -408,6 +410,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
             mbar_arrive(&bars[BAR_DS]);
 
             // ---- dQ tile: read out of tensor memory and reduce into the fp32 accumulator
+            if (WITH_DQ) {
             mbar_wait(&bars[BAR_DQ], k & 1, ab);
             tcgen05_fence_after();
             if (kDqT) {
@@ -450,10 +453,15 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
                                    __uint_as_float(v[e + 3]));
                 }
             }
+            }
             ++k;
         }
         // ------------------------------------------------------------ epilogue: dV_j, dK_j
         // (the last BAR_DQ phase also covers the last dV / dK accumulation; dS carried the scale)
+        if (!WITH_DQ && k > 0) {
+            mbar_wait(&bars[BAR_DQ], (k - 1) & 1, ab);
+            tcgen05_fence_after();
+        }
         {
             constexpr int HALF = HD / 2;
             const int jc = jg < n ? jg : 0;   // rows past n take part in the warp-wide loads but store nothing
@@ -504,6 +512,7 @@ tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
 // running while the other half is in its exp / dS / reduction phase.
 enum { V2_KV = 0, V2_QFULL = 1, V2_QEMPTY = 3, V2_S = 5, V2_DP = 7, V2_P = 9, V2_DS = 11, V2_DQ = 13, V2_DQDONE = 15 };
 
+template <bool WITH_DQ>
 __global__ void __launch_bounds__(kThreadsV2, 1)
 tc_bwd_kernel_v2(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mK_,
                  const __grid_constant__ CUtensorMap mV, const __grid_constant__ CUtensorMap mdO, const BwdArgs a)
@@ -616,7 +625,7 @@ tc_bwd_kernel_v2(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
                 const uint32_t sQa = smem_u32(smem + L::oQ + s * L::kTile), sdOa = smem_u32(smem + L::odO + s * L::kTile);
                 const uint32_t kdO = desc_lo_kmajor(sdOa), mdO_ = desc_lo_mnmajor(sdOa, SLAB), mQ_ = desc_lo_mnmajor(sQa, SLAB);
                 // dP^T = V_j dO_i^T once both halves of the previous dQ^T have left T_dP
-                if (k > 0) {
+                if (WITH_DQ && k > 0) {
                     mbar_wait(&bars[V2_DQDONE], (k - 1) & 1, ab);
                     mbar_wait(&bars[V2_DQDONE + 1], (k - 1) & 1, ab);
                     tcgen05_fence_after();
@@ -654,7 +663,7 @@ tc_bwd_kernel_v2(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
                         mma_ss_lo(T_dK, kdS + h * kSlab + kk * 2, mQ_ + h * kHalf + kk * 128, idesc_dv,
                                   (k > 0) || (h > 0) || (kk > 0));
 #pragma unroll
-                    for (int kk = 0; kk < TK / 16; ++kk)
+                    for (int kk = 0; WITH_DQ && kk < TK / 16; ++kk)
                         mma_ss_lo(T_dP + 64 * h, mK + kk * 128, mdS + h * kSlab + kk * 128, idesc_dq, kk > 0);
                     mma_commit(&bars[V2_DQ + h]);
                 }
@@ -753,6 +762,7 @@ tc_bwd_kernel_v2(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
             tcgen05_fence_before();
             mbar_arrive(&bars[V2_DS + h]);
 
+            if (WITH_DQ) {
             mbar_wait(&bars[V2_DQ + h], k & 1, ab);
             tcgen05_fence_after();
             {
@@ -771,11 +781,13 @@ tc_bwd_kernel_v2(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
                         if (ig0 + e < n) red_add_f32(base + (size_t)e * HD, __uint_as_float(v0[e]));
                 }
             }
+            }
             ++k;
         }
         // ------------------------------------------------------------ epilogue: dV_j, dK_j (32 columns per warpgroup)
         if (k > 0) {
             // both halves' last products must have landed, not only this warpgroup's own
+            mbar_wait(&bars[V2_DQ + h], (k - 1) & 1, ab);
             mbar_wait(&bars[V2_DQ + (h ^ 1)], (k - 1) & 1, ab);
             tcgen05_fence_after();
         }
@@ -829,7 +841,7 @@ __global__ void __launch_bounds__(256) dq_convert_kernel(const float4 *__restric
     }
 }
 
-template <int HD>
+template <int HD, bool WITH_DQ>
 attn_status launch_bwd(const Problem &p)
 {
     using L = BwdSmem<HD>;
@@ -847,11 +859,11 @@ attn_status launch_bwd(const Problem &p)
     a.scale = p.scale;
     a.status = p.status;
     a.group = p.BH % 8 == 0 ? 8 : p.BH % 4 == 0 ? 4 : p.BH % 2 == 0 ? 2 : 1;
-    auto kernel = tc_bwd_kernel<HD>;
+    auto kernel = tc_bwd_kernel<HD, WITH_DQ>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::kBytes) != cudaSuccess)
         return ATTN_ERR_LAUNCH;
     const size_t acc_elems = (size_t)p.BH * p.n * HD;
-    if (cudaMemsetAsync(p.dQ_acc, 0, acc_elems * sizeof(float), p.stream) != cudaSuccess) return ATTN_ERR_LAUNCH;
+    if (WITH_DQ && cudaMemsetAsync(p.dQ_acc, 0, acc_elems * sizeof(float), p.stream) != cudaSuccess) return ATTN_ERR_LAUNCH;
     {
         const size_t rows = (size_t)p.BH * p.n;
         constexpr size_t rpw = 32 / (HD / 8);
@@ -864,16 +876,17 @@ attn_status launch_bwd(const Problem &p)
         if (cudaGetLastError() != cudaSuccess) return ATTN_ERR_LAUNCH;
     }
     const dim3 grid((unsigned)((p.n + TK - 1) / TK * a.group), (unsigned)(p.BH / a.group));
-    launch_begin("tc_bwd_fused", p.stream);
+    launch_begin(WITH_DQ ? "tc_bwd_fused" : "tc_bwd_dkdv", p.stream);
     if (HD == 128) {
-        if (cudaFuncSetAttribute(tc_bwd_kernel_v2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::kBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(tc_bwd_kernel_v2<WITH_DQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::kBytes) != cudaSuccess)
             return ATTN_ERR_LAUNCH;
-        tc_bwd_kernel_v2<<<grid, kThreadsV2, L::kBytes, p.stream>>>(mQ, mK, mV, mdO, a);
+        tc_bwd_kernel_v2<WITH_DQ><<<grid, kThreadsV2, L::kBytes, p.stream>>>(mQ, mK, mV, mdO, a);
     } else {
         kernel<<<grid, kThreads, L::kBytes, p.stream>>>(mQ, mK, mV, mdO, a);
     }
     launch_end(p.stream);
     if (cudaGetLastError() != cudaSuccess) return ATTN_ERR_LAUNCH;
+    if (!WITH_DQ) return tc_bwd_dq(p);   // deterministic path: dQ without atomics, from its own kernel
     const size_t n4 = acc_elems / 4;
     const unsigned blocks = (unsigned)((n4 + 255) / 256 < 148 * 16 ? (n4 + 255) / 256 : 148 * 16);
     launch_begin("bwd_dq_convert", p.stream);
@@ -888,8 +901,8 @@ size_t bwd_smem_bytes(int d) { return d == 64 ? BwdSmem<64>::kBytes : d == 128 ?
 
 attn_status tc_bwd(const Problem &p)
 {
-    if (p.d == 64) return launch_bwd<64>(p);
-    if (p.d == 128) return launch_bwd<128>(p);
+    if (p.d == 64) return p.cfg.deterministic ? launch_bwd<64, false>(p) : launch_bwd<64, true>(p);
+    if (p.d == 128) return p.cfg.deterministic ? launch_bwd<128, false>(p) : launch_bwd<128, true>(p);
     return ATTN_ERR_TILE;
 }
 

@@ -125,3 +125,34 @@ def test_materialized_rejects_block_sparse_and_auto_picks_it_for_d256():
     attn.attn_timing_enable(False)
     H.assert_within(errs, "bf16")
     assert "mat_phase1_P" in names and "mat_phase4_dQ" in names, names
+
+
+def fused_det():
+    from paper_2410_09397_b200 import binding as B
+    return B.Cfg(algo=B.ATTN_ALGO_FUSED, deterministic=1)
+
+
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("n", [128, 640, 1000])
+@pytest.mark.parametrize("mask_kind", [inputs.MASK_NONE, inputs.MASK_CAUSAL, inputs.MASK_BLOCK_SPARSE])
+def test_deterministic_backward_without_atomics(n, d, mask_kind):
+    """deterministic = 1: dK, dV from the key-stationary kernel, dQ from the query-stationary one."""
+    errs = H.run_case(1, 2, n, d, "bf16", mask_kind, seed=40, block=128, cfg=fused_det())
+    H.assert_within(errs, "bf16")
+
+
+def test_deterministic_backward_is_bitwise_repeatable():
+    import torch
+    import paper_2410_09397_b200 as attn
+    x = H.make_inputs(41, 2, 2, 768, 128, "bf16")
+    dev = {k: H.to_dev(v, "bf16") for k, v in x.items()}
+    mask = attn.Mask(kind=attn.ATTN_MASK_CAUSAL)
+    O, LSE = attn.attn_fwd(dev["Q"], dev["K"], dev["V"], mask=mask, cfg=fused_det())
+    runs = []
+    for _ in range(3):
+        g = attn.attn_bwd(dev["Q"], dev["K"], dev["V"], O, dev["dO"], LSE, mask=mask, cfg=fused_det())
+        torch.cuda.synchronize()
+        runs.append([t.clone() for t in g])
+    for other in runs[1:]:
+        for a, b in zip(runs[0], other):
+            assert torch.equal(a, b)
