@@ -445,7 +445,11 @@ def main():
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu
 # captures summarised under profiles/, keyed by (kernel, workload); absent = not measured
 # for the kernel as it stands.
-TRAFFIC: dict = {}
+TRAFFIC: dict = {
+    # profiles/tc_bwd_fused_C3.md: 294.0 MB on the 16-head case; the full workload has 32 heads and the
+    # traffic grows with the number of heads (heads are independent)
+    ("tc_bwd_fused", "C3"): 588.0e6,
+}
 
 
 if __name__ == "__main__":
