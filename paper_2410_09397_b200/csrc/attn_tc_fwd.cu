@@ -95,6 +95,12 @@ struct KeyIter {
     }
 };
 
+__device__ __forceinline__ float ex2_fast_f(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 __device__ __forceinline__ void named_bar_sync_f(int id, int count)
 {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
@@ -176,16 +182,16 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
         if (lane == 0 && niter > 0) {
             constexpr uint32_t idesc_s = idesc_bf16(128, TKF, 0, 0);
             constexpr uint32_t idesc_o = idesc_bf16(128, HD, 0, 1);
-            const uint32_t sQ = smem_u32(smem + C::oQ);
+            const uint32_t kQ = desc_lo_kmajor(smem_u32(smem + C::oQ));
             auto issue_S = [&](int k) {
                 const int s = k % NST;
                 mbar_wait(&bars[FB_KVFULL + s], (k / NST) & 1, ab);
                 tcgen05_fence_after();
-                const uint32_t sK = smem_u32(smem + C::oK + s * C::kKTile);
+                const uint32_t kK = desc_lo_kmajor(smem_u32(smem + C::oK + s * C::kKTile));
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk)
-                    mma_ss(tm + (k & 1) * 128, smem_desc_kmajor(sQ + (kk / 4) * C::kQSlab + (kk % 4) * 32),
-                           smem_desc_kmajor(sK + (kk / 4) * C::kKSlab + (kk % 4) * 32), idesc_s, kk > 0);
+                    mma_ss_lo(tm + (k & 1) * 128, kQ + (kk / 4) * (C::kQSlab >> 4) + (kk % 4) * 2,
+                              kK + (kk / 4) * (C::kKSlab >> 4) + (kk % 4) * 2, idesc_s, kk > 0);
                 mma_commit(&bars[FB_S + (k & 1)]);
             };
             mbar_wait(&bars[FB_Q], 0, ab);
@@ -195,11 +201,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
                 const int s = k % NST, b = k & 1;
                 mbar_wait(&bars[FB_P + b], (k >> 1) & 1, ab);
                 tcgen05_fence_after();
-                const uint32_t sV = smem_u32(smem + C::oV + s * C::kKTile);
+                const uint32_t mV_ = desc_lo_mnmajor(smem_u32(smem + C::oV + s * C::kKTile), C::kKSlab);
 #pragma unroll
                 for (int kk = 0; kk < TKF / 16; ++kk)
-                    mma_ts(T_O, tm + b * 128 + kk * 8, smem_desc_mnmajor(sV + kk * 2048, C::kKSlab), idesc_o,
-                           (k > 0) || (kk > 0));
+                    mma_ts_lo(T_O, tm + b * 128 + kk * 8, mV_ + kk * 128, idesc_o, (k > 0) || (kk > 0));
                 mma_commit(&bars[FB_KVEMPTY + s]);
                 mma_commit(&bars[FB_O]);
             }
@@ -227,7 +232,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
                 tmem_ld32(T_S + lane_addr + wg * CW + c, v);
                 tmem_wait_ld();
 #pragma unroll
-                for (int e = 0; e < 32; ++e) sv[c + e] = __uint_as_float(v[e]) * sl2;
+                for (int e = 0; e < 32; ++e) sv[c + e] = __uint_as_float(v[e]);   // raw scores; scale * log2e enters below
             }
             const bool need_mask = (a.mask_kind == ATTN_MASK_CAUSAL && j0 + TKF - 1 > i0) || j0 + TKF > n;
             float mx = -INFINITY;
@@ -244,11 +249,11 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
             float *xm = xmax + b * 256;
             xm[wg * 128 + row] = mx;
             named_bar_sync_f(1, kSoftmaxThreads);   // also: every S read of this tile is done
-            const float m_tile = fmaxf(xm[row], xm[128 + row]);
+            const float m_tile = fmaxf(xm[row], xm[128 + row]) * sl2;   // scale > 0: the maximum commutes with it
             const bool need = m_tile > m_ref + kRescaleThreshold || (m_ref == -INFINITY && m_tile != -INFINITY);
             if (__any_sync(0xffffffffu, need)) {
                 const float m_new = need ? fmaxf(m_ref, m_tile) : m_ref;
-                const float alpha = (need && m_ref != -INFINITY) ? exp2f(m_ref - m_new) : 1.f;
+                const float alpha = (need && m_ref != -INFINITY) ? ex2_fast_f(m_ref - m_new) : 1.f;
                 if (k > 0) {
                     mbar_wait(&bars[FB_O], (k - 1) & 1, ab);   // O += P V of the previous tile has landed
                     tcgen05_fence_after();
@@ -265,12 +270,12 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
                 l_part *= alpha;
                 m_ref = m_new;
             }
-            const float off = m_ref == -INFINITY ? 0.f : m_ref;
+            const float noff = m_ref == -INFINITY ? 0.f : -m_ref;
             uint32_t pp[CW / 2];
             float rs = 0.f;
 #pragma unroll
             for (int e = 0; e < CW; e += 2) {
-                const float p0 = exp2f(sv[e] - off), p1 = exp2f(sv[e + 1] - off);
+                const float p0 = ex2_fast_f(fmaf(sv[e], sl2, noff)), p1 = ex2_fast_f(fmaf(sv[e + 1], sl2, noff));
                 rs += p0 + p1;
                 pp[e / 2] = pack_bf16(p0, p1);
             }
