@@ -12,8 +12,9 @@
 //
 // S and dP are recomputed here (the key-stationary kernel computes them too), which is
 // the price of summing dQ in a fixed order: 7 products instead of 5 per tile pair.
-// Roles as in the forward: warps 0-7 split the key columns, warp 8 lane 0 issues MMAs,
-// warp 9 lane 0 runs TMA.  Tensor memory: S0 128, S1 128, dP 128, dQ d columns.
+// Roles: warps 0-15 = four warpgroups, warpgroup g owning key columns 32 g .. 32 g + 31 of every
+// tile (no barrier couples them, so their exp, dS and tensor-memory phases interleave freely);
+// warp 16 lane 0 issues MMAs, warp 17 lane 0 runs TMA.  Tensor memory: S0 128, S1 128, dP 128, dQ d columns.
 #include "attn_internal.h"
 #include "tc_common.cuh"
 
@@ -23,7 +24,7 @@ namespace {
 using namespace tc;
 
 constexpr int TQ = 128, TKD = 128;
-constexpr int kSoftmaxThreads = 256;
+constexpr int kSoftmaxThreads = 512;
 constexpr int kThreads = kSoftmaxThreads + 64;
 constexpr uint32_t SLAB = 128 * 128;
 
@@ -39,21 +40,22 @@ struct DqArgs {
 
 template <int HD>
 struct DqSmem {
-    static constexpr int NST = 2;
+    static constexpr int NSTK = 3, NSTV = 2;   // K_j is needed first (S) and released last (dQ): three stages; V_j: two
     static constexpr uint32_t kSlabs = HD / 64;
     static constexpr uint32_t kTile = kSlabs * SLAB;     // one [128][HD] bf16 tile
     static constexpr uint32_t oQ = 0;
     static constexpr uint32_t odO = oQ + kTile;
-    static constexpr uint32_t oK = odO + kTile;          // NST stages
-    static constexpr uint32_t oV = oK + NST * kTile;     // NST stages
-    static constexpr uint32_t oBar = oV + NST * kTile;
-    static constexpr uint32_t oMisc = oBar + 16 * 8;
+    static constexpr uint32_t oK = odO + kTile;          // NSTK stages
+    static constexpr uint32_t oV = oK + NSTK * kTile;    // NSTV stages
+    static constexpr uint32_t oBar = oV + NSTV * kTile;
+    static constexpr uint32_t oMisc = oBar + 24 * 8;
     static constexpr uint32_t kUsed = oMisc + 64;
     static constexpr uint32_t kBytes = kUsed < 117 * 1024 ? 117 * 1024 : kUsed;   // one CTA per SM (512 TMEM columns)
     static_assert(kUsed <= 227 * 1024, "shared memory budget");
 };
 
-enum { DB_Q = 0, DB_KVFULL = 1, DB_KVEMPTY = 3, DB_S = 5, DB_DP = 7, DB_DPFREE = 8, DB_DS = 9, DB_DQ = 11 };
+enum { DB_Q = 0, DB_KFULL = 1, DB_KEMPTY = 4, DB_VFULL = 7, DB_VEMPTY = 9, DB_S = 11, DB_DP = 13, DB_DPFREE = 14, DB_DS = 15,
+       DB_DQ = 17 };
 
 struct KeyIterD {
     int kind, n, sub, raw;
@@ -92,7 +94,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
                  const __grid_constant__ CUtensorMap mV, const __grid_constant__ CUtensorMap mdO, const DqArgs a)
 {
     using L = DqSmem<HD>;
-    constexpr int NST = L::NST;
+    constexpr int NSTK = L::NSTK, NSTV = L::NSTV;
     extern __shared__ __align__(1024) uint8_t smem[];
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::oBar);
     uint32_t *tmem_base_s = reinterpret_cast<uint32_t *>(smem + L::oMisc);
@@ -112,7 +114,8 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
     if (tid == 0) {
         *abort_flag = 0;
         mbar_init(&bars[DB_Q], 1);
-        for (int s = 0; s < NST; ++s) { mbar_init(&bars[DB_KVFULL + s], 1); mbar_init(&bars[DB_KVEMPTY + s], 1); }
+        for (int s = 0; s < NSTK; ++s) { mbar_init(&bars[DB_KFULL + s], 1); mbar_init(&bars[DB_KEMPTY + s], 1); }
+        for (int s = 0; s < NSTV; ++s) { mbar_init(&bars[DB_VFULL + s], 1); mbar_init(&bars[DB_VEMPTY + s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&bars[DB_S + b], 1); mbar_init(&bars[DB_DS + b], kSoftmaxThreads); }
         mbar_init(&bars[DB_DP], 1);
         mbar_init(&bars[DB_DPFREE], kSoftmaxThreads);
@@ -130,7 +133,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
     int niter = 0;
     for (int idx = 0; idx < iter.raw; ++idx) niter += iter.tile(idx) >= 0;
 
-    if (warp == 9) {
+    if (warp == 17) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             mbar_expect_tx(&bars[DB_Q], 2 * L::kTile);
@@ -143,20 +146,22 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
             for (int idx = 0; idx < iter.raw; ++idx) {
                 const int jt = iter.tile(idx);
                 if (jt < 0) continue;
-                const int s = k % NST;
-                if (k >= NST) mbar_wait(&bars[DB_KVEMPTY + s], ((k / NST) - 1) & 1, ab);
-                uint64_t *bar = &bars[DB_KVFULL + s];
-                mbar_expect_tx(bar, 2 * L::kTile);
+                const int sk = k % NSTK, sv = k % NSTV;
+                if (k >= NSTK) mbar_wait(&bars[DB_KEMPTY + sk], ((k / NSTK) - 1) & 1, ab);
+                mbar_expect_tx(&bars[DB_KFULL + sk], L::kTile);
 #pragma unroll
-                for (uint32_t sl = 0; sl < L::kSlabs; ++sl) {
-                    tma_load_3d(smem + L::oK + s * L::kTile + sl * SLAB, &mK, bar, sl * 64, jt * TKD, (int)bh);
-                    tma_load_3d(smem + L::oV + s * L::kTile + sl * SLAB, &mV, bar, sl * 64, jt * TKD, (int)bh);
-                }
+                for (uint32_t sl = 0; sl < L::kSlabs; ++sl)
+                    tma_load_3d(smem + L::oK + sk * L::kTile + sl * SLAB, &mK, &bars[DB_KFULL + sk], sl * 64, jt * TKD, (int)bh);
+                if (k >= NSTV) mbar_wait(&bars[DB_VEMPTY + sv], ((k / NSTV) - 1) & 1, ab);
+                mbar_expect_tx(&bars[DB_VFULL + sv], L::kTile);
+#pragma unroll
+                for (uint32_t sl = 0; sl < L::kSlabs; ++sl)
+                    tma_load_3d(smem + L::oV + sv * L::kTile + sl * SLAB, &mV, &bars[DB_VFULL + sv], sl * 64, jt * TKD, (int)bh);
                 ++k;
             }
             if (niter == 0) mbar_wait(&bars[DB_Q], 0, ab);   // let the Q / dO load land before exit
         }
-    } else if (warp == 8) {
+    } else if (warp == 16) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0 && niter > 0) {
             constexpr uint32_t idesc_s = idesc_bf16(128, 128, 0, 0);
@@ -164,8 +169,8 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
             constexpr uint32_t kSlab = SLAB >> 4;
             const uint32_t kQ = desc_lo_kmajor(smem_u32(smem + L::oQ)), kdO = desc_lo_kmajor(smem_u32(smem + L::odO));
             auto issue_S = [&](int k) {
-                const int s = k % NST;
-                mbar_wait(&bars[DB_KVFULL + s], (k / NST) & 1, ab);
+                const int s = k % NSTK;
+                mbar_wait(&bars[DB_KFULL + s], (k / NSTK) & 1, ab);
                 tcgen05_fence_after();
                 const uint32_t kK = desc_lo_kmajor(smem_u32(smem + L::oK + s * L::kTile));
 #pragma unroll
@@ -175,32 +180,41 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
                 }
                 mma_commit(&bars[DB_S + (k & 1)]);
             };
-            mbar_wait(&bars[DB_Q], 0, ab);
-            issue_S(0);
-            for (int k = 0; k < niter; ++k) {
-                const int s = k % NST, b = k & 1;
-                // dP = dO_i V_j^T once every thread has read the previous dP out of tensor memory
-                if (k > 0) {
-                    mbar_wait(&bars[DB_DPFREE], (k - 1) & 1, ab);
-                    tcgen05_fence_after();
-                }
-                const uint32_t kV = desc_lo_kmajor(smem_u32(smem + L::oV + s * L::kTile));
+            auto issue_dP = [&](int k) {
+                mbar_wait(&bars[DB_VFULL + k % NSTV], (k / NSTV) & 1, ab);
+                tcgen05_fence_after();
+                const uint32_t kV = desc_lo_kmajor(smem_u32(smem + L::oV + (k % NSTV) * L::kTile));
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk) {
                     const uint32_t off = (kk / 4) * kSlab + (kk % 4) * 2;
                     mma_ss_lo(T_dP, kdO + off, kV + off, idesc_s, kk > 0);
                 }
                 mma_commit(&bars[DB_DP]);
-                if (k + 1 < niter) issue_S(k + 1);
+                mma_commit(&bars[DB_VEMPTY + k % NSTV]);
+            };
+            // Queue order: S(k+1) and dP(k+1) are issued while the warps still work on tile k, so that
+            // neither is waited for; only dQ(k) needs the warps' result.
+            mbar_wait(&bars[DB_Q], 0, ab);
+            issue_S(0);
+            issue_dP(0);
+            for (int k = 0; k < niter; ++k) {
+                const int s = k % NSTK, b = k & 1;
+                if (k + 1 < niter) {
+                    issue_S(k + 1);   // its buffer held dS(k-1), which the dQ product queued last iteration has consumed
+                    // dP(k+1) once every thread has read dP(k) out of tensor memory
+                    mbar_wait(&bars[DB_DPFREE], k & 1, ab);
+                    tcgen05_fence_after();
+                    issue_dP(k + 1);
+                }
                 // dQ_i += dS K_j
                 mbar_wait(&bars[DB_DS + b], (k >> 1) & 1, ab);
                 tcgen05_fence_after();
                 const uint32_t mK_ = desc_lo_mnmajor(smem_u32(smem + L::oK + s * L::kTile), SLAB);
 #pragma unroll
                 for (int kk = 0; kk < TKD / 16; ++kk)
-                    mma_ts_lo(T_dQ, tm + b * 128 + (kk < 4 ? kk * 8 : 64 + (kk - 4) * 8), mK_ + kk * 128, idesc_dq,
+                    mma_ts_lo(T_dQ, tm + b * 128 + (kk / 2) * 32 + (kk % 2) * 8, mK_ + kk * 128, idesc_dq,
                               (k > 0) || (kk > 0));
-                mma_commit(&bars[DB_KVEMPTY + s]);
+                mma_commit(&bars[DB_KEMPTY + s]);
                 if (k == niter - 1) mma_commit(&bars[DB_DQ]);
             }
         }
@@ -217,52 +231,43 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
         for (int idx = 0; idx < iter.raw; ++idx) {
             const int jt = iter.tile(idx);
             if (jt < 0) continue;
-            const int b = k & 1, j0 = jt * TKD + wg * 64;
+            const int b = k & 1, j0 = jt * TKD + wg * 32;
             const uint32_t T_S = tm + b * 128;
             const bool masked = (a.mask_kind == ATTN_MASK_CAUSAL && jt * TKD + TKD - 1 > i0) || jt * TKD + TKD > n;
             mbar_wait(&bars[DB_S + b], (k >> 1) & 1, ab);
             tcgen05_fence_after();
-            float p[64];
+            float p[32];
             {
-                uint32_t sv0[32], sv1[32];
-                tmem_ld32(T_S + lane_addr + wg * 64, sv0);
-                tmem_ld32(T_S + lane_addr + wg * 64 + 32, sv1);
+                uint32_t sv0[32];
+                tmem_ld32(T_S + lane_addr + wg * 32, sv0);
                 tmem_wait_ld();
 #pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    p[e] = ex2_fast(fmaf(__uint_as_float(sv0[e]), sl2, nl));
-                    p[32 + e] = ex2_fast(fmaf(__uint_as_float(sv1[e]), sl2, nl));
-                }
+                for (int e = 0; e < 32; ++e) p[e] = ex2_fast(fmaf(__uint_as_float(sv0[e]), sl2, nl));
             }
             if (masked) {
                 const bool causal = a.mask_kind == ATTN_MASK_CAUSAL;
 #pragma unroll
-                for (int e = 0; e < 64; ++e) {
+                for (int e = 0; e < 32; ++e) {
                     const int jg = j0 + e;
                     if (jg >= n || (causal && jg > ig)) p[e] = 0.f;
                 }
             }
             mbar_wait(&bars[DB_DP], k & 1, ab);
             tcgen05_fence_after();
-            uint32_t dpack[32];
+            uint32_t dpack[16];
             {
-                uint32_t dv0[32], dv1[32];
-                tmem_ld32(T_dP + lane_addr + wg * 64, dv0);
-                tmem_ld32(T_dP + lane_addr + wg * 64 + 32, dv1);
+                uint32_t dv0[32];
+                tmem_ld32(T_dP + lane_addr + wg * 32, dv0);
                 tmem_wait_ld();
                 tcgen05_fence_before();
                 mbar_arrive(&bars[DB_DPFREE]);
 #pragma unroll
-                for (int e = 0; e < 32; e += 2) {
+                for (int e = 0; e < 32; e += 2)
                     dpack[e / 2] = pack_bf16(p[e] * fmaf(__uint_as_float(dv0[e]), a.scale, -dsi),
                                              p[e + 1] * fmaf(__uint_as_float(dv0[e + 1]), a.scale, -dsi));
-                    dpack[16 + e / 2] = pack_bf16(p[32 + e] * fmaf(__uint_as_float(dv1[e]), a.scale, -dsi),
-                                                  p[33 + e] * fmaf(__uint_as_float(dv1[e + 1]), a.scale, -dsi));
-                }
             }
-            // dS (bf16 pairs) over S columns this thread has read itself: keys 0..63 -> columns 0..31,
-            // keys 64..127 -> columns 64..95 of the S buffer
-            tmem_st32(T_S + lane_addr + wg * 64, dpack);
+            // dS (bf16 pairs) over the first 16 of the 32 S columns this thread has read itself
+            tmem_st16(T_S + lane_addr + wg * 32, dpack);
             tmem_wait_st();
             tcgen05_fence_before();
             mbar_arrive(&bars[DB_DS + b]);
@@ -273,14 +278,15 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
             mbar_wait(&bars[DB_DQ], 0, ab);
             tcgen05_fence_after();
         }
-        constexpr int HALF = HD / 2;
+        constexpr int OW = HD / 4;   // dQ columns per warpgroup: 32 or 16
         const int ic = ig < n ? ig : 0;
-        __nv_bfloat16 *pq = a.dQ + ((size_t)bh * n + ic) * HD + wg * HALF;
-#pragma unroll
-        for (int c = 0; c < HALF; c += 32) {
+        __nv_bfloat16 *pq = a.dQ + ((size_t)bh * n + ic) * HD + wg * OW;
+        {
+            constexpr int c = 0;
             uint32_t v[32];
             if (k > 0) {
-                tmem_ld32(T_dQ + lane_addr + wg * HALF + c, v);
+                if (OW == 32) tmem_ld32(T_dQ + lane_addr + wg * OW, v);
+                else tmem_ld16(T_dQ + lane_addr + wg * OW, *reinterpret_cast<uint32_t(*)[16]>(v));
                 tmem_wait_ld();
             } else {
 #pragma unroll
@@ -288,7 +294,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
             }
             if (ig < n) {
 #pragma unroll
-                for (int e = 0; e < 32; e += 8)
+                for (int e = 0; e < OW; e += 8)
                     *reinterpret_cast<uint4 *>(pq + c + e) =
                         make_uint4(pack_bf16(__uint_as_float(v[e]), __uint_as_float(v[e + 1])),
                                    pack_bf16(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3])),
