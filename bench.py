@@ -414,6 +414,30 @@ def main():
                     "frac_of_burst_peak": ach / peaks["bf16_tflops"], "peak_source": peaks["source"] + " sustained",
                     "avg_launch_ms": avg_ms, "launches_timed": len(kernel_ms[top]), "flops_per_launch": alg,
                     "flops_note": note, "traffic": TRAFFIC.get((top, w.name)), "kernel_time_share": share}
+    # the memory-bound step of the path (D pre-pass) against the measured copy bandwidth
+    roofline_hbm = None
+    for name in ("tc_bwd_preprocess", "mat_preprocess", "bwd_preprocess_D"):
+        if name in kernel_ms:
+            elem = 2 if w.bf16 else 4
+            rows = w.batch * w.heads * w.n
+            by = rows * (2 * w.d * elem + (12 if name != "bwd_preprocess_D" else 4))
+            avg = sum(kernel_ms[name]) / len(kernel_ms[name])
+            gbs = by / (avg * 1e-3) / 1e9
+            roofline_hbm = {"bound": "hbm", "kernel": name, "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                            "frac": gbs / peaks["hbm_gbs"], "avg_launch_ms": avg, "bytes_per_launch": by,
+                            "peak_source": peaks["source"]}
+            break
+    # the paper's I/O bound (Theorem 1.1 / 1.2, constant 1, elements -> bytes) at this configuration's on-chip size
+    elem = 2 if w.bf16 else 4
+    M = attn.attn_cfg_onchip_elems(w.d, dt_code, cfg, True)
+    if w.mask == inputs.MASK_BLOCK_SPARSE:
+        bound_el = attn.attn_io_bound_sparse_elems(w.n * w.d, kept_entries(w, bmask), M) if M else None
+    else:
+        bound_el = attn.attn_io_bound_elems(w.n, w.d, M, True) * (0.5 if w.mask == inputs.MASK_CAUSAL else 1.0) if M else None
+    comp = (8 * w.n * w.d * elem + 2 * 4 * w.n) * w.batch * w.heads
+    io = {"backward_compulsory_bytes": comp, "onchip_elems_M": M,
+          "paper_bound_bytes_at_M": bound_el * elem * w.batch * w.heads if bound_el else None,
+          "dram_bytes_measured_dominant_kernel": TRAFFIC.get((max(tot, key=tot.get), w.name)) if tot else None}
     line = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": step_ms / args.steps, "higher_is_better": True, "scaling": "weak",
@@ -427,7 +451,7 @@ def main():
         "fwd_ms": fwd_ms / args.steps, "bwd_ms": bwd_ms / args.steps, "wall_ms_per_step": wall_ms / args.steps,
         "frac_of_sustained_peak": value / world / peaks["bf16_tflops_sustained"],
         "clocks": clocks, "gpu_launches": int(launches_all),
-        "roofline": roofline,
+        "roofline": roofline, "roofline_hbm": roofline_hbm, "io": io,
     }
     if not args.no_e2e:
         elem = 2 if w.bf16 else 4

@@ -420,6 +420,34 @@ __global__ void __launch_bounds__(256) preprocess_kernel(const T *__restrict__ O
     const size_t warp = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) / 32;
     const size_t nwarps = (size_t)gridDim.x * blockDim.x / 32;
     const int sub = lane / lanes_per_row, lr = lane % lanes_per_row;
+    if (vec_per_row == lanes_per_row) {
+        // one vector per lane and row: four row groups per step, all eight loads in flight before any is used
+        constexpr int U = 4;
+        const size_t step = (size_t)rows_per_warp * U;
+        for (size_t base = warp * step; base < rows; base += nwarps * step) {
+            uint4 xo[U], xg[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const size_t row = base + (size_t)u * rows_per_warp + sub;
+                xo[u] = xg[u] = make_uint4(0u, 0u, 0u, 0u);
+                if (row < rows) {
+                    xo[u] = __ldcs(reinterpret_cast<const uint4 *>(O + row * d) + lr);
+                    xg[u] = __ldcs(reinterpret_cast<const uint4 *>(dO + row * d) + lr);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const size_t row = base + (size_t)u * rows_per_warp + sub;
+                const T *eo = reinterpret_cast<const T *>(&xo[u]), *eg = reinterpret_cast<const T *>(&xg[u]);
+                float s = 0.f;
+#pragma unroll
+                for (int e = 0; e < VE; ++e) s = fmaf(to_f(eo[e]), to_f(eg[e]), s);
+                for (int o = lanes_per_row / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+                if (row < rows && lr == 0) D[row] = s;
+            }
+        }
+        return;
+    }
     for (size_t base = warp * rows_per_warp; base < rows; base += nwarps * rows_per_warp) {
         const size_t row = base + sub;
         float s = 0.f;
@@ -542,7 +570,7 @@ attn_status preprocess_D(const void *O, const void *dO, float *D, size_t rows, i
     const size_t rows_per_warp = 32 / lanes;
     const size_t warps = (rows + rows_per_warp - 1) / rows_per_warp;
     size_t blocks = (warps + 7) / 8;
-    const size_t cap = 148 * 8 * 4;  // a few resident CTAs per SM, grid-stride beyond that
+    const size_t cap = 148 * 8;      // eight resident CTAs of 256 threads per SM, grid-stride beyond that
     if (blocks > cap) blocks = cap;
     launch_begin("bwd_preprocess_D", s);
     if (dt == ATTN_F32)

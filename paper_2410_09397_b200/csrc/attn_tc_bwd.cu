@@ -138,30 +138,40 @@ __global__ void __launch_bounds__(256) tc_preprocess_kernel(const __nv_bfloat16 
 {
     constexpr int LPR = HD / 8;   // lanes per row
     constexpr int RPW = 32 / LPR; // rows per warp
+    constexpr int U = 4;          // row groups per step: eight 16-byte loads in flight per lane
     const int lane = threadIdx.x % 32, sub = lane / LPR, lr = lane % LPR;
     const size_t warp = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) / 32;
     const size_t nwarps = (size_t)gridDim.x * blockDim.x / 32;
-    for (size_t base = warp * RPW; base < rows; base += nwarps * RPW) {
-        const size_t row = base + sub;
-        float acc = 0.f;
-        if (row < rows) {
-            const uint4 xo = __ldg(reinterpret_cast<const uint4 *>(O + row * HD) + lr);
-            const uint4 xg = __ldg(reinterpret_cast<const uint4 *>(dO + row * HD) + lr);
-            const __nv_bfloat162 *eo = reinterpret_cast<const __nv_bfloat162 *>(&xo);
-            const __nv_bfloat162 *eg = reinterpret_cast<const __nv_bfloat162 *>(&xg);
+    for (size_t base = warp * RPW * U; base < rows; base += nwarps * RPW * U) {
+        uint4 xo[U], xg[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t row = base + (size_t)u * RPW + sub;
+            xo[u] = xg[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (row < rows) {
+                xo[u] = __ldcs(reinterpret_cast<const uint4 *>(O + row * HD) + lr);
+                xg[u] = __ldcs(reinterpret_cast<const uint4 *>(dO + row * HD) + lr);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t row = base + (size_t)u * RPW + sub;
+            const __nv_bfloat162 *eo = reinterpret_cast<const __nv_bfloat162 *>(&xo[u]);
+            const __nv_bfloat162 *eg = reinterpret_cast<const __nv_bfloat162 *>(&xg[u]);
+            float acc = 0.f;
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const float2 fo = __bfloat1622float2(eo[e]), fg = __bfloat1622float2(eg[e]);
                 acc = fmaf(fo.x, fg.x, acc);
                 acc = fmaf(fo.y, fg.y, acc);
             }
-        }
 #pragma unroll
-        for (int o = LPR / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-        if (row < rows && lr == 0) {
-            Ds[row] = acc * scale;
-            const float l = LSE[row];
-            nlse2[row] = l == -INFINITY ? -INFINITY : -l * 1.4426950408889634f;
+            for (int o = LPR / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+            if (row < rows && lr == 0) {
+                Ds[row] = acc * scale;
+                const float l = LSE[row];
+                nlse2[row] = l == -INFINITY ? -INFINITY : -l * 1.4426950408889634f;
+            }
         }
     }
 }
