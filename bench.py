@@ -400,14 +400,16 @@ def main():
         top = max(tot, key=tot.get)
         avg_ms = tot[top] / len(kernel_ms[top])
         share = {k: round(v / sum(tot.values()), 4) for k, v in tot.items()}
-        if "bwd" in top and "preprocess" not in top:
-            # fraction of the backward's algorithmic FLOPs this kernel carries
-            names_bwd = [k for k in tot if "bwd" in k and "preprocess" not in k and "convert" not in k]
-            alg = fb if len(names_bwd) == 1 else fb * (0.8 if "dkdv" in top else 0.6)
-            note = ("algorithmic FLOPs of the five backward products" if len(names_bwd) == 1 else
-                    "this kernel's own products (the split backward recomputes S and dP in both kernels)")
-        else:
-            alg, note = ff, "algorithmic FLOPs of the two forward products"
+        # FLOPs one launch of each kernel executes, as a share of the forward (F) / backward (B) algorithmic
+        # count: the backward's five products are 0.2 B each; the split kernels recompute S and dP
+        own = {"tc_fwd": ("F", 1.0), "simt_fwd": ("F", 1.0), "tc_bwd_fused": ("B", 1.0),
+               "tc_bwd_dkdv": ("B", 0.8), "tc_bwd_dq": ("B", 0.6), "simt_bwd_dkdv": ("B", 0.8), "simt_bwd_dq": ("B", 0.6),
+               "mat_phase1_P": ("B", 0.2), "mat_phase2_dP": ("B", 0.2), "mat_phase4_dV": ("B", 0.2),
+               "mat_phase4_dK": ("B", 0.2), "mat_phase4_dQ": ("B", 0.2)}
+        which, share_ = own.get(top, ("B", 1.0))
+        alg = (ff if which == "F" else fb) * share_
+        note = ("algorithmic FLOPs of the five backward products" if top == "tc_bwd_fused" else
+                f"this kernel's own products: {share_:g} x the {'forward' if which == 'F' else 'backward'} count")
         ach = alg / (avg_ms * 1e-3) / 1e12
         roofline = {"bound": "tensor", "kernel": top, "achieved": ach, "peak": peaks["bf16_tflops_sustained"],
                     "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"],
@@ -473,6 +475,8 @@ TRAFFIC: dict = {
     # profiles/tc_bwd_fused_C3.md: 294.0 MB on the 16-head case; the full workload has 32 heads and the
     # traffic grows with the number of heads (heads are independent)
     ("tc_bwd_fused", "C3"): 588.0e6,
+    # profiles/mat_bwd_C4_tile_sweep.md: 94.6 MB on the 4-head case, 8 heads in the full workload
+    ("mat_phase1_P", "C4"): 189.2e6,
 }
 
 
