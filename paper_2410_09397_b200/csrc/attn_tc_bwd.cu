@@ -40,6 +40,7 @@ constexpr uint32_t SLAB = 128 * 128;   // bytes of one [128 rows][64 bf16] slab
 // dQ tile orientation at d = 128: transposed (lane = head-dimension index, coalesced scalar
 // reductions) or plain (lane = query, 16-byte vector reductions)
 constexpr bool kDqTransposed128 = true;
+constexpr bool kReducerWarps = true;   // d = 128 fused path: dedicated warps for the dQ reductions (tc_bwd_kernel_v4)
 
 struct BwdArgs {
     const float *nLSE2, *Ds;   // -LSE log2(e) and scale * D per row (workspace)
@@ -842,6 +843,359 @@ tc_bwd_kernel_v2(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
     if (warp == 0) tmem_dealloc(tm, 512);
 }
 
+// ---------------------------------------------------------------------------------------
+// d = 128, pipelined variant with reducer warps.  As tc_bwd_kernel_v2<true>, plus eight warps
+// (16-23) that do nothing but move finished dQ^T tiles from tensor memory into the fp32
+// accumulator: the red.global.add queue stalls them, not the warps on the tile loop.  To fit
+// 25 warps in the register file the exp/dS warps keep P only as the bf16 pairs they hand to
+// the dV product, and form dS from those.
+constexpr int kThreadsV4 = 256 + 256 + 64;   // 8 exp/dS warps, 8 reducer warps, issuer warp, TMA producer warp
+__global__ void __launch_bounds__(kThreadsV4, 1)
+tc_bwd_kernel_v4(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mK_,
+                 const __grid_constant__ CUtensorMap mV, const __grid_constant__ CUtensorMap mdO, const BwdArgs a)
+{
+    constexpr int HD = 128;
+    constexpr bool WITH_DQ = true;
+    constexpr int kHalfThreads = 128;     // exp / dS threads per half
+    constexpr int kReduceThreads = 128;   // reducer threads per half
+    using L = BwdSmem<HD>;
+    static_assert(L::oMisc - L::oBar >= 17 * 8, "barrier area");
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::oBar);
+    uint32_t *tmem_base_s = reinterpret_cast<uint32_t *>(smem + L::oMisc);
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(smem + L::oMisc + 4);
+    const Abort ab{abort_flag, a.status};
+
+    const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
+    // launch order: heads in groups of `a.group`, inside a group key tile major -- with a causal
+    // mask the CTAs of a group then start longest first, which evens out the tail of the grid
+    const int jt = blockIdx.x / a.group;
+    const long bh = (long)blockIdx.y * a.group + blockIdx.x % a.group;
+    const int j0 = jt * TK, n = a.n;
+
+    if ((smem_u32(smem) & 1023u) != 0) {
+        if (tid == 0) atomicExch(a.status, 9u);
+        return;
+    }
+    if (tid == 0) {
+        *abort_flag = 0;
+        mbar_init(&bars[V2_KV], 1);
+        for (int h = 0; h < 2; ++h) {
+            mbar_init(&bars[V2_QFULL + h], 1);
+            mbar_init(&bars[V2_QEMPTY + h], 1);
+            mbar_init(&bars[V2_S + h], 1);
+            mbar_init(&bars[V2_DP + h], 1);
+            mbar_init(&bars[V2_P + h], kHalfThreads);
+            mbar_init(&bars[V2_DS + h], kHalfThreads);
+            mbar_init(&bars[V2_DQ + h], 1);
+            mbar_init(&bars[V2_DQDONE + h], kReduceThreads);
+        }
+        fence_barrier_init();
+        prefetch_tensormap(&mQ); prefetch_tensormap(&mK_); prefetch_tensormap(&mV); prefetch_tensormap(&mdO);
+    }
+    if (warp == 0) tmem_alloc(tmem_base_s, 512);
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tm = *tmem_base_s;
+    const uint32_t T_S = tm, T_dP = tm + 128, T_dV = tm + 256, T_dK = tm + 256 + HD;
+    constexpr uint32_t HALF_ROWS = 64 * 128;   // byte offset of rows 64.. inside a [128][64] slab
+
+    const TileIter iter(a, jt, bh);
+
+    if (warp == 17) {
+        // ------------------------------------------------------------ TMA producer: every load, as soon as its stage is free
+        if (lane == 0) {
+            auto issue_load = [&](int it, int s) {
+                const int i0 = it * TQ;
+                const uint32_t rows = min(TQ, n - i0);
+                uint64_t *bar = &bars[V2_QFULL + s];
+                mbar_expect_tx(bar, 2 * L::kTile + 2 * rows * 4);
+#pragma unroll
+                for (uint32_t sl = 0; sl < L::kSlabs; ++sl) {
+                    tma_load_3d(smem + L::oQ + s * L::kTile + sl * SLAB, &mQ, bar, sl * 64, i0, (int)bh);
+                    tma_load_3d(smem + L::odO + s * L::kTile + sl * SLAB, &mdO, bar, sl * 64, i0, (int)bh);
+                }
+                bulk_load_1d(smem + L::oLSE + s * 512, a.nLSE2 + bh * n + i0, rows * 4, bar);
+                bulk_load_1d(smem + L::oD + s * 512, a.Ds + bh * n + i0, rows * 4, bar);
+            };
+            mbar_expect_tx(&bars[V2_KV], 2 * L::kTile);
+#pragma unroll
+            for (uint32_t sl = 0; sl < L::kSlabs; ++sl) {
+                tma_load_3d(smem + L::oK + sl * SLAB, &mK_, &bars[V2_KV], sl * 64, j0, (int)bh);
+                tma_load_3d(smem + L::oV + sl * SLAB, &mV, &bars[V2_KV], sl * 64, j0, (int)bh);
+            }
+            int k = 0;
+            for (int idx = 0; idx < iter.raw; ++idx) {
+                const int it = iter.tile(idx);
+                if (it < 0) continue;
+                const int s = k & 1;
+                if (k >= 2) mbar_wait(&bars[V2_QEMPTY + s], ((k - 2) >> 1) & 1, ab);   // last read by dK of tile k-2
+                issue_load(it, s);
+                ++k;
+            }
+        }
+    } else if (warp == 16) {
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = idesc_bf16(128, 128, 0, 0);       // S^T, dP^T (both halves at once)
+            constexpr uint32_t idesc_dv = idesc_bf16(128, HD, 0, 1);       // dV (A tmem), dK (A K-major smem)
+            constexpr uint32_t idesc_dq = idesc_bf16(128, 128, 1, 1);      // dQ^T
+            // low descriptor words (tc_common.cuh): per-step offsets are added as (bytes >> 4)
+            const uint32_t kK = desc_lo_kmajor(smem_u32(smem + L::oK)), kV = desc_lo_kmajor(smem_u32(smem + L::oV));
+            const uint32_t mK = desc_lo_mnmajor(smem_u32(smem + L::oK), SLAB);
+            const uint32_t kdS = desc_lo_kmajor(smem_u32(smem + L::odS)), mdS = desc_lo_mnmajor(smem_u32(smem + L::odS), SLAB);
+            constexpr uint32_t kHalf = HALF_ROWS >> 4, kSlab = SLAB >> 4;
+            // S^T = K_j Q_i^T for the whole tile in stage s; one commit per half's barrier
+            auto issue_S = [&](int s) {
+                const uint32_t kQ = desc_lo_kmajor(smem_u32(smem + L::oQ + s * L::kTile));
+#pragma unroll
+                for (int kk = 0; kk < HD / 16; ++kk) {
+                    const uint32_t off = (kk / 4) * kSlab + (kk % 4) * 2;
+                    mma_ss_lo(T_S, kK + off, kQ + off, idesc_s, kk > 0);
+                }
+                mma_commit(&bars[V2_S]);
+                mma_commit(&bars[V2_S + 1]);
+            };
+            int idx = 0, it = -1;
+            while (idx < iter.raw && (it = iter.tile(idx)) < 0) ++idx;
+            if (it >= 0) {
+                mbar_wait(&bars[V2_QFULL], 0, ab);
+                mbar_wait(&bars[V2_KV], 0, ab);
+                tcgen05_fence_after();
+                issue_S(0);
+            }
+            int k = 0;
+            while (idx < iter.raw) {
+                const int s = k & 1;
+                int nidx = idx + 1, nit = -1;
+                while (nidx < iter.raw && (nit = iter.tile(nidx)) < 0) ++nidx;
+                const uint32_t sQa = smem_u32(smem + L::oQ + s * L::kTile), sdOa = smem_u32(smem + L::odO + s * L::kTile);
+                const uint32_t kdO = desc_lo_kmajor(sdOa), mdO_ = desc_lo_mnmajor(sdOa, SLAB), mQ_ = desc_lo_mnmajor(sQa, SLAB);
+                // dP^T = V_j dO_i^T once both halves of the previous dQ^T have left T_dP
+                if (WITH_DQ && k > 0) {
+                    mbar_wait(&bars[V2_DQDONE], (k - 1) & 1, ab);
+                    mbar_wait(&bars[V2_DQDONE + 1], (k - 1) & 1, ab);
+                    tcgen05_fence_after();
+                }
+#pragma unroll
+                for (int kk = 0; kk < HD / 16; ++kk) {
+                    const uint32_t off = (kk / 4) * kSlab + (kk % 4) * 2;
+                    mma_ss_lo(T_dP, kV + off, kdO + off, idesc_s, kk > 0);
+                }
+                mma_commit(&bars[V2_DP]);
+                mma_commit(&bars[V2_DP + 1]);
+                // dV += P_h^T dO_h
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    mbar_wait(&bars[V2_P + h], k & 1, ab);
+                    tcgen05_fence_after();
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        mma_ts_lo(T_dV, T_S + 64 * h + kk * 8, mdO_ + h * kHalf + kk * 128,
+                                  idesc_dv, (k > 0) || (h > 0) || (kk > 0));
+                }
+                // T_S is free again: S^T of the next tile runs while this tile's dS is being formed
+                if (nit >= 0) {
+                    mbar_wait(&bars[V2_QFULL + (s ^ 1)], ((k + 1) >> 1) & 1, ab);
+                    tcgen05_fence_after();
+                    issue_S(s ^ 1);
+                }
+                // dQ^T = K_j^T dS^T first (into T_dP, whose dP^T both halves have consumed): the reducer warps
+                // read it out while dK += dS^T Q_i runs, so dP^T of the next tile is not held up by dK
+                mbar_wait(&bars[V2_DS], k & 1, ab);
+                mbar_wait(&bars[V2_DS + 1], k & 1, ab);
+                tcgen05_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < TK / 16; ++kk)
+                    mma_ss_lo(T_dP, mK + kk * 128, mdS + kk * 128, idesc_dq, kk > 0);
+                mma_commit(&bars[V2_DQ]);
+                mma_commit(&bars[V2_DQ + 1]);
+#pragma unroll
+                for (int kk = 0; kk < TQ / 16; ++kk)
+                    mma_ss_lo(T_dK, kdS + (kk / 4) * kSlab + (kk % 4) * 2, mQ_ + kk * 128, idesc_dv, (k > 0) || (kk > 0));
+                mma_commit(&bars[V2_QEMPTY + s]);
+                ++k;
+                idx = nidx;
+            }
+        }
+    } else if (warp >= 8) {
+        // ------------------------------------------------------------ reducers: dQ_h^T tile -> fp32 accumulator
+        // lanes = head-dimension index c, columns = queries: one warp instruction adds 128 contiguous bytes
+        const int h = (warp - 8) / 4;
+        const int row = (warp % 4) * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)((warp % 4) * 32) << 16;
+        int k = 0;
+        for (int idx = 0; idx < iter.raw; ++idx) {
+            const int it = iter.tile(idx);
+            if (it < 0) continue;
+            const int ig0 = it * TQ + h * 64;
+            mbar_wait(&bars[V2_DQ + h], k & 1, ab);
+            tcgen05_fence_after();
+            uint32_t v0[32], v1[32];
+            tmem_ld32(T_dP + lane_addr + h * 64, v0);
+            tmem_ld32(T_dP + lane_addr + h * 64 + 32, v1);
+            tmem_wait_ld();
+            tcgen05_fence_before();
+            mbar_arrive(&bars[V2_DQDONE + h]);   // T_dP half h is free again; the reductions proceed from registers
+            float *base = a.dQ_acc + ((size_t)bh * n + ig0) * HD + row;
+            if (ig0 + 64 <= n) {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) red_add_f32(base + (size_t)e * HD, __uint_as_float(v0[e]));
+#pragma unroll
+                for (int e = 0; e < 32; ++e) red_add_f32(base + (size_t)(32 + e) * HD, __uint_as_float(v1[e]));
+            } else {
+#pragma unroll
+                for (int e = 0; e < 32; ++e)
+                    if (ig0 + e < n) red_add_f32(base + (size_t)e * HD, __uint_as_float(v0[e]));
+#pragma unroll
+                for (int e = 0; e < 32; ++e)
+                    if (ig0 + 32 + e < n) red_add_f32(base + (size_t)(32 + e) * HD, __uint_as_float(v1[e]));
+            }
+            ++k;
+        }
+    } else {
+        // ------------------------------------------------------------ warpgroup h owns queries 64 h .. 64 h + 63 of every tile
+        const int h = warp / 4;
+        const int row = (warp % 4) * 32 + lane;        // tensor-memory lane = key row inside the tile
+        const uint32_t lane_addr = (uint32_t)((warp % 4) * 32) << 16;
+        const int jg = j0 + row;
+        const float sl2 = a.scale * 1.4426950408889634f;
+        int k = 0;
+        for (int idx = 0; idx < iter.raw; ++idx) {
+            const int it = iter.tile(idx);
+            if (it < 0) continue;
+            const int s = k & 1, i0 = it * TQ;
+            const float4 *sNL = reinterpret_cast<const float4 *>(smem + L::oLSE + s * 512 + h * 256);
+            const float4 *sDs = reinterpret_cast<const float4 *>(smem + L::oD + s * 512 + h * 256);
+            const bool diag = a.mask_kind == ATTN_MASK_CAUSAL && it == jt;
+            const bool masked = diag || i0 + TQ > n || j0 + TK > n;
+            const int ig0 = i0 + h * 64;
+            const uint32_t c0 = h * 64;                // this thread's first column in T_S / T_dP
+            mbar_wait(&bars[V2_QFULL + s], (k >> 1) & 1, ab);
+            mbar_wait(&bars[V2_S + h], k & 1, ab);
+            tcgen05_fence_after();
+            uint32_t ppack[32];   // P as bf16 pairs: what dV uses, and what dS is formed from
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch) {   // 16 columns at a time keeps the register count down
+                float p[16];
+                uint32_t sv0[16];
+                tmem_ld16(T_S + lane_addr + c0 + ch * 16, sv0);
+                tmem_wait_ld();
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const float4 nl = sNL[ch * 4 + q];
+                    const uint32_t *sv = &sv0[q * 4];
+                    p[q * 4 + 0] = ex2_approx(fmaf(__uint_as_float(sv[0]), sl2, nl.x));
+                    p[q * 4 + 1] = ex2_approx(fmaf(__uint_as_float(sv[1]), sl2, nl.y));
+                    p[q * 4 + 2] = ex2_approx(fmaf(__uint_as_float(sv[2]), sl2, nl.z));
+                    p[q * 4 + 3] = ex2_approx(fmaf(__uint_as_float(sv[3]), sl2, nl.w));
+                }
+                if (masked) {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        const int ig = ig0 + ch * 16 + e;
+                        const bool ok = ig < n && jg < n && (!diag || jg <= ig);
+                        p[e] = ok ? p[e] : 0.f;
+                    }
+                }
+#pragma unroll
+                for (int e = 0; e < 8; ++e) ppack[ch * 8 + e] = pack_bf16(p[2 * e], p[2 * e + 1]);
+            }
+            // P^T (bf16 pairs) over the first 32 of this half's 64 S^T columns: only this thread's own
+            // lane is read and written, so no cross-thread ordering is needed
+            tmem_st32(T_S + lane_addr + c0, ppack);
+            tmem_wait_st();
+            tcgen05_fence_before();
+            mbar_arrive(&bars[V2_P + h]);
+
+            mbar_wait(&bars[V2_DP + h], k & 1, ab);
+            tcgen05_fence_after();
+            {
+                uint8_t *slab = smem + L::odS + h * SLAB;
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    uint32_t dv[16];
+                    tmem_ld16(T_dP + lane_addr + c0 + ch * 16, dv);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int g = 0; g < 2; ++g) {    // 8 query columns = one 16-byte chunk
+                        float ds[8], p[8];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const uint32_t pk = ppack[ch * 8 + g * 4 + e];   // bf16 -> fp32 is a 16-bit shift
+                            p[2 * e] = __uint_as_float(pk << 16);
+                            p[2 * e + 1] = __uint_as_float(pk & 0xffff0000u);
+                        }
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            const float4 dsc = sDs[ch * 4 + g * 2 + u];
+                            const uint32_t *d4 = &dv[g * 8 + u * 4];
+                            ds[u * 4 + 0] = p[u * 4 + 0] * fmaf(__uint_as_float(d4[0]), a.scale, -dsc.x);
+                            ds[u * 4 + 1] = p[u * 4 + 1] * fmaf(__uint_as_float(d4[1]), a.scale, -dsc.y);
+                            ds[u * 4 + 2] = p[u * 4 + 2] * fmaf(__uint_as_float(d4[2]), a.scale, -dsc.z);
+                            ds[u * 4 + 3] = p[u * 4 + 3] * fmaf(__uint_as_float(d4[3]), a.scale, -dsc.w);
+                        }
+                        if (masked) {   // stale tail entries of the row vectors may be anything: select, do not multiply
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) ds[e] = p[e] != 0.f ? ds[e] : 0.f;
+                        }
+                        *reinterpret_cast<uint4 *>(slab + sw128_offset(row, ch * 16 + g * 8)) =
+                            make_uint4(pack_bf16(ds[0], ds[1]), pack_bf16(ds[2], ds[3]), pack_bf16(ds[4], ds[5]),
+                                       pack_bf16(ds[6], ds[7]));
+                    }
+                }
+            }
+            fence_proxy_async_smem();
+            tcgen05_fence_before();
+            mbar_arrive(&bars[V2_DS + h]);
+            ++k;
+        }
+        // ------------------------------------------------------------ epilogue: dV_j, dK_j (32 columns per warpgroup)
+        if (k > 0) {
+            // the last tile's dK product is the last thing the issuer queued before this commit
+            mbar_wait(&bars[V2_QEMPTY + ((k - 1) & 1)], ((k - 1) >> 1) & 1, ab);
+            tcgen05_fence_after();
+        }
+        {
+            constexpr int HALF = 32;
+            const int cq0 = (warp / 4) * 64;
+            const int jc = jg < n ? jg : 0;
+#pragma unroll
+            for (int cq = cq0; cq < cq0 + 64; cq += 32) {
+                __nv_bfloat16 *pv = a.dV + ((size_t)bh * n + jc) * HD + cq;
+                __nv_bfloat16 *pk = a.dK + ((size_t)bh * n + jc) * HD + cq;
+                uint32_t v[32], w[32];
+                if (k > 0) {
+                    tmem_ld32(T_dV + lane_addr + cq, v);
+                    tmem_ld32(T_dK + lane_addr + cq, w);
+                    tmem_wait_ld();
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) v[e] = w[e] = 0u;
+                }
+                if (jg < n) {
+#pragma unroll
+                    for (int e = 0; e < 32; e += 8) {
+                        *reinterpret_cast<uint4 *>(pv + e) =
+                            make_uint4(pack_bf16(__uint_as_float(v[e]), __uint_as_float(v[e + 1])),
+                                       pack_bf16(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3])),
+                                       pack_bf16(__uint_as_float(v[e + 4]), __uint_as_float(v[e + 5])),
+                                       pack_bf16(__uint_as_float(v[e + 6]), __uint_as_float(v[e + 7])));
+                        *reinterpret_cast<uint4 *>(pk + e) =
+                            make_uint4(pack_bf16(__uint_as_float(w[e]), __uint_as_float(w[e + 1])),
+                                       pack_bf16(__uint_as_float(w[e + 2]), __uint_as_float(w[e + 3])),
+                                       pack_bf16(__uint_as_float(w[e + 4]), __uint_as_float(w[e + 5])),
+                                       pack_bf16(__uint_as_float(w[e + 6]), __uint_as_float(w[e + 7])));
+                    }
+                }
+            }
+        }
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tm, 512);
+}
+
 // fp32 accumulator -> bf16 dQ
 __global__ void __launch_bounds__(256) dq_convert_kernel(const float4 *__restrict__ acc, uint2 *__restrict__ out, size_t n4)
 {
@@ -887,7 +1241,11 @@ attn_status launch_bwd(const Problem &p)
     }
     const dim3 grid((unsigned)((p.n + TK - 1) / TK * a.group), (unsigned)(p.BH / a.group));
     launch_begin(WITH_DQ ? "tc_bwd_fused" : "tc_bwd_dkdv", p.stream);
-    if (HD == 128) {
+    if (HD == 128 && WITH_DQ && kReducerWarps) {
+        if (cudaFuncSetAttribute(tc_bwd_kernel_v4, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::kBytes) != cudaSuccess)
+            return ATTN_ERR_LAUNCH;
+        tc_bwd_kernel_v4<<<grid, kThreadsV4, L::kBytes, p.stream>>>(mQ, mK, mV, mdO, a);
+    } else if (HD == 128) {
         if (cudaFuncSetAttribute(tc_bwd_kernel_v2<WITH_DQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::kBytes) != cudaSuccess)
             return ATTN_ERR_LAUNCH;
         tc_bwd_kernel_v2<WITH_DQ><<<grid, kThreadsV2, L::kBytes, p.stream>>>(mQ, mK, mV, mdO, a);
