@@ -37,6 +37,16 @@
  * steps of the paper's no-cache algorithm (Appendix C.1) literally, without the
  * max shift, materialising the n x n matrices; it is a second implementation that
  * the tests compare the first one with on small inputs.
+ *
+ * The attention weights (the paper's own gradient target):
+ *   attn_oracle_project      S = A1 X and h = A3 Y, the two products of phase 1 of the
+ *                            large-cache algorithm (Appendix D): out = A W per unit
+ *   attn_oracle_weight_grad  dL/dX = A1^T p A2 (Definition 3.2) given G = p A2, i.e. the
+ *                            plain product g = A^T G; with G = f^T dO it is dL/dY
+ *                            (O = f A3 Y is linear in Y).  Units that share a weight
+ *                            matrix add their gradients.
+ * Unit u (= batch index * heads + head) uses weight matrix u mod weight_units, so
+ * weight_units is 1 (one matrix for all), heads (shared over the batch) or batch*heads.
  */
 #include <math.h>
 #include <stdint.h>
@@ -235,4 +245,37 @@ void attn_oracle_dense(const double *Q, const double *K, const double *V, const 
     if (q_out) memcpy(q_out, q, sizeof(double) * nn);
     if (v_fq_out) memcpy(v_fq_out, v, sizeof(double) * (size_t)n);
     free(A); free(l); free(f); free(q); free(v);
+}
+
+/* out_u = A_u W_{u mod weight_units}; A, out: [units][n][d]; W: [weight_units][d][d], row = input
+ * feature, column = output feature (S = A1 X and h = A3 Y of Appendix D, phase 1). */
+void attn_oracle_project(const double *A, const double *W, double *out, int n, int d, long units, long weight_units)
+{
+#pragma omp parallel for schedule(static)
+    for (long r = 0; r < units * n; ++r) {
+        const long u = r / n;
+        const double *a = A + r * d;
+        const double *w = W + (u % weight_units) * (long)d * d;
+        double *o = out + r * d;
+        for (int c = 0; c < d; ++c) {
+            double acc = 0.0;
+            for (int k = 0; k < d; ++k) acc += a[k] * w[(long)k * d + c];
+            o[c] = acc;
+        }
+    }
+}
+
+/* g_w = sum over the units u with u mod weight_units = w of A_u^T G_u; A, G: [units][n][d];
+ * g: [weight_units][d][d] (Definition 3.2 with G = p A2: g = A1^T p A2). */
+void attn_oracle_weight_grad(const double *A, const double *G, double *g, int n, int d, long units, long weight_units)
+{
+    for (long w = 0; w < weight_units; ++w)
+        for (int a = 0; a < d; ++a)
+            for (int b = 0; b < d; ++b) {
+                double acc = 0.0;
+                for (long u = w; u < units; u += weight_units)
+                    for (int i = 0; i < n; ++i)
+                        acc += A[(u * n + i) * d + a] * G[(u * n + i) * d + b];
+                g[(w * d + a) * d + b] = acc;
+            }
 }

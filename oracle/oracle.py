@@ -8,6 +8,9 @@ All tensors are numpy float64 arrays shaped ``[batch, heads, n, d]`` (LSE
 (uint8 ``[mask_heads, nb, nb]``), 3 explicit element mask (uint8 ``[mask_heads, n, n]``,
 used only to cross-check the other kinds by brute force).
 
+``project`` / ``weight_grad`` / ``attn_weights_bwd`` cover the paper's own gradient target,
+the attention weights X and Y (Definition 3.2, Appendix D).
+
 Also here: ``io_bound_*`` -- the paper's closed-form I/O bounds (Theorem 1.1 and the
 sparse lower bound, Theorem 1.2 / 4.5) written out literally, used to check the
 library's bound calculators.
@@ -110,6 +113,40 @@ def attn_dense(Q, K, V, dO, *, mask_kind=MASK_NONE, block=128, mask_bits=None, s
                               ctypes.c_double(scale), _p(out["l"]), _p(out["f"]), _p(out["q"]), _p(out["p"]),
                               _p(out["v_fq"]))
     return out
+
+
+def project(A, W):
+    """``out[b, h] = A[b, h] @ W[(b*heads + h) % weight_units]`` -- S = A1 X or h = A3 Y
+    (Appendix D, phase 1).  ``A`` is ``[batch, heads, n, d]``, ``W`` is ``[weight_units, d, d]``."""
+    A, W = _f64(A), _f64(W)
+    b, h, n, d = A.shape
+    assert W.shape[1:] == (d, d) and W.shape[0] in (1, h, b * h)
+    out = np.empty_like(A)
+    _load().attn_oracle_project(_p(A), _p(W), _p(out), n, d, ctypes.c_long(b * h), ctypes.c_long(W.shape[0]))
+    return out
+
+
+def weight_grad(A, G, weight_units: int):
+    """``g[w] = sum over units u with u % weight_units == w of A[u]^T @ G[u]`` -- Definition 3.2
+    with ``G = p A2`` (the gradient with respect to S = A1 X)."""
+    A, G = _f64(A), _f64(G)
+    b, h, n, d = A.shape
+    assert weight_units in (1, h, b * h)
+    g = np.empty((weight_units, d, d), dtype=np.float64)
+    _load().attn_oracle_weight_grad(_p(A), _p(G), _p(g), n, d, ctypes.c_long(b * h), ctypes.c_long(weight_units))
+    return g
+
+
+def attn_weights_bwd(A1, A2, A3, X, Y, dO, *, mask_kind=MASK_NONE, block=128, mask_bits=None, scale=None):
+    """The paper's backward problem with its own inputs: S = A1 X, h = A3 Y (phase 1), the forward for
+    O and l, then dL/dX = A1^T p A2 and dL/dY = A3^T f^T dO.  Returns a dict with S, h, O, LSE, dS
+    (the gradient of S, = scale * p A2), dK, dh, gX, gY."""
+    S, h = project(A1, X), project(A3, Y)
+    kw = dict(mask_kind=mask_kind, block=block, mask_bits=mask_bits, scale=scale)
+    O, LSE = attn_fwd(S, A2, h, **kw)
+    dS, dK, dh = attn_bwd(S, A2, h, O, dO, LSE, **kw)
+    return {"S": S, "h": h, "O": O, "LSE": LSE, "dS": dS, "dK": dK, "dh": dh,
+            "gX": weight_grad(A1, dS, np.asarray(X).shape[0]), "gY": weight_grad(A3, dh, np.asarray(Y).shape[0])}
 
 
 # ---- closed-form I/O bounds, constants taken as 1 (Theorem 1.1; Theorem 1.2 / 4.5) ----
