@@ -118,6 +118,48 @@ attn_status attn_bwd(const void *Q, const void *K, const void *V, const void *O,
 attn_status attn_bwd_preprocess(const void *O, const void *dO, float *D, size_t rows, int d, int dt,
                                 void *cuda_stream);
 
+/* ---- The attention weights (the paper's own inputs and gradient target) ------------
+ *
+ * Definition 3.1 writes the scores as A1 X A2^T and the values as A3 Y with d x d weight
+ * matrices X (query and key weights folded into one) and Y; Definition 3.2 asks for
+ * dL/dX = A1^T p A2.  With S = A1 X the library's Q is S, its K is A2, its V is h = A3 Y,
+ * and dL/dS = attn_bwd's dQ, so dL/dX = A1^T dQ and dL/dY = A3^T dV.
+ *
+ * Tensors A, out, G: [batch, heads, n, d] like Q.  Weights W: [weight_units][d][d],
+ * element (k, c) multiplies input feature k into output feature c; unit u = batch index *
+ * heads + head uses matrix u mod weight_units, and weight_units is 1 (one matrix for
+ * all units), heads (shared over the batch) or batch * heads.  d is a multiple of 8, at
+ * most 256.  bf16 with d in {64, 128, 256} runs on the tensor cores, everything else on
+ * fp32 FMAs.  `workspace` (device, 256-byte aligned, at least 256 bytes for the first two
+ * calls) holds the status word that attn_workspace_status() reads.  All pointers are
+ * caller-owned device memory, 16-byte aligned; the calls are asynchronous on cuda_stream. */
+
+/* out = A W per unit: S = A1 X or h = A3 Y (Appendix D, phase 1 of the large-cache
+ * algorithm).  out has the dtype of A and is fully overwritten. */
+attn_status attn_project(const void *A, const void *W, void *out, int n, int d, int heads, int batch,
+                         int weight_units, int dt, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* g[w] = sum over the units u with u mod weight_units = w of A_u^T G_u, float
+ * [weight_units][d][d], fully overwritten (Definition 3.2 with G = p A2; the last two
+ * products of phase 2 of the large-cache algorithm, Appendix D).  The sum over units and
+ * row tiles uses fp32 atomic adds: results vary in the last bits from run to run. */
+attn_status attn_weight_grad(const void *A, const void *G, float *g, int n, int d, int heads, int batch,
+                             int weight_units, int dt, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Phase 2 of the large-cache algorithm as a whole (Appendix D): from A1, A2, A3, the
+ * projected S = A1 X and h = A3 Y, the forward's O and LSE (= ln l) and dO, computes
+ * gX = dL/dX = A1^T p A2 (times `scale` when the scores carry one) and, unless gY is NULL
+ * (the paper treats Y as fixed), gY = dL/dY = A3^T f^T dO.  Runs attn_bwd with Q = S,
+ * K = A2, V = h into workspace buffers, then attn_weight_grad twice.  mask, scale, cfg as
+ * in attn_bwd; workspace of attn_weights_bwd_workspace_bytes() bytes. */
+attn_status attn_weights_bwd(const void *A1, const void *A2, const void *A3, const void *S, const void *h,
+                             const void *O, const void *dO, const float *LSE, float *gX, float *gY,
+                             int n, int d, int heads, int batch, int weight_units, const attn_mask *mask,
+                             int dt, float scale, const attn_cfg *cfg,
+                             void *workspace, size_t workspace_bytes, void *cuda_stream);
+size_t attn_weights_bwd_workspace_bytes(int n, int d, int heads, int batch, const attn_mask *mask, int dt,
+                                        const attn_cfg *cfg);
+
 /* attn_bwd for callers that cannot allocate device memory (the paper has no
  * counterpart: this is a convenience of the library, not a step of the method).
  *

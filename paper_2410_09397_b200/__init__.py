@@ -13,4 +13,5 @@ from .binding import (  # noqa: F401
     attn_bwd_workspace_bytes, attn_cfg_onchip_elems, attn_fwd, attn_fwd_workspace_bytes, attn_io_bound_elems,
     attn_io_bound_sparse_elems, attn_kernel_launches, attn_noalloc_scratch_bytes, attn_supported_cfgs, attn_timing_collect, attn_timing_enable,
     attn_workspace_status, status_str,
+    attn_project, attn_weight_grad, attn_weights_bwd, attn_weights_bwd_workspace_bytes,
 )

@@ -28,6 +28,7 @@ EXPORTS = (
     "attn_workspace_status", "attn_supported_cfgs", "attn_cfg_onchip_elems", "attn_io_bound_elems",
     "attn_io_bound_sparse_elems", "attn_status_str", "attn_kernel_launches", "attn_timing_enable",
     "attn_timing_collect", "attn_bwd_noalloc", "attn_noalloc_scratch_bytes",
+    "attn_project", "attn_weight_grad", "attn_weights_bwd", "attn_weights_bwd_workspace_bytes",
 )
 
 
@@ -101,6 +102,15 @@ def lib() -> ctypes.CDLL:
     for f in (L.attn_fwd_workspace_bytes, L.attn_bwd_workspace_bytes):
         f.restype = sz
         f.argtypes = [ci, ci, ci, ci, ctypes.POINTER(CMask), ci, ctypes.POINTER(CCfg)]
+    L.attn_project.restype = ci
+    L.attn_project.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, ci, vp, sz, vp]
+    L.attn_weight_grad.restype = ci
+    L.attn_weight_grad.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, ci, vp, sz, vp]
+    L.attn_weights_bwd.restype = ci
+    L.attn_weights_bwd.argtypes = [vp] * 10 + [ci, ci, ci, ci, ci, ctypes.POINTER(CMask), ci, cf,
+                                               ctypes.POINTER(CCfg), vp, sz, vp]
+    L.attn_weights_bwd_workspace_bytes.restype = sz
+    L.attn_weights_bwd_workspace_bytes.argtypes = [ci, ci, ci, ci, ctypes.POINTER(CMask), ci, ctypes.POINTER(CCfg)]
     L.attn_workspace_status.restype = ci
     L.attn_workspace_status.argtypes = [vp, vp]
     L.attn_supported_cfgs.restype = ci
@@ -220,6 +230,64 @@ def attn_bwd_preprocess(O, dO, D=None):
     if st != ATTN_OK:
         raise AttnError(st, "attn_bwd_preprocess")
     return D
+
+
+def attn_project(A, W, out=None, *, workspace=None):
+    """out[b, h] = A[b, h] @ W[(b * heads + h) % weight_units]; ``W`` is ``[weight_units, d, d]``."""
+    import torch
+    _check_tensors(A, W)
+    b, h, n, d = A.shape
+    out = torch.empty_like(A) if out is None else out
+    workspace = _workspace(256, A) if workspace is None else workspace
+    st = lib().attn_project(A.data_ptr(), W.data_ptr(), out.data_ptr(), n, d, h, b, W.shape[0], _dtype_code(A),
+                            workspace.data_ptr(), workspace.numel(), _stream())
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_project")
+    return out
+
+
+def attn_weight_grad(A, G, weight_units: int, g=None, *, workspace=None):
+    """g[w] = sum of A[u]^T @ G[u] over the units u with u % weight_units == w; float32 ``[weight_units, d, d]``."""
+    import torch
+    _check_tensors(A, G)
+    b, h, n, d = A.shape
+    g = torch.empty((weight_units, d, d), dtype=torch.float32, device=A.device) if g is None else g
+    workspace = _workspace(256, A) if workspace is None else workspace
+    st = lib().attn_weight_grad(A.data_ptr(), G.data_ptr(), g.data_ptr(), n, d, h, b, weight_units, _dtype_code(A),
+                                workspace.data_ptr(), workspace.numel(), _stream())
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_weight_grad")
+    return g
+
+
+def attn_weights_bwd_workspace_bytes(n, d, heads, batch, mask: Mask | None, dt: int, cfg: Cfg | None) -> int:
+    return int(lib().attn_weights_bwd_workspace_bytes(n, d, heads, batch, _ref(mask.c() if mask else None), dt,
+                                                      _ref(cfg.c() if cfg else None)))
+
+
+def attn_weights_bwd(A1, A2, A3, S, h, O, dO, LSE, weight_units: int, gX=None, gY=None, *, want_gY: bool = True,
+                     mask: Mask | None = None, scale: float = 0.0, cfg: Cfg | None = None, workspace=None):
+    """gX = dL/dX, gY = dL/dY (None when ``want_gY`` is false) given S = A1 X, h = A3 Y and the forward's O, LSE."""
+    import torch
+    _check_tensors(A1, A2, S, h, O, dO, LSE)
+    b, nh, n, d = S.shape
+    dt = _dtype_code(S)
+    gX = torch.empty((weight_units, d, d), dtype=torch.float32, device=S.device) if gX is None else gX
+    if want_gY:
+        _check_tensors(A3)
+        gY = torch.empty((weight_units, d, d), dtype=torch.float32, device=S.device) if gY is None else gY
+    else:
+        gY = None
+    if workspace is None:
+        workspace = _workspace(attn_weights_bwd_workspace_bytes(n, d, nh, b, mask, dt, cfg), S)
+    cm, cc = (mask.c() if mask else None), (cfg.c() if cfg else None)
+    st = lib().attn_weights_bwd(A1.data_ptr(), A2.data_ptr(), A3.data_ptr() if A3 is not None else None, S.data_ptr(),
+                                h.data_ptr(), O.data_ptr(), dO.data_ptr(), LSE.data_ptr(), gX.data_ptr(),
+                                gY.data_ptr() if gY is not None else None, n, d, nh, b, weight_units, _ref(cm), dt,
+                                scale, _ref(cc), workspace.data_ptr(), workspace.numel(), _stream())
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_weights_bwd")
+    return gX, gY
 
 
 def attn_workspace_status(workspace) -> int:

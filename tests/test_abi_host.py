@@ -115,3 +115,43 @@ def test_workspace_sizes_and_cfgs(lib):
     for c in cfgs:
         assert B.attn_cfg_onchip_elems(64, B.ATTN_F32, c, True) > 0
     assert B.attn_cfg_onchip_elems(64, B.ATTN_F32, B.Cfg(tile_q=48, algo=B.ATTN_ALGO_SIMT), True) == 0
+
+
+def test_weight_entry_points_validate_before_any_launch(lib):
+    fake = 0x10000  # never dereferenced
+
+    def proj(A=fake, W=fake, out=fake, n=128, d=64, heads=2, batch=3, wu=2, dt=B.ATTN_BF16, w=fake, wb=256):
+        return lib.attn_project(A, W, out, n, d, heads, batch, wu, dt, w, wb, None)
+
+    def grad(A=fake, G=fake, g=fake, n=128, d=64, heads=2, batch=3, wu=6, dt=B.ATTN_BF16, w=fake, wb=256):
+        return lib.attn_weight_grad(A, G, g, n, d, heads, batch, wu, dt, w, wb, None)
+
+    for f in (proj, grad):
+        assert f(A=None) == B.ATTN_ERR_NULL
+        assert f(n=0) == B.ATTN_ERR_SHAPE
+        assert f(d=12) == B.ATTN_ERR_SHAPE
+        assert f(d=264) == B.ATTN_ERR_SHAPE
+        assert f(wu=3) == B.ATTN_ERR_SHAPE            # neither 1, heads nor batch * heads
+        assert f(wu=0) == B.ATTN_ERR_SHAPE
+        assert f(dt=5) == B.ATTN_ERR_DTYPE
+        assert f(w=None) == B.ATTN_ERR_WORKSPACE
+        assert f(wb=16) == B.ATTN_ERR_WORKSPACE
+        assert f(w=fake + 16) == B.ATTN_ERR_ALIGN
+        assert f(A=fake + 8) == B.ATTN_ERR_ALIGN
+    assert proj(out=None) == B.ATTN_ERR_NULL
+    assert grad(g=None) == B.ATTN_ERR_NULL
+
+    def wbwd(gX=fake, gY=fake, A3=fake, wb=1 << 30, wu=2, cfg=None, dt=B.ATTN_BF16):
+        return lib.attn_weights_bwd(fake, fake, A3, fake, fake, fake, fake, fake, gX, gY, 128, 64, 2, 3, wu, None, dt,
+                                    0.0, cfg, fake, wb, None)
+
+    assert wbwd(gX=None) == B.ATTN_ERR_NULL
+    assert wbwd(A3=None) == B.ATTN_ERR_NULL           # gY wanted but no A3
+    assert wbwd(wu=5) == B.ATTN_ERR_SHAPE
+    assert wbwd(wb=4096) == B.ATTN_ERR_WORKSPACE
+    bad_tile = B.CCfg(48, 0, 0, B.ATTN_ALGO_SIMT, 0)
+    assert wbwd(cfg=ctypes.byref(bad_tile)) == B.ATTN_ERR_TILE
+    need = B.attn_weights_bwd_workspace_bytes(128, 64, 2, 3, None, B.ATTN_BF16, None)
+    inner = B.attn_bwd_workspace_bytes(128, 64, 2, 3, None, B.ATTN_BF16, None)
+    assert need >= inner + 3 * 128 * 64 * 6 * 2
+    assert B.attn_weights_bwd_workspace_bytes(0, 64, 2, 3, None, B.ATTN_BF16, None) == 0

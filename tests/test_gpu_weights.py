@@ -1,0 +1,151 @@
+"""GPU parity of the attention-weight entry points (S = A1 X, h = A3 Y of Appendix D phase 1;
+dL/dX = A1^T p A2 of Definition 3.2 and dL/dY) against the float64 oracle, through the C ABI."""
+import numpy as np
+import pytest
+
+from oracle import oracle as orc
+from paper_2410_09397_b200 import inputs
+
+from tests.helpers import TOL, rel_err, to_dev, to_np
+
+pytestmark = pytest.mark.gpu
+
+
+def weights(seed, tid, units, d, dtype):
+    """d x d weights of standard deviation 1/sqrt(d): the projections of N(0, 1) rows are N(0, 1) again."""
+    w = inputs.normal_tensor(seed, tid, (units, d, d), bf16=False).astype(np.float64) / np.sqrt(d)
+    return inputs.round_to_bf16(w.astype(np.float32)) if dtype == "bf16" else w.astype(np.float32)
+
+
+def units_of(wu, b, h):
+    return {"one": 1, "heads": h, "all": b * h}[wu]
+
+
+PROJ_CASES = [
+    # b, h, n, d, dtype, weight sharing
+    (1, 1, 128, 64, "f32", "one"),          # the smallest workload's shape
+    (2, 3, 300, 64, "bf16", "heads"),       # several 128-row tiles and a ragged tail
+    (2, 3, 300, 128, "bf16", "all"),
+    (1, 2, 392, 256, "bf16", "one"),
+    (1, 1, 8, 128, "bf16", "one"),          # a single partial tile
+    (2, 2, 200, 40, "bf16", "heads"),       # head size without a tensor-core kernel
+    (1, 2, 100, 24, "f32", "all"),
+]
+
+
+@pytest.mark.parametrize("b,h,n,d,dtype,wu", PROJ_CASES)
+def test_project_matches_oracle(b, h, n, d, dtype, wu):
+    import torch
+    import paper_2410_09397_b200 as attn
+    A = inputs.normal_tensor(31, 0, (b, h, n, d), bf16=dtype == "bf16")
+    W = weights(31, 4, units_of(wu, b, h), d, dtype)
+    ref = orc.project(A, W)
+    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    out = attn.attn_project(to_dev(A, dtype), to_dev(W, dtype), workspace=ws)
+    torch.cuda.synchronize()
+    assert attn.attn_workspace_status(ws) == attn.ATTN_OK
+    assert rel_err(to_np(out), ref) <= TOL[dtype]
+
+
+GRAD_CASES = [
+    (1, 1, 128, 64, "f32", "one"),
+    (2, 3, 300, 64, "bf16", "heads"),
+    (2, 3, 300, 128, "bf16", "all"),
+    (1, 2, 392, 256, "bf16", "one"),
+    (1, 1, 8, 128, "bf16", "one"),
+    (2, 3, 4096, 64, "bf16", "heads"),      # more tiles than SMs: CTAs run through several tiles and weights
+    (2, 3, 4096, 128, "bf16", "all"),
+    (2, 3, 4096, 128, "bf16", "one"),
+    (2, 3, 2048, 256, "bf16", "heads"),
+    (2, 2, 200, 40, "bf16", "heads"),
+    (1, 2, 100, 24, "f32", "all"),
+]
+
+
+@pytest.mark.parametrize("b,h,n,d,dtype,wu", GRAD_CASES)
+def test_weight_grad_matches_oracle(b, h, n, d, dtype, wu):
+    import torch
+    import paper_2410_09397_b200 as attn
+    A = inputs.normal_tensor(32, 0, (b, h, n, d), bf16=dtype == "bf16")
+    G = inputs.normal_tensor(32, 3, (b, h, n, d), bf16=dtype == "bf16")
+    units = units_of(wu, b, h)
+    ref = orc.weight_grad(A, G, units)
+    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    dA, dG = to_dev(A, dtype), to_dev(G, dtype)
+    g = torch.full((units, d, d), 7.0, dtype=torch.float32, device="cuda")      # must be overwritten, not added to
+    for _ in range(2):                                                         # and a second call gives the same
+        attn.attn_weight_grad(dA, dG, units, g, workspace=ws)
+        torch.cuda.synchronize()
+        assert attn.attn_workspace_status(ws) == attn.ATTN_OK
+        assert rel_err(to_np(g), ref) <= TOL[dtype]
+
+
+E2E_CASES = [
+    # b, h, n, d, dtype, sharing, mask
+    (1, 1, 128, 64, "f32", "one", inputs.MASK_NONE),
+    (2, 2, 300, 64, "bf16", "heads", inputs.MASK_CAUSAL),
+    (2, 2, 392, 128, "bf16", "heads", inputs.MASK_NONE),
+    (1, 2, 392, 128, "bf16", "all", inputs.MASK_CAUSAL),
+    (1, 2, 264, 256, "bf16", "one", inputs.MASK_NONE),     # backward through the materialised algorithm
+]
+
+
+@pytest.mark.parametrize("b,h,n,d,dtype,wu,mask_kind", E2E_CASES)
+def test_weight_gradients_of_the_whole_path(b, h, n, d, dtype, wu, mask_kind):
+    """A1, A2, A3, X, Y, dO in; gX, gY out: projections, forward, phase 2 all on the GPU, against the oracle
+    run in float64 on the same (storage-rounded) inputs."""
+    import torch
+    import paper_2410_09397_b200 as attn
+    from paper_2410_09397_b200 import binding as B
+    bf = dtype == "bf16"
+    A1, A2, A3, dO = (inputs.normal_tensor(33, t, (b, h, n, d), bf16=bf) for t in range(4))
+    units = units_of(wu, b, h)
+    X, Y = weights(33, 4, units, d, dtype), weights(33, 5, units, d, dtype)
+    ref = orc.attn_weights_bwd(A1, A2, A3, X, Y, dO, mask_kind=mask_kind)
+
+    dev = {k: to_dev(v, dtype) for k, v in dict(A1=A1, A2=A2, A3=A3, dO=dO, X=X, Y=Y).items()}
+    mask = None if mask_kind == inputs.MASK_NONE else B.Mask(kind=mask_kind)
+    S, hh = attn.attn_project(dev["A1"], dev["X"]), attn.attn_project(dev["A3"], dev["Y"])
+    O, LSE = attn.attn_fwd(S, dev["A2"], hh, mask=mask)
+    dt = B.ATTN_BF16 if bf else B.ATTN_F32
+    ws = torch.zeros(B.attn_weights_bwd_workspace_bytes(n, d, h, b, mask, dt, None), dtype=torch.uint8, device="cuda")
+    gX, gY = attn.attn_weights_bwd(dev["A1"], dev["A2"], dev["A3"], S, hh, O, dev["dO"], LSE, units, mask=mask,
+                                   workspace=ws)
+    torch.cuda.synchronize()
+    assert attn.attn_workspace_status(ws) == attn.ATTN_OK
+    errs = {"S": rel_err(to_np(S), ref["S"]), "h": rel_err(to_np(hh), ref["h"]), "O": rel_err(to_np(O), ref["O"]),
+            "gX": rel_err(to_np(gX), ref["gX"]), "gY": rel_err(to_np(gY), ref["gY"])}
+    assert all(v <= TOL[dtype] for v in errs.values()), errs
+    # Y fixed, as in the paper's statement: only gX is produced
+    gX2, none = attn.attn_weights_bwd(dev["A1"], dev["A2"], None, S, hh, O, dev["dO"], LSE, units, want_gY=False,
+                                      mask=mask, workspace=ws)
+    torch.cuda.synchronize()
+    assert none is None and rel_err(to_np(gX2), ref["gX"]) <= TOL[dtype]
+
+
+def test_weight_kernels_at_headline_size_on_sampled_units():
+    """batch 2 x 16 heads, n = 8192, d = 128, bf16: the launch shape the benchmark times; the oracle checks
+    two sampled units of the projection and of the per-unit weight gradient."""
+    import torch
+    import paper_2410_09397_b200 as attn
+    w = inputs.WORKLOADS["C3"]
+    b, h, n, d = w.batch, w.heads, w.n, w.d
+    sample = [3, 29]
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    A = torch.randn((b, h, n, d), generator=gen, device="cuda").to(torch.bfloat16)
+    G = torch.randn((b, h, n, d), generator=gen, device="cuda").to(torch.bfloat16)
+    for u in sample:      # the sampled units get the repository's own seeded values
+        bi, hi = divmod(u, h)
+        A[bi, hi] = to_dev(inputs.normal_tensor(34, 0, (n, d), bf16=True), "bf16")
+        G[bi, hi] = to_dev(inputs.normal_tensor(34 + u, 3, (n, d), bf16=True), "bf16")
+    W = to_dev(weights(34, 4, h, d, "bf16"), "bf16")
+    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    out = attn.attn_project(A, W, workspace=ws)
+    g = attn.attn_weight_grad(A, G, b * h, workspace=ws)
+    torch.cuda.synchronize()
+    assert attn.attn_workspace_status(ws) == attn.ATTN_OK
+    for u in sample:
+        bi, hi = divmod(u, h)
+        a, gg = to_np(A[bi, hi])[None, None], to_np(G[bi, hi])[None, None]
+        assert rel_err(to_np(out[bi, hi]), orc.project(a, to_np(W[hi])[None])[0, 0]) <= TOL["bf16"]
+        assert rel_err(to_np(g[u]), orc.weight_grad(a, gg, 1)[0]) <= TOL["bf16"]
