@@ -232,6 +232,52 @@ def workload_name(w):
     return f"{w.name}: batch={w.batch} heads={w.heads} n={w.n} d={w.d} {w.dtype} {mask}"
 
 
+def weights_leg(attn, torch, w, dev, peaks, steps=20):
+    """The memory-bound kernels around the attention proper, timed on their own after the main loop: the
+    projection out = A W (S = A1 X, h = A3 Y) and the weight gradient g = A^T G, on tensors of the workload's
+    shape with one weight matrix per head.  Returns per-kernel HBM rooflines (algorithmic bytes / event time)."""
+    elem = 2 if w.bf16 else 4
+    tdtype = torch.bfloat16 if w.bf16 else torch.float32
+    W = torch.from_numpy(inputs.normal_tensor(w.seed, 4, (w.heads, w.d, w.d), bf16=False) / np.sqrt(w.d)).to(tdtype).cuda()
+    out = torch.empty_like(dev["Q"])
+    g = torch.empty((w.heads, w.d, w.d), dtype=torch.float32, device="cuda")
+    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+
+    def step():
+        attn.attn_project(dev["Q"], W, out, workspace=ws)
+        attn.attn_weight_grad(dev["Q"], dev["dO"], w.heads, g, workspace=ws)
+
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    attn.attn_timing_enable(True)
+    attn.attn_timing_collect()
+    ms: dict[str, list[float]] = {}
+    for _ in range(steps):
+        step()
+        for name, t in attn.attn_timing_collect():
+            ms.setdefault(name, []).append(t)
+    attn.attn_timing_enable(False)
+    if attn.attn_workspace_status(ws) != attn.ATTN_OK:
+        raise SystemExit("weight kernel reported a device-side error")
+    units = w.batch * w.heads
+    nbytes = {"wproj": units * w.n * w.d * 2 * elem + w.heads * w.d * w.d * elem,
+              "wgrad": units * w.n * w.d * 2 * elem + w.heads * w.d * w.d * 4}
+    res = {}
+    for name, lst in ms.items():
+        key = name.replace("_simt", "")
+        if key not in nbytes:
+            continue
+        avg = sum(lst) / len(lst)
+        gbs = nbytes[key] / (avg * 1e-3) / 1e9
+        res[name] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": gbs / peaks["hbm_gbs"], "avg_launch_ms": avg, "min_launch_ms": min(lst),
+                     "bytes_per_launch": nbytes[key], "launches_timed": len(lst), "peak_source": peaks["source"]}
+    res["note"] = ("out = A W and g = A^T G on tensors of the workload's shape, one d x d weight per head; "
+                   "timed separately from the step above")
+    return res
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -250,9 +296,11 @@ def main():
                     help="for runs under ncu: allow fewer than 3 warm-up steps, skip e2e and the CPU baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-weights", action="store_true",
+                    help="skip the separately timed projection / weight-gradient kernels")
     args = ap.parse_args()
     if args.profile:
-        args.no_e2e = args.no_cpu_baseline = True
+        args.no_e2e = args.no_cpu_baseline = args.no_weights = True
     elif args.impl == "ours":
         args.warmup = max(args.warmup, 3)
 
@@ -461,6 +509,8 @@ def main():
         line["e2e"] = {"value": fb_all / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
                        "h2d_bytes_per_step": 4 * per, "d2h_bytes_per_step": 3 * per, "ms_per_step": e2e_ms,
                        "note": "backward FLOPs / (H2D of Q,K,V,dO + forward + backward + D2H of dQ,dK,dV)"}
+    if world == 1 and not args.no_weights:
+        line["weights"] = weights_leg(attn, torch, w, dev, peaks)
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(w, bmask)
     print(json.dumps(line), flush=True)

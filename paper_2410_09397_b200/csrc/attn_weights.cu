@@ -25,7 +25,7 @@ __device__ __forceinline__ void red_add_v4(float *p, float a, float b, float c, 
     asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
 
-// ===================================================================== out = A W (bf16)
+// ===================================================================== out = A W (bf16), one tile per CTA (d = 256)
 // One CTA per 128-row tile of one unit.  A tile K-major (contraction along d), W MN-major
 // (rows of W are the contraction index), accumulator [128 rows][HD] in tensor memory.
 template <int HD> struct ProjSmem {
@@ -133,6 +133,183 @@ wproj_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ CUt
     if (warp == 0) tmem_dealloc(tm, kTmemCols);
 }
 
+// ===================================================================== out = A W, persistent (d = 64, 128)
+// CTA c takes a contiguous range of the (unit, 128-row tile) list.  A tiles arrive through a
+// ring of TMA stages, W is loaded when the range starts and again whenever the unit's weight
+// index changes, the accumulator is double-buffered in tensor memory, and the bf16 result
+// leaves through a double-buffered staging tile and TMA stores, so that loads, products and
+// stores of neighbouring tiles overlap.
+template <int HD> struct ProjPSmem {
+    static constexpr int kStages = HD == 128 ? 3 : 4;
+    static constexpr uint32_t kASlab = 128 * 128;
+    static constexpr uint32_t kATile = (HD / 64) * kASlab;
+    static constexpr uint32_t kWSlab = HD * 128;
+    static constexpr uint32_t kW = (HD / 64) * kWSlab;
+    static constexpr uint32_t oA = 0;
+    static constexpr uint32_t oW = oA + kStages * kATile;
+    static constexpr uint32_t oOut = oW + kW;
+    static constexpr uint32_t oBar = oOut + 2 * kATile;
+    static constexpr uint32_t oMisc = oBar + 256;
+    static constexpr uint32_t kBytes = oMisc + 64;
+    static_assert(oW % 1024 == 0 && oOut % 1024 == 0, "tile bases are 1024-byte aligned");
+    static_assert(kBytes <= 227 * 1024, "shared memory budget");
+};
+
+struct ProjPArgs {
+    uint32_t *status;
+    int tiles_per_unit;
+    long total_tiles, weight_units;
+};
+
+template <int HD>
+__global__ void __launch_bounds__(kProjThreads)
+wproj_persistent_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ CUtensorMap mW,
+                        const __grid_constant__ CUtensorMap mOut, const ProjPArgs g)
+{
+    using L = ProjPSmem<HD>;
+    constexpr int kStages = L::kStages;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint64_t *afull = reinterpret_cast<uint64_t *>(smem + L::oBar);
+    uint64_t *aempty = afull + kStages;
+    uint64_t *wfull = aempty + kStages;
+    uint64_t *wfree = wfull + 1;
+    uint64_t *accfull = wfree + 1;
+    uint64_t *accempty = accfull + 2;
+    uint32_t *tmem_base_s = reinterpret_cast<uint32_t *>(smem + L::oMisc);
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(smem + L::oMisc + 4);
+    const Abort ab{abort_flag, g.status};
+    constexpr uint32_t kTmemCols = 2 * HD;
+
+    const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
+    const long t0 = g.total_tiles * blockIdx.x / gridDim.x, t1 = g.total_tiles * (blockIdx.x + 1) / gridDim.x;
+
+    if ((smem_u32(smem) & 1023u) != 0) {
+        if (tid == 0) atomicExch(g.status, 9u);
+        return;
+    }
+    auto load_W = [&](long wi) {
+        mbar_expect_tx(wfull, L::kW);
+#pragma unroll
+        for (int sl = 0; sl < HD / 64; ++sl) tma_load_3d(smem + L::oW + sl * L::kWSlab, &mW, wfull, sl * 64, 0, (int)wi);
+    };
+    auto load_A = [&](int kt, long t) {
+        const int s = kt % kStages;
+        const int unit = (int)(t / g.tiles_per_unit), r0 = (int)(t % g.tiles_per_unit) * 128;
+        mbar_expect_tx(&afull[s], L::kATile);
+#pragma unroll
+        for (int sl = 0; sl < HD / 64; ++sl)
+            tma_load_3d(smem + L::oA + s * L::kATile + sl * L::kASlab, &mA, &afull[s], sl * 64, r0, unit);
+    };
+    // tiles the producer can fetch before anything else is set up: the first ring-full that shares the first weight
+    const long w_first = (t0 / g.tiles_per_unit) % g.weight_units;
+    int early = 0;
+    while (early < kStages && t0 + early < t1 && ((t0 + early) / g.tiles_per_unit) % g.weight_units == w_first) ++early;
+    if (tid == 0) {
+        *abort_flag = 0;
+        for (int b = 0; b < 2; ++b) { mbar_init(&accfull[b], 1); mbar_init(&accempty[b], 128); }
+        fence_barrier_init();
+        prefetch_tensormap(&mOut);
+    }
+    if (tid == 4 * 32) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(&afull[s], 1); mbar_init(&aempty[s], 1); }
+        mbar_init(wfull, 1);
+        mbar_init(wfree, 1);
+        fence_barrier_init();
+        load_W(w_first);
+        for (int kt = 0; kt < early; ++kt) load_A(kt, t0 + kt);
+    }
+    if (warp == 0) tmem_alloc(tmem_base_s, kTmemCols);
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tm = *tmem_base_s;
+
+    if (warp == 4) {
+        if (lane == 0) {
+            int kt = early, wloads = 1;
+            long wprev = w_first;
+            for (long t = t0 + early; t < t1; ++t, ++kt) {
+                const long wi = (t / g.tiles_per_unit) % g.weight_units;
+                if (wi != wprev) {
+                    mbar_wait(wfree, (wloads - 1) & 1, ab);   // products with the old W are done
+                    load_W(wi);
+                    ++wloads;
+                    wprev = wi;
+                }
+                if (kt >= kStages) mbar_wait(&aempty[kt % kStages], ((kt / kStages) - 1) & 1, ab);
+                load_A(kt, t);
+            }
+        }
+    } else if (warp == 5) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = idesc_bf16(128, HD, 0, 1);
+            const uint32_t bW = desc_lo_mnmajor(smem_u32(smem + L::oW), L::kWSlab);
+            int kt = 0, wloads = 0;
+            long wprev = -1;
+            for (long t = t0; t < t1; ++t, ++kt) {
+                const long wi = (t / g.tiles_per_unit) % g.weight_units;
+                if (wi != wprev) {
+                    mbar_wait(wfull, wloads & 1, ab);
+                    ++wloads;
+                    wprev = wi;
+                }
+                const int s = kt % kStages, b = kt & 1;
+                if (kt >= 2) mbar_wait(&accempty[b], ((kt / 2) - 1) & 1, ab);
+                mbar_wait(&afull[s], (kt / kStages) & 1, ab);
+                tcgen05_fence_after();
+                const uint32_t sA = smem_u32(smem + L::oA + s * L::kATile);
+#pragma unroll
+                for (int ks = 0; ks < HD / 16; ++ks)
+                    mma_ss_lo(tm + b * HD, desc_lo_kmajor(sA + (ks / 4) * L::kASlab + (ks % 4) * 32), bW + ks * (2048 >> 4),
+                              idesc, ks > 0);
+                mma_commit(&aempty[s]);
+                mma_commit(&accfull[b]);
+                if (t + 1 < t1 && ((t + 1) / g.tiles_per_unit) % g.weight_units != wi) mma_commit(wfree);
+            }
+        }
+    } else {
+        const int row = warp * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+        int kt = 0;
+        for (long t = t0; t < t1; ++t, ++kt) {
+            const int b = kt & 1;
+            const int unit = (int)(t / g.tiles_per_unit), r0 = (int)(t % g.tiles_per_unit) * 128;
+            uint8_t *stage = smem + L::oOut + b * L::kATile;
+            mbar_wait(&accfull[b], (kt / 2) & 1, ab);
+            tcgen05_fence_after();
+            if (tid == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");   // the store two tiles back has read `stage`
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+#pragma unroll 1
+            for (int c = 0; c < HD; c += 32) {
+                uint32_t v[32];
+                tmem_ld32(tm + lane_addr + b * HD + c, v);
+                tmem_wait_ld();
+                uint8_t *slab = stage + (c / 64) * L::kASlab;
+#pragma unroll
+                for (int e = 0; e < 32; e += 8)
+                    *reinterpret_cast<uint4 *>(slab + sw128_offset(row, (c % 64) + e)) = make_uint4(
+                        pack_bf16(__uint_as_float(v[e]), __uint_as_float(v[e + 1])),
+                        pack_bf16(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3])),
+                        pack_bf16(__uint_as_float(v[e + 4]), __uint_as_float(v[e + 5])),
+                        pack_bf16(__uint_as_float(v[e + 6]), __uint_as_float(v[e + 7])));
+            }
+            tcgen05_fence_before();
+            mbar_arrive(&accempty[b]);
+            fence_proxy_async_smem();
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (tid == 0 && !*abort_flag) {
+#pragma unroll
+                for (int sl = 0; sl < HD / 64; ++sl) tma_store_3d(&mOut, stage + sl * L::kASlab, sl * 64, r0, unit);
+                tma_store_commit();
+            }
+        }
+        if (tid == 0) tma_store_wait_all();
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tm, kTmemCols);
+}
+
 // ===================================================================== g += A^T G (bf16 in, fp32 out)
 // Persistent: CTA c takes a contiguous range of the (unit, row tile) list, accumulates the
 // d x d product of consecutive tiles that belong to the same weight matrix in tensor
@@ -183,13 +360,29 @@ wgrad_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ CUt
         if (tid == 0) atomicExch(g.status, 9u);
         return;
     }
+    auto load_stage = [&](int kt, long t) {
+        const int s = kt % kStages;
+        const int unit = (int)(t / g.tiles_per_unit), r0 = (int)(t % g.tiles_per_unit) * TR;
+        uint8_t *sA = smem + s * L::kStage, *sG = sA + L::kTile;
+        mbar_expect_tx(&full[s], L::kStage);
+#pragma unroll
+        for (int sl = 0; sl < HD / 64; ++sl) {
+            tma_load_3d(sA + sl * L::kSlab, &mA, &full[s], sl * 64, r0, unit);
+            tma_load_3d(sG + sl * L::kSlab, &mG, &full[s], sl * 64, r0, unit);
+        }
+    };
+    const int early = (int)((t1 - t0) < kStages ? (t1 - t0) : kStages);
     if (tid == 0) {
         *abort_flag = 0;
-        for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
         mbar_init(done, 1);
         mbar_init(tfree, 128);
         fence_barrier_init();
-        prefetch_tensormap(&mA); prefetch_tensormap(&mG);
+    }
+    if (tid == 4 * 32) {
+        // the producer sets up its own ring and fills it before the CTA-wide setup is over
+        for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        fence_barrier_init();
+        for (int kt = 0; kt < early; ++kt) load_stage(kt, t0 + kt);
     }
     if (HD == 64) {
         for (uint32_t i = tid; i < L::kSlab / 16; i += kGradThreads)
@@ -204,18 +397,10 @@ wgrad_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ CUt
 
     if (warp == 4) {
         if (lane == 0) {
-            int kt = 0;
-            for (long t = t0; t < t1; ++t, ++kt) {
-                const int s = kt % kStages;
-                if (kt >= kStages) mbar_wait(&empty[s], ((kt / kStages) - 1) & 1, ab);
-                const int unit = (int)(t / g.tiles_per_unit), r0 = (int)(t % g.tiles_per_unit) * TR;
-                uint8_t *sA = smem + s * L::kStage, *sG = sA + L::kTile;
-                mbar_expect_tx(&full[s], L::kStage);
-#pragma unroll
-                for (int sl = 0; sl < HD / 64; ++sl) {
-                    tma_load_3d(sA + sl * L::kSlab, &mA, &full[s], sl * 64, r0, unit);
-                    tma_load_3d(sG + sl * L::kSlab, &mG, &full[s], sl * 64, r0, unit);
-                }
+            int kt = early;
+            for (long t = t0 + early; t < t1; ++t, ++kt) {
+                mbar_wait(&empty[kt % kStages], ((kt / kStages) - 1) & 1, ab);
+                load_stage(kt, t);
             }
         }
     } else if (warp == 5) {
@@ -381,6 +566,32 @@ attn_status launch_project(const void *A, const void *W, void *out, int n, long 
 }
 
 template <int HD>
+attn_status launch_project_persistent(const void *A, const void *W, void *out, int n, long BH, long wu, uint32_t *status,
+                                      cudaStream_t s)
+{
+    using L = ProjPSmem<HD>;
+    CUtensorMap mA, mW, mOut;
+    if (!make_tmap_bf16_3d(&mA, A, HD, (uint64_t)n, (uint64_t)BH, 128) ||
+        !make_tmap_bf16_3d(&mW, W, HD, HD, (uint64_t)wu, HD) ||
+        !make_tmap_bf16_3d(&mOut, out, HD, (uint64_t)n, (uint64_t)BH, 128))
+        return ATTN_ERR_LAUNCH;
+    if (cudaFuncSetAttribute(wproj_persistent_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::kBytes) !=
+        cudaSuccess)
+        return ATTN_ERR_LAUNCH;
+    ProjPArgs a{};
+    a.status = status;
+    a.tiles_per_unit = (n + 127) / 128;
+    a.total_tiles = (long)a.tiles_per_unit * BH;
+    a.weight_units = wu;
+    const long ctas = (long)sm_count() * (HD == 64 ? 2 : 1);
+    const unsigned grid = (unsigned)(a.total_tiles < ctas ? a.total_tiles : ctas);
+    launch_begin("wproj", s);
+    wproj_persistent_kernel<HD><<<grid, kProjThreads, L::kBytes, s>>>(mA, mW, mOut, a);
+    launch_end(s);
+    return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_LAUNCH;
+}
+
+template <int HD>
 attn_status launch_grad(const void *A, const void *G, float *g, int n, long BH, long wu, uint32_t *status, cudaStream_t s)
 {
     using L = GradSmem<HD>;
@@ -431,9 +642,9 @@ attn_status project_impl(const void *A, const void *W, void *out, int n, int d, 
                          cudaStream_t s)
 {
     if (use_tc(d, dt)) {
-        if (d == 64) return launch_project<64>(A, W, out, n, BH, wu, status, s);
-        if (d == 128) return launch_project<128>(A, W, out, n, BH, wu, status, s);
-        return launch_project<256>(A, W, out, n, BH, wu, status, s);
+        if (d == 64) return launch_project_persistent<64>(A, W, out, n, BH, wu, status, s);
+        if (d == 128) return launch_project_persistent<128>(A, W, out, n, BH, wu, status, s);
+        return launch_project<256>(A, W, out, n, BH, wu, status, s);   // W alone takes 128 KB: one tile per CTA
     }
     if (dt == ATTN_F32) return launch_simt_project<float>(A, W, out, n, d, BH, wu, s);
     return launch_simt_project<__nv_bfloat16>(A, W, out, n, d, BH, wu, s);
