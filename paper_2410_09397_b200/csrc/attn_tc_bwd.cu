@@ -844,6 +844,328 @@ tc_bwd_kernel_v2(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
 }
 
 // ---------------------------------------------------------------------------------------
+// d = 128, dK and dV only: the key-stationary half of the path without atomics (dQ comes from the
+// query-stationary kernel).  Without the dQ product dS^T never has to be in shared memory: it
+// is written over dP^T in tensor memory as bf16 pairs, exactly as P^T over S^T, and
+// dK += dS^T Q takes it from there.  The 32 KB this frees hold a third Q stage, and Q, dO and
+// the row statistics are released separately (dO after dV, Q after dK, LSE / D after the dS
+// phase), so loads run up to two tiles ahead.  Products execute on the tensor pipe in issue
+// order, so S^T of tile k+1 is queued right behind dV of tile k, and dP^T of tile k+1 behind
+// dK of tile k, with no wait in between.
+struct DkdvSmem {
+    static constexpr uint32_t kTile = 2 * SLAB;             // one [128][128] bf16 tile
+    static constexpr uint32_t oK = 0;
+    static constexpr uint32_t oV = oK + kTile;
+    static constexpr uint32_t oQ = oV + kTile;              // 3 stages
+    static constexpr uint32_t odO = oQ + 3 * kTile;         // 2 stages
+    static constexpr uint32_t oLSE = odO + 2 * kTile;       // 2 stages x 128 floats
+    static constexpr uint32_t oD = oLSE + 2 * 128 * 4;
+    static constexpr uint32_t oBar = oD + 2 * 128 * 4;
+    static constexpr uint32_t oMisc = oBar + 24 * 8;
+    static constexpr uint32_t kBytes = oMisc + 64;
+    static_assert(kBytes <= 227 * 1024, "shared memory budget");
+};
+enum { KD_KV = 0, KD_QFULL = 1, KD_QEMPTY = 4, KD_OFULL = 7, KD_OEMPTY = 9, KD_LFULL = 11, KD_LEMPTY = 13,
+       KD_S = 15, KD_DP = 17, KD_P = 19, KD_DS = 21, KD_DONE = 23 };
+constexpr int kThreadsDkdv = 512 + 64;   // 16 exp/dS warps, MMA issuer warp, TMA producer warp
+
+__global__ void __launch_bounds__(kThreadsDkdv, 1)
+tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mK_,
+                   const __grid_constant__ CUtensorMap mV, const __grid_constant__ CUtensorMap mdO, const BwdArgs a)
+{
+    constexpr int HD = 128;
+    constexpr int kHalfThreads = 256;
+    using L = DkdvSmem;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::oBar);
+    uint32_t *tmem_base_s = reinterpret_cast<uint32_t *>(smem + L::oMisc);
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(smem + L::oMisc + 4);
+    const Abort ab{abort_flag, a.status};
+
+    const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
+    const int jt = blockIdx.x / a.group;
+    const long bh = (long)blockIdx.y * a.group + blockIdx.x % a.group;
+    const int j0 = jt * TK, n = a.n;
+
+    if ((smem_u32(smem) & 1023u) != 0) {
+        if (tid == 0) atomicExch(a.status, 9u);
+        return;
+    }
+    if (tid == 0) {
+        *abort_flag = 0;
+        mbar_init(&bars[KD_KV], 1);
+        for (int s = 0; s < 3; ++s) { mbar_init(&bars[KD_QFULL + s], 1); mbar_init(&bars[KD_QEMPTY + s], 1); }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&bars[KD_OFULL + s], 1);
+            mbar_init(&bars[KD_OEMPTY + s], 1);
+            mbar_init(&bars[KD_LFULL + s], 1);
+            mbar_init(&bars[KD_LEMPTY + s], 2 * kHalfThreads);
+            mbar_init(&bars[KD_S + s], 1);
+            mbar_init(&bars[KD_DP + s], 1);
+            mbar_init(&bars[KD_P + s], kHalfThreads);
+            mbar_init(&bars[KD_DS + s], kHalfThreads);
+        }
+        mbar_init(&bars[KD_DONE], 1);
+        fence_barrier_init();
+        prefetch_tensormap(&mQ); prefetch_tensormap(&mK_); prefetch_tensormap(&mV); prefetch_tensormap(&mdO);
+    }
+    if (warp == 0) tmem_alloc(tmem_base_s, 512);
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tm = *tmem_base_s;
+    const uint32_t T_S = tm, T_dP = tm + 128, T_dV = tm + 256, T_dK = tm + 256 + HD;
+    constexpr uint32_t HALF_ROWS = 64 * 128;   // byte offset of rows 64.. inside a [128][64] slab
+
+    const TileIter iter(a, jt, bh);
+
+    if (warp == 17) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            mbar_expect_tx(&bars[KD_KV], 2 * L::kTile);
+#pragma unroll
+            for (uint32_t sl = 0; sl < 2; ++sl) {
+                tma_load_3d(smem + L::oK + sl * SLAB, &mK_, &bars[KD_KV], sl * 64, j0, (int)bh);
+                tma_load_3d(smem + L::oV + sl * SLAB, &mV, &bars[KD_KV], sl * 64, j0, (int)bh);
+            }
+            int k = 0;
+            for (int idx = 0; idx < iter.raw; ++idx) {
+                const int it = iter.tile(idx);
+                if (it < 0) continue;
+                const int i0 = it * TQ, sq = k % 3, s2 = k & 1;
+                const uint32_t rows = min(TQ, n - i0);
+                if (k >= 3) mbar_wait(&bars[KD_QEMPTY + sq], ((k / 3) - 1) & 1, ab);
+                mbar_expect_tx(&bars[KD_QFULL + sq], L::kTile);
+#pragma unroll
+                for (uint32_t sl = 0; sl < 2; ++sl)
+                    tma_load_3d(smem + L::oQ + sq * L::kTile + sl * SLAB, &mQ, &bars[KD_QFULL + sq], sl * 64, i0, (int)bh);
+                if (k >= 2) mbar_wait(&bars[KD_LEMPTY + s2], ((k >> 1) - 1) & 1, ab);
+                mbar_expect_tx(&bars[KD_LFULL + s2], 2 * rows * 4);
+                bulk_load_1d(smem + L::oLSE + s2 * 512, a.nLSE2 + bh * n + i0, rows * 4, &bars[KD_LFULL + s2]);
+                bulk_load_1d(smem + L::oD + s2 * 512, a.Ds + bh * n + i0, rows * 4, &bars[KD_LFULL + s2]);
+                if (k >= 2) mbar_wait(&bars[KD_OEMPTY + s2], ((k >> 1) - 1) & 1, ab);
+                mbar_expect_tx(&bars[KD_OFULL + s2], L::kTile);
+#pragma unroll
+                for (uint32_t sl = 0; sl < 2; ++sl)
+                    tma_load_3d(smem + L::odO + s2 * L::kTile + sl * SLAB, &mdO, &bars[KD_OFULL + s2], sl * 64, i0, (int)bh);
+                ++k;
+            }
+        }
+    } else if (warp == 16) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = idesc_bf16(128, 128, 0, 0);       // S^T, dP^T
+            constexpr uint32_t idesc_dv = idesc_bf16(128, HD, 0, 1);       // dV, dK: A in tensor memory, B MN-major
+            const uint32_t kK = desc_lo_kmajor(smem_u32(smem + L::oK)), kV = desc_lo_kmajor(smem_u32(smem + L::oV));
+            constexpr uint32_t kHalf = HALF_ROWS >> 4, kSlab = SLAB >> 4;
+            auto issue_S = [&](int k) {
+                const uint32_t kQ = desc_lo_kmajor(smem_u32(smem + L::oQ + (k % 3) * L::kTile));
+#pragma unroll
+                for (int kk = 0; kk < HD / 16; ++kk) {
+                    const uint32_t off = (kk / 4) * kSlab + (kk % 4) * 2;
+                    mma_ss_lo(T_S, kK + off, kQ + off, idesc_s, kk > 0);
+                }
+                mma_commit(&bars[KD_S]);
+                mma_commit(&bars[KD_S + 1]);
+            };
+            auto issue_dP = [&](int k) {
+                const uint32_t kdO = desc_lo_kmajor(smem_u32(smem + L::odO + (k & 1) * L::kTile));
+#pragma unroll
+                for (int kk = 0; kk < HD / 16; ++kk) {
+                    const uint32_t off = (kk / 4) * kSlab + (kk % 4) * 2;
+                    mma_ss_lo(T_dP, kV + off, kdO + off, idesc_s, kk > 0);
+                }
+                mma_commit(&bars[KD_DP]);
+                mma_commit(&bars[KD_DP + 1]);
+            };
+            int idx = 0, it = -1;
+            while (idx < iter.raw && (it = iter.tile(idx)) < 0) ++idx;
+            if (it >= 0) {
+                mbar_wait(&bars[KD_KV], 0, ab);
+                mbar_wait(&bars[KD_QFULL], 0, ab);
+                tcgen05_fence_after();
+                issue_S(0);
+                mbar_wait(&bars[KD_OFULL], 0, ab);
+                tcgen05_fence_after();
+                issue_dP(0);
+            }
+            int k = 0;
+            while (idx < iter.raw) {
+                int nidx = idx + 1, nit = -1;
+                while (nidx < iter.raw && (nit = iter.tile(nidx)) < 0) ++nidx;
+                const uint32_t mdO_ = desc_lo_mnmajor(smem_u32(smem + L::odO + (k & 1) * L::kTile), SLAB);
+                const uint32_t mQ_ = desc_lo_mnmajor(smem_u32(smem + L::oQ + (k % 3) * L::kTile), SLAB);
+                // dV += P_h^T dO_h
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    mbar_wait(&bars[KD_P + h], k & 1, ab);
+                    tcgen05_fence_after();
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        mma_ts_lo(T_dV, T_S + 64 * h + (kk < 2 ? kk * 8 : 48 + (kk - 2) * 8), mdO_ + h * kHalf + kk * 128,
+                                  idesc_dv, (k > 0) || (h > 0) || (kk > 0));
+                }
+                mma_commit(&bars[KD_OEMPTY + (k & 1)]);
+                if (nit >= 0) {
+                    mbar_wait(&bars[KD_QFULL + (k + 1) % 3], ((k + 1) / 3) & 1, ab);
+                    tcgen05_fence_after();
+                    issue_S(k + 1);
+                }
+                // dK += dS_h^T Q_h
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    mbar_wait(&bars[KD_DS + h], k & 1, ab);
+                    tcgen05_fence_after();
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        mma_ts_lo(T_dK, T_dP + 64 * h + (kk < 2 ? kk * 8 : 48 + (kk - 2) * 8), mQ_ + h * kHalf + kk * 128,
+                                  idesc_dv, (k > 0) || (h > 0) || (kk > 0));
+                }
+                mma_commit(&bars[KD_QEMPTY + k % 3]);
+                if (nit >= 0) {
+                    mbar_wait(&bars[KD_OFULL + ((k + 1) & 1)], ((k + 1) >> 1) & 1, ab);
+                    tcgen05_fence_after();
+                    issue_dP(k + 1);
+                }
+                ++k;
+                idx = nidx;
+            }
+            mma_commit(&bars[KD_DONE]);
+        }
+    } else {
+        // ------------------------------------------------------------ warpgroup 2h + qq owns queries 64 h + 32 qq .. + 31
+        const int h = warp / 8, qq = (warp / 4) & 1;
+        const int row = (warp % 4) * 32 + lane;        // tensor-memory lane = key row inside the tile
+        const uint32_t lane_addr = (uint32_t)((warp % 4) * 32) << 16;
+        const int jg = j0 + row;
+        const float sl2 = a.scale * 1.4426950408889634f;
+        int k = 0;
+        for (int idx = 0; idx < iter.raw; ++idx) {
+            const int it = iter.tile(idx);
+            if (it < 0) continue;
+            const int s2 = k & 1, i0 = it * TQ;
+            const float4 *sNL = reinterpret_cast<const float4 *>(smem + L::oLSE + s2 * 512 + h * 256 + qq * 128);
+            const float4 *sDs = reinterpret_cast<const float4 *>(smem + L::oD + s2 * 512 + h * 256 + qq * 128);
+            const bool diag = a.mask_kind == ATTN_MASK_CAUSAL && it == jt;
+            const bool masked = diag || i0 + TQ > n || j0 + TK > n;
+            const int ig0 = i0 + h * 64 + qq * 32;
+            const uint32_t c0 = h * 64 + qq * 32;      // this thread's first column in T_S / T_dP
+            // bf16 pairs go over columns this very thread has just read -- quarter 0 to columns
+            // 0..15 of the half, quarter 1 to columns 48..63 -- so no thread overwrites entries
+            // another thread still has to read
+            const uint32_t cpack = h * 64 + qq * 48;
+            mbar_wait(&bars[KD_LFULL + s2], (k >> 1) & 1, ab);
+            mbar_wait(&bars[KD_S + h], k & 1, ab);
+            tcgen05_fence_after();
+            float p[32];
+            {
+                uint32_t sv0[32];
+                tmem_ld32(T_S + lane_addr + c0, sv0);
+                tmem_wait_ld();
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const float4 nl = sNL[q];
+                    const uint32_t *sv = &sv0[q * 4];
+                    p[q * 4 + 0] = ex2_approx(fmaf(__uint_as_float(sv[0]), sl2, nl.x));
+                    p[q * 4 + 1] = ex2_approx(fmaf(__uint_as_float(sv[1]), sl2, nl.y));
+                    p[q * 4 + 2] = ex2_approx(fmaf(__uint_as_float(sv[2]), sl2, nl.z));
+                    p[q * 4 + 3] = ex2_approx(fmaf(__uint_as_float(sv[3]), sl2, nl.w));
+                }
+            }
+            if (masked) {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                    const int ig = ig0 + e;
+                    const bool ok = ig < n && jg < n && (!diag || jg <= ig);
+                    p[e] = ok ? p[e] : 0.f;
+                }
+            }
+            {
+                uint32_t ppack[16];
+#pragma unroll
+                for (int e = 0; e < 16; ++e) ppack[e] = pack_bf16(p[2 * e], p[2 * e + 1]);
+                tmem_st16(T_S + lane_addr + cpack, ppack);
+                tmem_wait_st();
+            }
+            tcgen05_fence_before();
+            mbar_arrive(&bars[KD_P + h]);
+
+            mbar_wait(&bars[KD_DP + h], k & 1, ab);
+            tcgen05_fence_after();
+            {
+                uint32_t dv0[32], dpack[16];
+                tmem_ld32(T_dP + lane_addr + c0, dv0);
+                tmem_wait_ld();
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const float4 dsc = sDs[q];
+                    const uint32_t *dv = &dv0[q * 4];
+                    // a masked entry has p = 0 and a finite dP, so its dS is an exact zero
+                    const float d0 = p[q * 4 + 0] * fmaf(__uint_as_float(dv[0]), a.scale, -dsc.x);
+                    const float d1 = p[q * 4 + 1] * fmaf(__uint_as_float(dv[1]), a.scale, -dsc.y);
+                    const float d2 = p[q * 4 + 2] * fmaf(__uint_as_float(dv[2]), a.scale, -dsc.z);
+                    const float d3 = p[q * 4 + 3] * fmaf(__uint_as_float(dv[3]), a.scale, -dsc.w);
+                    dpack[q * 2 + 0] = pack_bf16(d0, d1);
+                    dpack[q * 2 + 1] = pack_bf16(d2, d3);
+                }
+                if (masked) {
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        if (p[2 * e] == 0.f) dpack[e] &= 0xffff0000u;
+                        if (p[2 * e + 1] == 0.f) dpack[e] &= 0x0000ffffu;
+                    }
+                }
+                tmem_st16(T_dP + lane_addr + cpack, dpack);
+                tmem_wait_st();
+            }
+            tcgen05_fence_before();
+            mbar_arrive(&bars[KD_DS + h]);
+            mbar_arrive(&bars[KD_LEMPTY + s2]);
+            ++k;
+        }
+        // ------------------------------------------------------------ epilogue: dV_j, dK_j (32 columns per warpgroup)
+        if (k > 0) {
+            mbar_wait(&bars[KD_DONE], 0, ab);
+            tcgen05_fence_after();
+        }
+        {
+            const int cq = (warp / 4) * 32;
+            const int jc = jg < n ? jg : 0;
+            __nv_bfloat16 *pv = a.dV + ((size_t)bh * n + jc) * HD + cq;
+            __nv_bfloat16 *pk = a.dK + ((size_t)bh * n + jc) * HD + cq;
+            uint32_t v[32], w[32];
+            if (k > 0) {
+                tmem_ld32(T_dV + lane_addr + cq, v);
+                tmem_ld32(T_dK + lane_addr + cq, w);
+                tmem_wait_ld();
+            } else {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) v[e] = w[e] = 0u;
+            }
+            if (jg < n) {
+#pragma unroll
+                for (int e = 0; e < 32; e += 8) {
+                    uint4 ov, ok;
+                    ov.x = pack_bf16(__uint_as_float(v[e]), __uint_as_float(v[e + 1]));
+                    ov.y = pack_bf16(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
+                    ov.z = pack_bf16(__uint_as_float(v[e + 4]), __uint_as_float(v[e + 5]));
+                    ov.w = pack_bf16(__uint_as_float(v[e + 6]), __uint_as_float(v[e + 7]));
+                    ok.x = pack_bf16(__uint_as_float(w[e]), __uint_as_float(w[e + 1]));
+                    ok.y = pack_bf16(__uint_as_float(w[e + 2]), __uint_as_float(w[e + 3]));
+                    ok.z = pack_bf16(__uint_as_float(w[e + 4]), __uint_as_float(w[e + 5]));
+                    ok.w = pack_bf16(__uint_as_float(w[e + 6]), __uint_as_float(w[e + 7]));
+                    *reinterpret_cast<uint4 *>(pv + e) = ov;
+                    *reinterpret_cast<uint4 *>(pk + e) = ok;
+                }
+            }
+        }
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tm, 512);
+}
+
+// ---------------------------------------------------------------------------------------
 // d = 128, pipelined variant with reducer warps.  As tc_bwd_kernel_v2<true>, plus eight warps
 // (16-23) that do nothing but move finished dQ^T tiles from tensor memory into the fp32
 // accumulator: the red.global.add queue stalls them, not the warps on the tile loop.  To fit
@@ -1245,6 +1567,10 @@ attn_status launch_bwd(const Problem &p)
         if (cudaFuncSetAttribute(tc_bwd_kernel_v4, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::kBytes) != cudaSuccess)
             return ATTN_ERR_LAUNCH;
         tc_bwd_kernel_v4<<<grid, kThreadsV4, L::kBytes, p.stream>>>(mQ, mK, mV, mdO, a);
+    } else if (HD == 128 && !WITH_DQ) {
+        if (cudaFuncSetAttribute(tc_bwd_dkdv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DkdvSmem::kBytes) != cudaSuccess)
+            return ATTN_ERR_LAUNCH;
+        tc_bwd_dkdv_kernel<<<grid, kThreadsDkdv, DkdvSmem::kBytes, p.stream>>>(mQ, mK, mV, mdO, a);
     } else if (HD == 128) {
         if (cudaFuncSetAttribute(tc_bwd_kernel_v2<WITH_DQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::kBytes) != cudaSuccess)
             return ATTN_ERR_LAUNCH;
