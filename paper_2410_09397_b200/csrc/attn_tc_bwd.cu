@@ -1171,7 +1171,13 @@ tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
 // accumulator: the red.global.add queue stalls them, not the warps on the tile loop.  To fit
 // 25 warps in the register file the exp/dS warps keep P only as the bf16 pairs they hand to
 // the dV product, and form dS from those.
-constexpr int kThreadsV4 = 256 + 256 + 64;   // 8 exp/dS warps, 8 reducer warps, issuer warp, TMA producer warp
+constexpr int kThreadsV4 = 256 + 256 + 128;  // 8 exp/dS warps, 8 reducer warps, issuer warp, TMA producer warp, 2 idle warps
+// Registers per thread after the warpgroups have traded them (setmaxnreg): the kernel starts with 96 everywhere;
+// the issuer / producer warpgroup and the reducers give up 40 and 16 each, which the exp / dS warpgroups take:
+// 256 x 128 + 256 x 80 + 128 x 56 = 60,416 of the 61,440 allocated at launch.
+constexpr int kRegsExp = 120, kRegsReduce = 80, kRegsIssue = 72;
+template <int N> __device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 __global__ void __launch_bounds__(kThreadsV4, 1)
 tc_bwd_kernel_v4(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mK_,
                  const __grid_constant__ CUtensorMap mV, const __grid_constant__ CUtensorMap mdO, const BwdArgs a)
@@ -1225,7 +1231,11 @@ tc_bwd_kernel_v4(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
 
     const TileIter iter(a, jt, bh);
 
-    if (warp == 17) {
+    if (warp >= 16) {
+        setmaxnreg_dec<kRegsIssue>();   // whole warpgroup 16-19; warps 18 and 19 exist only to complete it
+    }
+    if (warp >= 18) {
+    } else if (warp == 17) {
         // ------------------------------------------------------------ TMA producer: every load, as soon as its stage is free
         if (lane == 0) {
             auto issue_load = [&](int it, int s) {
@@ -1341,6 +1351,7 @@ tc_bwd_kernel_v4(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
             }
         }
     } else if (warp >= 8) {
+        setmaxnreg_dec<kRegsReduce>();
         // ------------------------------------------------------------ reducers: dQ_h^T tile -> fp32 accumulator
         // lanes = head-dimension index c, columns = queries: one warp instruction adds 128 contiguous bytes
         const int h = (warp - 8) / 4;
@@ -1377,6 +1388,7 @@ tc_bwd_kernel_v4(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
         }
     } else {
         // ------------------------------------------------------------ warpgroup h owns queries 64 h .. 64 h + 63 of every tile
+        setmaxnreg_inc<kRegsExp>();
         const int h = warp / 4;
         const int row = (warp % 4) * 32 + lane;        // tensor-memory lane = key row inside the tile
         const uint32_t lane_addr = (uint32_t)((warp % 4) * 32) << 16;
@@ -1397,12 +1409,14 @@ tc_bwd_kernel_v4(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
             mbar_wait(&bars[V2_S + h], k & 1, ab);
             tcgen05_fence_after();
             uint32_t ppack[32];   // P as bf16 pairs: what dV uses, and what dS is formed from
+            uint32_t svb[2][16];   // two chunks in flight: the load of chunk ch + 1 runs under the arithmetic of chunk ch
+            tmem_ld16(T_S + lane_addr + c0, svb[0]);
 #pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {   // 16 columns at a time keeps the register count down
+            for (int ch = 0; ch < 4; ++ch) {   // 16 columns at a time
                 float p[16];
-                uint32_t sv0[16];
-                tmem_ld16(T_S + lane_addr + c0 + ch * 16, sv0);
                 tmem_wait_ld();
+                if (ch < 3) tmem_ld16(T_S + lane_addr + c0 + (ch + 1) * 16, svb[(ch + 1) & 1]);
+                const uint32_t *sv0 = svb[ch & 1];
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                     const float4 nl = sNL[ch * 4 + q];
@@ -1434,11 +1448,13 @@ tc_bwd_kernel_v4(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
             tcgen05_fence_after();
             {
                 uint8_t *slab = smem + L::odS + h * SLAB;
+                uint32_t dvb[2][16];
+                tmem_ld16(T_dP + lane_addr + c0, dvb[0]);
 #pragma unroll
                 for (int ch = 0; ch < 4; ++ch) {
-                    uint32_t dv[16];
-                    tmem_ld16(T_dP + lane_addr + c0 + ch * 16, dv);
                     tmem_wait_ld();
+                    if (ch < 3) tmem_ld16(T_dP + lane_addr + c0 + (ch + 1) * 16, dvb[(ch + 1) & 1]);
+                    const uint32_t *dv = dvb[ch & 1];
 #pragma unroll
                     for (int g = 0; g < 2; ++g) {    // 8 query columns = one 16-byte chunk
                         float ds[8], p[8];
