@@ -1178,12 +1178,14 @@ constexpr int kThreadsV4 = 256 + 256 + 128;  // 8 exp/dS warps, 8 reducer warps,
 constexpr int kRegsExp = 120, kRegsReduce = 80, kRegsIssue = 72;
 template <int N> __device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int HD>
 __global__ void __launch_bounds__(kThreadsV4, 1)
 tc_bwd_kernel_v4(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mK_,
                  const __grid_constant__ CUtensorMap mV, const __grid_constant__ CUtensorMap mdO, const BwdArgs a)
 {
-    constexpr int HD = 128;
     constexpr bool WITH_DQ = true;
+    // d = 64: the dQ^T product needs M = 128, so the K tile's second 64-wide slab of M is an all-zero slab
+    constexpr uint32_t oZero = (BwdSmem<HD>::kBytes + 1023u) & ~1023u;
     constexpr int kHalfThreads = 128;     // exp / dS threads per half
     constexpr int kReduceThreads = 128;   // reducer threads per half
     using L = BwdSmem<HD>;
@@ -1220,6 +1222,10 @@ tc_bwd_kernel_v4(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
         }
         fence_barrier_init();
         prefetch_tensormap(&mQ); prefetch_tensormap(&mK_); prefetch_tensormap(&mV); prefetch_tensormap(&mdO);
+    }
+    if (HD == 64) {
+        for (uint32_t i = tid; i < SLAB / 16; i += kThreadsV4) reinterpret_cast<uint4 *>(smem + oZero)[i] = make_uint4(0, 0, 0, 0);
+        fence_proxy_async_smem();
     }
     if (warp == 0) tmem_alloc(tmem_base_s, 512);
     tcgen05_fence_before();
@@ -1274,7 +1280,7 @@ tc_bwd_kernel_v4(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
             constexpr uint32_t idesc_dq = idesc_bf16(128, 128, 1, 1);      // dQ^T
             // low descriptor words (tc_common.cuh): per-step offsets are added as (bytes >> 4)
             const uint32_t kK = desc_lo_kmajor(smem_u32(smem + L::oK)), kV = desc_lo_kmajor(smem_u32(smem + L::oV));
-            const uint32_t mK = desc_lo_mnmajor(smem_u32(smem + L::oK), SLAB);
+            const uint32_t mK = desc_lo_mnmajor(smem_u32(smem + L::oK), HD == 64 ? oZero - L::oK : SLAB);
             const uint32_t kdS = desc_lo_kmajor(smem_u32(smem + L::odS)), mdS = desc_lo_mnmajor(smem_u32(smem + L::odS), SLAB);
             constexpr uint32_t kHalf = HALF_ROWS >> 4, kSlab = SLAB >> 4;
             // S^T = K_j Q_i^T for the whole tile in stage s; one commit per half's barrier
@@ -1365,13 +1371,17 @@ tc_bwd_kernel_v4(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
             mbar_wait(&bars[V2_DQ + h], k & 1, ab);
             tcgen05_fence_after();
             uint32_t v0[32], v1[32];
-            tmem_ld32(T_dP + lane_addr + h * 64, v0);
-            tmem_ld32(T_dP + lane_addr + h * 64 + 32, v1);
-            tmem_wait_ld();
+            const bool live = (warp % 4) * 32 < HD;   // d = 64: lanes 64..127 of the padded product hold zeros
+            if (live) {
+                tmem_ld32(T_dP + lane_addr + h * 64, v0);
+                tmem_ld32(T_dP + lane_addr + h * 64 + 32, v1);
+                tmem_wait_ld();
+            }
             tcgen05_fence_before();
             mbar_arrive(&bars[V2_DQDONE + h]);   // T_dP half h is free again; the reductions proceed from registers
             float *base = a.dQ_acc + ((size_t)bh * n + ig0) * HD + row;
-            if (ig0 + 64 <= n) {
+            if (!live) {
+            } else if (ig0 + 64 <= n) {
 #pragma unroll
                 for (int e = 0; e < 32; ++e) red_add_f32(base + (size_t)e * HD, __uint_as_float(v0[e]));
 #pragma unroll
@@ -1496,10 +1506,10 @@ tc_bwd_kernel_v4(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
         }
         {
             constexpr int HALF = 32;
-            const int cq0 = (warp / 4) * 64;
+            const int cq0 = (warp / 4) * (HD / 2);
             const int jc = jg < n ? jg : 0;
 #pragma unroll
-            for (int cq = cq0; cq < cq0 + 64; cq += 32) {
+            for (int cq = cq0; cq < cq0 + HD / 2; cq += 32) {
                 __nv_bfloat16 *pv = a.dV + ((size_t)bh * n + jc) * HD + cq;
                 __nv_bfloat16 *pk = a.dK + ((size_t)bh * n + jc) * HD + cq;
                 uint32_t v[32], w[32];
@@ -1579,10 +1589,11 @@ attn_status launch_bwd(const Problem &p)
     }
     const dim3 grid((unsigned)((p.n + TK - 1) / TK * a.group), (unsigned)(p.BH / a.group));
     launch_begin(WITH_DQ ? "tc_bwd_fused" : "tc_bwd_dkdv", p.stream);
-    if (HD == 128 && WITH_DQ && kReducerWarps) {
-        if (cudaFuncSetAttribute(tc_bwd_kernel_v4, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::kBytes) != cudaSuccess)
+    if (WITH_DQ && kReducerWarps) {
+        constexpr uint32_t bytes = HD == 64 ? ((L::kBytes + 1023u) & ~1023u) + SLAB : L::kBytes;
+        if (cudaFuncSetAttribute(tc_bwd_kernel_v4<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
             return ATTN_ERR_LAUNCH;
-        tc_bwd_kernel_v4<<<grid, kThreadsV4, L::kBytes, p.stream>>>(mQ, mK, mV, mdO, a);
+        tc_bwd_kernel_v4<HD><<<grid, kThreadsV4, bytes, p.stream>>>(mQ, mK, mV, mdO, a);
     } else if (HD == 128 && !WITH_DQ) {
         if (cudaFuncSetAttribute(tc_bwd_dkdv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DkdvSmem::kBytes) != cudaSuccess)
             return ATTN_ERR_LAUNCH;
