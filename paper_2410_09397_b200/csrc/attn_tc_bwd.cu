@@ -13,17 +13,19 @@
 //                                                        the scale of dQ and dK is folded in here)
 //   dV_j += P^T  dO_i      A = P^T  in tensor memory (bf16), B = dO_i MN-major smem
 //   dK_j += dS^T Q_i       A = dS^T K-major smem,            B = Q_i  MN-major smem
-//   dQ_i += dS K_j         computed as dQ^T = K_j^T dS^T for d = 128 (so that the fp32
-//                          reductions into global memory are coalesced), as dS K_j for d = 64
+//   dQ_i += dS K_j         computed as dQ^T = K_j^T dS^T (lane = head-dimension index), so that
+//                          the fp32 reductions into global memory are coalesced; at d = 64 the
+//                          product is padded to M = 128 with an all-zero slab
 //
 // dQ partial tiles are added into an fp32 accumulator in the workspace with
 // red.global.add (the one place where summation order is not fixed); a small kernel
 // converts it to bf16 at the end.  Tensor memory (512 columns): S^T / P^T 128,
-// dP^T then dQ 128, dV d, dK d.
+// dP^T then dQ^T 128, dV d, dK d.
 //
-// Roles: warps 0-7 = two warpgroups that split the 128 query columns of each tile
-// between them (softmax, dS, dQ reduction, epilogue); warp 8 lane 0 = TMA producer and
-// MMA issuer.  All waits are bounded (tc_common.cuh).
+// Two kernels: tc_bwd_kernel_v4 (all five products, the default) and tc_bwd_dkdv_kernel
+// (without the dQ product; `deterministic = 1` pairs it with the query-stationary dQ kernel of
+// attn_tc_bwd_dq.cu).  Warp roles are described at each kernel.  All waits are bounded
+// (tc_common.cuh).
 #include "attn_internal.h"
 #include "tc_common.cuh"
 
@@ -33,15 +35,7 @@ namespace {
 using namespace tc;
 
 constexpr int TQ = 128, TK = 128;
-constexpr int kSoftmaxThreads = 256;
-constexpr int kThreads = kSoftmaxThreads + 32;
-constexpr int kThreadsV2 = 512 + 32;   // pipelined d = 128 kernel: 16 softmax warps + issuer warp
 constexpr uint32_t SLAB = 128 * 128;   // bytes of one [128 rows][64 bf16] slab
-// dQ tile orientation at d = 128: transposed (lane = head-dimension index, coalesced scalar
-// reductions) or plain (lane = query, 16-byte vector reductions)
-constexpr bool kDqTransposed128 = true;
-constexpr bool kReducerWarps = true;   // d = 128 fused path: dedicated warps for the dQ reductions (tc_bwd_kernel_v4)
-
 struct BwdArgs {
     const float *nLSE2, *Ds;   // -LSE log2(e) and scale * D per row (workspace)
     float *dQ_acc;
@@ -71,7 +65,6 @@ struct BwdSmem {
     static_assert(kBytes <= 227 * 1024, "shared memory budget");
 };
 
-enum { BAR_KV = 0, BAR_QFULL = 1, BAR_QEMPTY = 3, BAR_S = 5, BAR_P = 6, BAR_DQ = 7, BAR_DQDONE = 8, BAR_DP = 9, BAR_DS = 10 };
 
 struct TileIter {
     // Enumerates the query tiles a key tile jt has to visit.
@@ -108,17 +101,9 @@ __device__ __forceinline__ void bulk_load_1d(void *dst, const void *src, uint32_
                  ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(smem_u32(bar))
                  : "memory");
 }
-__device__ __forceinline__ void named_bar_sync(int id, int count)
-{
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
-}
 __device__ __forceinline__ void red_add_f32(float *p, float v)
 {
     asm volatile("red.global.add.f32 [%0], %1;" ::"l"(p), "f"(v) : "memory");
-}
-__device__ __forceinline__ void red_add_v4(float *p, float a, float b, float c, float d)
-{
-    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
 
 __device__ __forceinline__ float ex2_approx(float x)
@@ -177,674 +162,11 @@ __global__ void __launch_bounds__(256) tc_preprocess_kernel(const __nv_bfloat16 
     }
 }
 
-// WITH_DQ = false leaves the dQ product and its reductions out (dK and dV only): the
-// deterministic path computes dQ in a kernel of its own (attn_tc_bwd_dq.cu).
-template <int HD, bool WITH_DQ>
-__global__ void __launch_bounds__(kThreads, 1)
-tc_bwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mK,
-              const __grid_constant__ CUtensorMap mV, const __grid_constant__ CUtensorMap mdO, const BwdArgs a)
-{
-    using L = BwdSmem<HD>;
-    extern __shared__ __align__(1024) uint8_t smem[];
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::oBar);
-    uint32_t *tmem_base_s = reinterpret_cast<uint32_t *>(smem + L::oMisc);
-    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(smem + L::oMisc + 4);
-    const Abort ab{abort_flag, a.status};
-
-    const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
-    // launch order: heads in groups of `a.group`, inside a group key tile major -- with a causal
-    // mask the CTAs of a group then start longest first, which evens out the tail of the grid
-    const int jt = blockIdx.x / a.group;
-    const long bh = (long)blockIdx.y * a.group + blockIdx.x % a.group;
-    const int j0 = jt * TK, n = a.n;
-
-    if ((smem_u32(smem) & 1023u) != 0) {   // operand tiles need 1024-byte alignment
-        if (tid == 0) atomicExch(a.status, 9u);
-        return;
-    }
-    if (tid == 0) {
-        *abort_flag = 0;
-        mbar_init(&bars[BAR_KV], 1);
-        mbar_init(&bars[BAR_QFULL], 1); mbar_init(&bars[BAR_QFULL + 1], 1);
-        mbar_init(&bars[BAR_QEMPTY], 1); mbar_init(&bars[BAR_QEMPTY + 1], 1);
-        mbar_init(&bars[BAR_S], 1);
-        mbar_init(&bars[BAR_DP], 1);
-        mbar_init(&bars[BAR_P], kSoftmaxThreads);
-        mbar_init(&bars[BAR_DS], kSoftmaxThreads);
-        mbar_init(&bars[BAR_DQ], 1);
-        mbar_init(&bars[BAR_DQDONE], kSoftmaxThreads);
-        fence_barrier_init();
-        prefetch_tensormap(&mQ); prefetch_tensormap(&mK); prefetch_tensormap(&mV); prefetch_tensormap(&mdO);
-    }
-    if (warp == 0) tmem_alloc(tmem_base_s, 512);
-    tcgen05_fence_before();
-    __syncthreads();
-    tcgen05_fence_after();
-    const uint32_t tm = *tmem_base_s;
-    const uint32_t T_S = tm, T_dP = tm + 128, T_dV = tm + 256, T_dK = tm + 256 + HD;
-
-    const TileIter iter(a, jt, bh);
-    constexpr bool kDqT = HD == 128 && kDqTransposed128;
-
-    if (warp == 8) {
-        // ------------------------------------------------------------ producer + MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc_s = idesc_bf16(128, 128, 0, 0);       // S^T, dP^T
-            constexpr uint32_t idesc_dv = idesc_bf16(128, HD, 0, 1);       // dV (A tmem), dK (A K-major smem)
-            constexpr uint32_t idesc_dq = kDqT ? idesc_bf16(128, 128, 1, 1) : idesc_bf16(128, HD, 1, 1);
-            const uint32_t sK = smem_u32(smem + L::oK), sV = smem_u32(smem + L::oV), sdS = smem_u32(smem + L::odS);
-            auto issue_load = [&](int it, int s) {
-                const int i0 = it * TQ;
-                const uint32_t rows = min(TQ, n - i0);
-                uint64_t *bar = &bars[BAR_QFULL + s];
-                mbar_expect_tx(bar, 2 * L::kTile + 2 * rows * 4);
-#pragma unroll
-                for (uint32_t sl = 0; sl < L::kSlabs; ++sl) {
-                    tma_load_3d(smem + L::oQ + s * L::kTile + sl * SLAB, &mQ, bar, sl * 64, i0, (int)bh);
-                    tma_load_3d(smem + L::odO + s * L::kTile + sl * SLAB, &mdO, bar, sl * 64, i0, (int)bh);
-                }
-                bulk_load_1d(smem + L::oLSE + s * 512, a.nLSE2 + bh * n + i0, rows * 4, bar);
-                bulk_load_1d(smem + L::oD + s * 512, a.Ds + bh * n + i0, rows * 4, bar);
-            };
-            // S^T = K_j Q_i^T for the tile in stage s
-            auto issue_S = [&](int s) {
-                const uint32_t sQ = smem_u32(smem + L::oQ + s * L::kTile);
-#pragma unroll
-                for (int kk = 0; kk < HD / 16; ++kk) {
-                    const uint32_t off = (kk / 4) * SLAB + (kk % 4) * 32;
-                    mma_ss(T_S, smem_desc_kmajor(sK + off), smem_desc_kmajor(sQ + off), idesc_s, kk > 0);
-                }
-                mma_commit(&bars[BAR_S]);
-            };
-            mbar_expect_tx(&bars[BAR_KV], 2 * L::kTile);
-#pragma unroll
-            for (uint32_t sl = 0; sl < L::kSlabs; ++sl) {
-                tma_load_3d(smem + L::oK + sl * SLAB, &mK, &bars[BAR_KV], sl * 64, j0, (int)bh);
-                tma_load_3d(smem + L::oV + sl * SLAB, &mV, &bars[BAR_KV], sl * 64, j0, (int)bh);
-            }
-            // first valid tile
-            int idx = 0, it = -1;
-            while (idx < iter.raw && (it = iter.tile(idx)) < 0) ++idx;
-            if (it >= 0) {
-                issue_load(it, 0);
-                mbar_wait(&bars[BAR_QFULL], 0, ab);
-                mbar_wait(&bars[BAR_KV], 0, ab);
-                tcgen05_fence_after();
-                issue_S(0);
-            }
-            int k = 0;   // count of processed tiles
-            while (idx < iter.raw) {
-                const int s = k & 1;
-                // look ahead for the next valid tile and prefetch it
-                int nidx = idx + 1, nit = -1;
-                while (nidx < iter.raw && (nit = iter.tile(nidx)) < 0) ++nidx;
-                if (nit >= 0) {
-                    if (k >= 1) mbar_wait(&bars[BAR_QEMPTY + (s ^ 1)], ((k - 1) >> 1) & 1, ab);
-                    issue_load(nit, s ^ 1);
-                }
-                const uint32_t sQ = smem_u32(smem + L::oQ + s * L::kTile), sdO = smem_u32(smem + L::odO + s * L::kTile);
-                if (WITH_DQ && k > 0) {   // the dQ tile of the previous pair has been read out of T_dP
-                    mbar_wait(&bars[BAR_DQDONE], (k - 1) & 1, ab);
-                    tcgen05_fence_after();
-                }
-                // dP^T = V_j dO_i^T
-#pragma unroll
-                for (int kk = 0; kk < HD / 16; ++kk) {
-                    const uint32_t off = (kk / 4) * SLAB + (kk % 4) * 32;
-                    mma_ss(T_dP, smem_desc_kmajor(sV + off), smem_desc_kmajor(sdO + off), idesc_s, kk > 0);
-                }
-                mma_commit(&bars[BAR_DP]);
-                // dV += P^T dO_i as soon as P^T is in tensor memory
-                mbar_wait(&bars[BAR_P], k & 1, ab);
-                tcgen05_fence_after();
-#pragma unroll
-                for (int kk = 0; kk < TQ / 16; ++kk)
-                    mma_ts(T_dV, T_S + kk * 8, smem_desc_mnmajor(sdO + kk * 2048, SLAB), idesc_dv, (k > 0) || (kk > 0));
-                // dK += dS^T Q_i and the dQ tile once dS^T is in shared memory
-                mbar_wait(&bars[BAR_DS], k & 1, ab);
-                tcgen05_fence_after();
-#pragma unroll
-                for (int kk = 0; kk < TQ / 16; ++kk) {
-                    const uint32_t offa = (kk / 4) * SLAB + (kk % 4) * 32;
-                    mma_ss(T_dK, smem_desc_kmajor(sdS + offa), smem_desc_mnmajor(sQ + kk * 2048, SLAB), idesc_dv,
-                           (k > 0) || (kk > 0));
-                }
-#pragma unroll
-                for (int kk = 0; WITH_DQ && kk < TK / 16; ++kk) {
-                    if (kDqT)        // dQ^T = K_j^T dS^T : A = K_j MN-major, B = dS^T MN-major
-                        mma_ss(T_dP, smem_desc_mnmajor(sK + kk * 2048, SLAB), smem_desc_mnmajor(sdS + kk * 2048, SLAB),
-                               idesc_dq, kk > 0);
-                    else             // dQ = dS K_j : A = dS^T read MN-major, B = K_j MN-major
-                        mma_ss(T_dP, smem_desc_mnmajor(sdS + kk * 2048, SLAB), smem_desc_mnmajor(sK + kk * 2048, SLAB),
-                               idesc_dq, kk > 0);
-                }
-                mma_commit(&bars[BAR_DQ]);
-                mma_commit(&bars[BAR_QEMPTY + s]);
-                // S^T of the next pair runs while the dQ tile is being read out
-                if (nit >= 0) {
-                    mbar_wait(&bars[BAR_QFULL + (s ^ 1)], ((k + 1) >> 1) & 1, ab);
-                    tcgen05_fence_after();
-                    issue_S(s ^ 1);
-                }
-                ++k;
-                idx = nidx;
-            }
-        }
-    } else {
-        // ------------------------------------------------------------ softmax / dS / dQ reduction warpgroups
-        const int wg = warp / 4;                       // which half of the query columns
-        const int row = (warp % 4) * 32 + lane;        // tensor-memory lane = key row inside the tile
-        const uint32_t lane_addr = (uint32_t)((warp % 4) * 32) << 16;
-        const int jg = j0 + row;
-        const float sl2 = a.scale * 1.4426950408889634f;
-        int k = 0;
-        for (int idx = 0; idx < iter.raw; ++idx) {
-            const int it = iter.tile(idx);
-            if (it < 0) continue;
-            const int s = k & 1, i0 = it * TQ;
-            const float4 *sNL = reinterpret_cast<const float4 *>(smem + L::oLSE + s * 512 + wg * 256);
-            const float4 *sDs = reinterpret_cast<const float4 *>(smem + L::oD + s * 512 + wg * 256);
-            const bool diag = a.mask_kind == ATTN_MASK_CAUSAL && it == jt;
-            const bool masked = diag || i0 + TQ > n || j0 + TK > n;   // uniform over the CTA
-            const int ig0 = i0 + wg * 64;                             // first query column of this thread
-            mbar_wait(&bars[BAR_QFULL + s], (k >> 1) & 1, ab);        // -LSE_i log2e and scale * D_i visible
-            mbar_wait(&bars[BAR_S], k & 1, ab);
-            tcgen05_fence_after();
-            // ---- P^T = exp2(S^T scale log2e - LSE log2e)
-            float p[64];
-            {
-                uint32_t sv0[32], sv1[32];
-                tmem_ld32(T_S + lane_addr + wg * 64, sv0);
-                tmem_ld32(T_S + lane_addr + wg * 64 + 32, sv1);
-                tmem_wait_ld();
-#pragma unroll
-                for (int q = 0; q < 16; ++q) {
-                    const float4 nl = sNL[q];
-                    const uint32_t *sv = q < 8 ? &sv0[q * 4] : &sv1[(q - 8) * 4];
-                    p[q * 4 + 0] = ex2_approx(fmaf(__uint_as_float(sv[0]), sl2, nl.x));
-                    p[q * 4 + 1] = ex2_approx(fmaf(__uint_as_float(sv[1]), sl2, nl.y));
-                    p[q * 4 + 2] = ex2_approx(fmaf(__uint_as_float(sv[2]), sl2, nl.z));
-                    p[q * 4 + 3] = ex2_approx(fmaf(__uint_as_float(sv[3]), sl2, nl.w));
-                }
-            }
-            if (masked) {
-#pragma unroll
-                for (int e = 0; e < 64; ++e) {
-                    const int ig = ig0 + e;
-                    const bool ok = ig < n && jg < n && (!diag || jg <= ig);
-                    p[e] = ok ? p[e] : 0.f;
-                }
-            }
-            uint32_t ppack[32];
-#pragma unroll
-            for (int e = 0; e < 32; ++e) ppack[e] = pack_bf16(p[2 * e], p[2 * e + 1]);
-            // every thread has finished reading S^T before anyone overwrites it with P^T
-            named_bar_sync(1, kSoftmaxThreads);
-            tmem_st32(T_S + lane_addr + wg * 32, ppack);
-            tmem_wait_st();
-            tcgen05_fence_before();
-            mbar_arrive(&bars[BAR_P]);
-
-            // ---- dS^T = P^T o (scale dP^T - scale D): written once to shared memory
-            mbar_wait(&bars[BAR_DP], k & 1, ab);
-            tcgen05_fence_after();
-            {
-                uint32_t dv0[32], dv1[32];
-                tmem_ld32(T_dP + lane_addr + wg * 64, dv0);
-                tmem_ld32(T_dP + lane_addr + wg * 64 + 32, dv1);
-                tmem_wait_ld();
-                uint8_t *slab = smem + L::odS + wg * SLAB;
-#pragma unroll
-                for (int q8 = 0; q8 < 8; ++q8) {    // 8 query columns = one 16-byte chunk
-                    float ds[8];
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const int q = q8 * 2 + h;
-                        const float4 dsc = sDs[q];
-                        const uint32_t *dv = q < 8 ? &dv0[q * 4] : &dv1[(q - 8) * 4];
-                        ds[h * 4 + 0] = p[q * 4 + 0] * fmaf(__uint_as_float(dv[0]), a.scale, -dsc.x);
-                        ds[h * 4 + 1] = p[q * 4 + 1] * fmaf(__uint_as_float(dv[1]), a.scale, -dsc.y);
-                        ds[h * 4 + 2] = p[q * 4 + 2] * fmaf(__uint_as_float(dv[2]), a.scale, -dsc.z);
-                        ds[h * 4 + 3] = p[q * 4 + 3] * fmaf(__uint_as_float(dv[3]), a.scale, -dsc.w);
-                    }
-                    if (masked) {   // stale tail entries of the row vectors may be anything: select, do not multiply
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) ds[e] = p[q8 * 8 + e] != 0.f ? ds[e] : 0.f;
-                    }
-                    *reinterpret_cast<uint4 *>(slab + sw128_offset(row, q8 * 8)) =
-                        make_uint4(pack_bf16(ds[0], ds[1]), pack_bf16(ds[2], ds[3]), pack_bf16(ds[4], ds[5]),
-                                   pack_bf16(ds[6], ds[7]));
-                }
-            }
-            fence_proxy_async_smem();
-            tcgen05_fence_before();
-            mbar_arrive(&bars[BAR_DS]);
-
-            // ---- dQ tile: read out of tensor memory and reduce into the fp32 accumulator
-            if (WITH_DQ) {
-            mbar_wait(&bars[BAR_DQ], k & 1, ab);
-            tcgen05_fence_after();
-            if (kDqT) {
-                // lanes = head-dimension index c, columns = queries: a warp adds 128 contiguous bytes
-                float *base = a.dQ_acc + ((size_t)bh * n + ig0) * HD + row;
-                uint32_t v0[32], v1[32];
-                tmem_ld32(T_dP + lane_addr + wg * 64, v0);
-                tmem_ld32(T_dP + lane_addr + wg * 64 + 32, v1);
-                tmem_wait_ld();
-                tcgen05_fence_before();
-                mbar_arrive(&bars[BAR_DQDONE]);   // T_dP is free again; the reductions proceed from registers
-                if (!masked || i0 + TQ <= n) {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) red_add_f32(base + (size_t)e * HD, __uint_as_float(v0[e]));
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) red_add_f32(base + (size_t)(32 + e) * HD, __uint_as_float(v1[e]));
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e)
-                        if (ig0 + e < n) red_add_f32(base + (size_t)e * HD, __uint_as_float(v0[e]));
-#pragma unroll
-                    for (int e = 0; e < 32; ++e)
-                        if (ig0 + 32 + e < n) red_add_f32(base + (size_t)(32 + e) * HD, __uint_as_float(v1[e]));
-                }
-            } else {
-                // lanes = queries, columns = head-dimension index: 16-byte vector reductions
-                constexpr int HALF = HD / 2;
-                uint32_t v[HALF];
-#pragma unroll
-                for (int c = 0; c < HALF; c += 32)
-                    tmem_ld32(T_dP + lane_addr + wg * HALF + c, *reinterpret_cast<uint32_t(*)[32]>(&v[c]));
-                tmem_wait_ld();
-                tcgen05_fence_before();
-                mbar_arrive(&bars[BAR_DQDONE]);
-                if (i0 + row < n) {
-                    float *base = a.dQ_acc + ((size_t)bh * n + i0 + row) * HD + wg * HALF;
-#pragma unroll
-                    for (int e = 0; e < HALF; e += 4)
-                        red_add_v4(base + e, __uint_as_float(v[e]), __uint_as_float(v[e + 1]), __uint_as_float(v[e + 2]),
-                                   __uint_as_float(v[e + 3]));
-                }
-            }
-            }
-            ++k;
-        }
-        // ------------------------------------------------------------ epilogue: dV_j, dK_j
-        // (the last BAR_DQ phase also covers the last dV / dK accumulation; dS carried the scale)
-        if (!WITH_DQ && k > 0) {
-            mbar_wait(&bars[BAR_DQ], (k - 1) & 1, ab);
-            tcgen05_fence_after();
-        }
-        {
-            constexpr int HALF = HD / 2;
-            const int jc = jg < n ? jg : 0;   // rows past n take part in the warp-wide loads but store nothing
-            __nv_bfloat16 *pv = a.dV + ((size_t)bh * n + jc) * HD + wg * HALF;
-            __nv_bfloat16 *pk = a.dK + ((size_t)bh * n + jc) * HD + wg * HALF;
-#pragma unroll
-            for (int c = 0; c < HALF; c += 32) {
-                uint32_t v[32], w[32];
-                if (k > 0) {
-                    tmem_ld32(T_dV + lane_addr + wg * HALF + c, v);
-                    tmem_ld32(T_dK + lane_addr + wg * HALF + c, w);
-                    tmem_wait_ld();
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) v[e] = w[e] = 0u;
-                }
-                if (jg < n) {
-#pragma unroll
-                    for (int e = 0; e < 32; e += 8) {
-                        uint4 ov, ok;
-                        ov.x = pack_bf16(__uint_as_float(v[e]), __uint_as_float(v[e + 1]));
-                        ov.y = pack_bf16(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
-                        ov.z = pack_bf16(__uint_as_float(v[e + 4]), __uint_as_float(v[e + 5]));
-                        ov.w = pack_bf16(__uint_as_float(v[e + 6]), __uint_as_float(v[e + 7]));
-                        ok.x = pack_bf16(__uint_as_float(w[e]), __uint_as_float(w[e + 1]));
-                        ok.y = pack_bf16(__uint_as_float(w[e + 2]), __uint_as_float(w[e + 3]));
-                        ok.z = pack_bf16(__uint_as_float(w[e + 4]), __uint_as_float(w[e + 5]));
-                        ok.w = pack_bf16(__uint_as_float(w[e + 6]), __uint_as_float(w[e + 7]));
-                        *reinterpret_cast<uint4 *>(pv + c + e) = ov;
-                        *reinterpret_cast<uint4 *>(pk + c + e) = ok;
-                    }
-                }
-            }
-        }
-    }
-    tcgen05_fence_before();
-    __syncthreads();
-    if (warp == 0) tmem_dealloc(tm, 512);
-}
-
-// ---------------------------------------------------------------------------------------
-// d = 128, pipelined variant.  Same tiles, same shared-memory and tensor-memory layout as
-// tc_bwd_kernel, but every 128-query tile is handled as two independent halves of 64
-// queries (every barrier exists once per half) and sixteen warps share the exp / dS /
-// reduction work: warpgroups 2h and 2h+1 own the two 32-query quarters of half h, so
-// each scheduler has four warps to hide tensor-memory and MUFU latency.  The MMA issuer interleaves the two halves and issues
-// S^T of the next tile as soon as a half's dQ product is queued, so the tensor pipe keeps
-// running while the other half is in its exp / dS / reduction phase.
+// barrier indices of the fused kernel: every barrier exists once per 64-query half of a tile
 enum { V2_KV = 0, V2_QFULL = 1, V2_QEMPTY = 3, V2_S = 5, V2_DP = 7, V2_P = 9, V2_DS = 11, V2_DQ = 13, V2_DQDONE = 15 };
 
-template <bool WITH_DQ>
-__global__ void __launch_bounds__(kThreadsV2, 1)
-tc_bwd_kernel_v2(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mK_,
-                 const __grid_constant__ CUtensorMap mV, const __grid_constant__ CUtensorMap mdO, const BwdArgs a)
-{
-    constexpr int HD = 128;
-    constexpr int kHalfThreads = 256;
-    using L = BwdSmem<HD>;
-    static_assert(L::oMisc - L::oBar >= 17 * 8, "barrier area");
-    extern __shared__ __align__(1024) uint8_t smem[];
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::oBar);
-    uint32_t *tmem_base_s = reinterpret_cast<uint32_t *>(smem + L::oMisc);
-    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(smem + L::oMisc + 4);
-    const Abort ab{abort_flag, a.status};
-
-    const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
-    // launch order: heads in groups of `a.group`, inside a group key tile major -- with a causal
-    // mask the CTAs of a group then start longest first, which evens out the tail of the grid
-    const int jt = blockIdx.x / a.group;
-    const long bh = (long)blockIdx.y * a.group + blockIdx.x % a.group;
-    const int j0 = jt * TK, n = a.n;
-
-    if ((smem_u32(smem) & 1023u) != 0) {
-        if (tid == 0) atomicExch(a.status, 9u);
-        return;
-    }
-    if (tid == 0) {
-        *abort_flag = 0;
-        mbar_init(&bars[V2_KV], 1);
-        for (int h = 0; h < 2; ++h) {
-            mbar_init(&bars[V2_QFULL + h], 1);
-            mbar_init(&bars[V2_QEMPTY + h], 1);
-            mbar_init(&bars[V2_S + h], 1);
-            mbar_init(&bars[V2_DP + h], 1);
-            mbar_init(&bars[V2_P + h], kHalfThreads);
-            mbar_init(&bars[V2_DS + h], kHalfThreads);
-            mbar_init(&bars[V2_DQ + h], 1);
-            mbar_init(&bars[V2_DQDONE + h], kHalfThreads);
-        }
-        fence_barrier_init();
-        prefetch_tensormap(&mQ); prefetch_tensormap(&mK_); prefetch_tensormap(&mV); prefetch_tensormap(&mdO);
-    }
-    if (warp == 0) tmem_alloc(tmem_base_s, 512);
-    tcgen05_fence_before();
-    __syncthreads();
-    tcgen05_fence_after();
-    const uint32_t tm = *tmem_base_s;
-    const uint32_t T_S = tm, T_dP = tm + 128, T_dV = tm + 256, T_dK = tm + 256 + HD;
-    constexpr uint32_t HALF_ROWS = 64 * 128;   // byte offset of rows 64.. inside a [128][64] slab
-
-    const TileIter iter(a, jt, bh);
-
-    if (warp == 16) {
-        if (lane == 0) {
-            constexpr uint32_t idesc_s = idesc_bf16(128, 128, 0, 0);       // S^T, dP^T (both halves at once)
-            constexpr uint32_t idesc_dv = idesc_bf16(128, HD, 0, 1);       // dV (A tmem), dK (A K-major smem)
-            constexpr uint32_t idesc_dq = idesc_bf16(128, 64, 1, 1);       // dQ^T half
-            // low descriptor words (tc_common.cuh): per-step offsets are added as (bytes >> 4)
-            const uint32_t kK = desc_lo_kmajor(smem_u32(smem + L::oK)), kV = desc_lo_kmajor(smem_u32(smem + L::oV));
-            const uint32_t mK = desc_lo_mnmajor(smem_u32(smem + L::oK), SLAB);
-            const uint32_t kdS = desc_lo_kmajor(smem_u32(smem + L::odS)), mdS = desc_lo_mnmajor(smem_u32(smem + L::odS), SLAB);
-            constexpr uint32_t kHalf = HALF_ROWS >> 4, kSlab = SLAB >> 4;
-            auto issue_load = [&](int it, int s) {
-                const int i0 = it * TQ;
-                const uint32_t rows = min(TQ, n - i0);
-                uint64_t *bar = &bars[V2_QFULL + s];
-                mbar_expect_tx(bar, 2 * L::kTile + 2 * rows * 4);
-#pragma unroll
-                for (uint32_t sl = 0; sl < L::kSlabs; ++sl) {
-                    tma_load_3d(smem + L::oQ + s * L::kTile + sl * SLAB, &mQ, bar, sl * 64, i0, (int)bh);
-                    tma_load_3d(smem + L::odO + s * L::kTile + sl * SLAB, &mdO, bar, sl * 64, i0, (int)bh);
-                }
-                bulk_load_1d(smem + L::oLSE + s * 512, a.nLSE2 + bh * n + i0, rows * 4, bar);
-                bulk_load_1d(smem + L::oD + s * 512, a.Ds + bh * n + i0, rows * 4, bar);
-            };
-            // S^T = K_j Q_i^T for the whole tile in stage s; one commit per half's barrier
-            auto issue_S = [&](int s) {
-                const uint32_t kQ = desc_lo_kmajor(smem_u32(smem + L::oQ + s * L::kTile));
-#pragma unroll
-                for (int kk = 0; kk < HD / 16; ++kk) {
-                    const uint32_t off = (kk / 4) * kSlab + (kk % 4) * 2;
-                    mma_ss_lo(T_S, kK + off, kQ + off, idesc_s, kk > 0);
-                }
-                mma_commit(&bars[V2_S]);
-                mma_commit(&bars[V2_S + 1]);
-            };
-            mbar_expect_tx(&bars[V2_KV], 2 * L::kTile);
-#pragma unroll
-            for (uint32_t sl = 0; sl < L::kSlabs; ++sl) {
-                tma_load_3d(smem + L::oK + sl * SLAB, &mK_, &bars[V2_KV], sl * 64, j0, (int)bh);
-                tma_load_3d(smem + L::oV + sl * SLAB, &mV, &bars[V2_KV], sl * 64, j0, (int)bh);
-            }
-            int idx = 0, it = -1;
-            while (idx < iter.raw && (it = iter.tile(idx)) < 0) ++idx;
-            if (it >= 0) {
-                issue_load(it, 0);
-                mbar_wait(&bars[V2_QFULL], 0, ab);
-                mbar_wait(&bars[V2_KV], 0, ab);
-                tcgen05_fence_after();
-                issue_S(0);
-            }
-            int k = 0;
-            while (idx < iter.raw) {
-                const int s = k & 1;
-                int nidx = idx + 1, nit = -1;
-                while (nidx < iter.raw && (nit = iter.tile(nidx)) < 0) ++nidx;
-                if (nit >= 0) {
-                    if (k >= 1) mbar_wait(&bars[V2_QEMPTY + (s ^ 1)], ((k - 1) >> 1) & 1, ab);
-                    issue_load(nit, s ^ 1);
-                }
-                const uint32_t sQa = smem_u32(smem + L::oQ + s * L::kTile), sdOa = smem_u32(smem + L::odO + s * L::kTile);
-                const uint32_t kdO = desc_lo_kmajor(sdOa), mdO_ = desc_lo_mnmajor(sdOa, SLAB), mQ_ = desc_lo_mnmajor(sQa, SLAB);
-                // dP^T = V_j dO_i^T once both halves of the previous dQ^T have left T_dP
-                if (WITH_DQ && k > 0) {
-                    mbar_wait(&bars[V2_DQDONE], (k - 1) & 1, ab);
-                    mbar_wait(&bars[V2_DQDONE + 1], (k - 1) & 1, ab);
-                    tcgen05_fence_after();
-                }
-#pragma unroll
-                for (int kk = 0; kk < HD / 16; ++kk) {
-                    const uint32_t off = (kk / 4) * kSlab + (kk % 4) * 2;
-                    mma_ss_lo(T_dP, kV + off, kdO + off, idesc_s, kk > 0);
-                }
-                mma_commit(&bars[V2_DP]);
-                mma_commit(&bars[V2_DP + 1]);
-                // dV += P_h^T dO_h
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    mbar_wait(&bars[V2_P + h], k & 1, ab);
-                    tcgen05_fence_after();
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)
-                        mma_ts_lo(T_dV, T_S + 64 * h + (kk < 2 ? kk * 8 : 48 + (kk - 2) * 8), mdO_ + h * kHalf + kk * 128,
-                                  idesc_dv, (k > 0) || (h > 0) || (kk > 0));
-                }
-                // T_S is free again: S^T of the next tile runs while this tile's dS is being formed
-                if (nit >= 0) {
-                    mbar_wait(&bars[V2_QFULL + (s ^ 1)], ((k + 1) >> 1) & 1, ab);
-                    tcgen05_fence_after();
-                    issue_S(s ^ 1);
-                }
-                // dK += dS_h^T Q_h ; dQ_h^T = K_j^T dS_h^T
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    mbar_wait(&bars[V2_DS + h], k & 1, ab);
-                    tcgen05_fence_after();
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)
-                        mma_ss_lo(T_dK, kdS + h * kSlab + kk * 2, mQ_ + h * kHalf + kk * 128, idesc_dv,
-                                  (k > 0) || (h > 0) || (kk > 0));
-#pragma unroll
-                    for (int kk = 0; WITH_DQ && kk < TK / 16; ++kk)
-                        mma_ss_lo(T_dP + 64 * h, mK + kk * 128, mdS + h * kSlab + kk * 128, idesc_dq, kk > 0);
-                    mma_commit(&bars[V2_DQ + h]);
-                }
-                mma_commit(&bars[V2_QEMPTY + s]);
-                ++k;
-                idx = nidx;
-            }
-        }
-    } else {
-        // ------------------------------------------------------------ warpgroup 2h + qq owns queries 64 h + 32 qq .. + 31
-        const int h = warp / 8, qq = (warp / 4) & 1;
-        const int row = (warp % 4) * 32 + lane;        // tensor-memory lane = key row inside the tile
-        const uint32_t lane_addr = (uint32_t)((warp % 4) * 32) << 16;
-        const int jg = j0 + row;
-        const float sl2 = a.scale * 1.4426950408889634f;
-        int k = 0;
-        for (int idx = 0; idx < iter.raw; ++idx) {
-            const int it = iter.tile(idx);
-            if (it < 0) continue;
-            const int s = k & 1, i0 = it * TQ;
-            const float4 *sNL = reinterpret_cast<const float4 *>(smem + L::oLSE + s * 512 + h * 256 + qq * 128);
-            const float4 *sDs = reinterpret_cast<const float4 *>(smem + L::oD + s * 512 + h * 256 + qq * 128);
-            const bool diag = a.mask_kind == ATTN_MASK_CAUSAL && it == jt;
-            const bool masked = diag || i0 + TQ > n || j0 + TK > n;
-            const int ig0 = i0 + h * 64 + qq * 32;
-            const uint32_t c0 = h * 64 + qq * 32;      // this thread's first column in T_S / T_dP
-            mbar_wait(&bars[V2_QFULL + s], (k >> 1) & 1, ab);
-            mbar_wait(&bars[V2_S + h], k & 1, ab);
-            tcgen05_fence_after();
-            float p[32];
-            {
-                uint32_t sv0[32];
-                tmem_ld32(T_S + lane_addr + c0, sv0);
-                tmem_wait_ld();
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const float4 nl = sNL[q];
-                    const uint32_t *sv = &sv0[q * 4];
-                    p[q * 4 + 0] = ex2_approx(fmaf(__uint_as_float(sv[0]), sl2, nl.x));
-                    p[q * 4 + 1] = ex2_approx(fmaf(__uint_as_float(sv[1]), sl2, nl.y));
-                    p[q * 4 + 2] = ex2_approx(fmaf(__uint_as_float(sv[2]), sl2, nl.z));
-                    p[q * 4 + 3] = ex2_approx(fmaf(__uint_as_float(sv[3]), sl2, nl.w));
-                }
-            }
-            if (masked) {
-#pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    const int ig = ig0 + e;
-                    const bool ok = ig < n && jg < n && (!diag || jg <= ig);
-                    p[e] = ok ? p[e] : 0.f;
-                }
-            }
-            {
-                // P^T (bf16 pairs) goes over columns this very thread has just read -- quarter 0
-                // to columns 0..15 of the half, quarter 1 to columns 48..63 -- so no thread
-                // overwrites S^T entries another thread still has to read
-                uint32_t ppack[16];
-#pragma unroll
-                for (int e = 0; e < 16; ++e) ppack[e] = pack_bf16(p[2 * e], p[2 * e + 1]);
-                tmem_st16(T_S + lane_addr + h * 64 + qq * 48, ppack);
-                tmem_wait_st();
-            }
-            tcgen05_fence_before();
-            mbar_arrive(&bars[V2_P + h]);
-
-            mbar_wait(&bars[V2_DP + h], k & 1, ab);
-            tcgen05_fence_after();
-            {
-                uint32_t dv0[32];
-                tmem_ld32(T_dP + lane_addr + c0, dv0);
-                tmem_wait_ld();
-                uint8_t *slab = smem + L::odS + h * SLAB;
-#pragma unroll
-                for (int q8 = 0; q8 < 4; ++q8) {
-                    float ds[8];
-#pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        const int q = q8 * 2 + u;
-                        const float4 dsc = sDs[q];
-                        const uint32_t *dv = &dv0[q * 4];
-                        ds[u * 4 + 0] = p[q * 4 + 0] * fmaf(__uint_as_float(dv[0]), a.scale, -dsc.x);
-                        ds[u * 4 + 1] = p[q * 4 + 1] * fmaf(__uint_as_float(dv[1]), a.scale, -dsc.y);
-                        ds[u * 4 + 2] = p[q * 4 + 2] * fmaf(__uint_as_float(dv[2]), a.scale, -dsc.z);
-                        ds[u * 4 + 3] = p[q * 4 + 3] * fmaf(__uint_as_float(dv[3]), a.scale, -dsc.w);
-                    }
-                    if (masked) {
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) ds[e] = p[q8 * 8 + e] != 0.f ? ds[e] : 0.f;
-                    }
-                    *reinterpret_cast<uint4 *>(slab + sw128_offset(row, qq * 32 + q8 * 8)) =
-                        make_uint4(pack_bf16(ds[0], ds[1]), pack_bf16(ds[2], ds[3]), pack_bf16(ds[4], ds[5]),
-                                   pack_bf16(ds[6], ds[7]));
-                }
-            }
-            fence_proxy_async_smem();
-            tcgen05_fence_before();
-            mbar_arrive(&bars[V2_DS + h]);
-
-            if (WITH_DQ) {
-            mbar_wait(&bars[V2_DQ + h], k & 1, ab);
-            tcgen05_fence_after();
-            {
-                float *base = a.dQ_acc + ((size_t)bh * n + ig0) * HD + row;
-                uint32_t v0[32];
-                tmem_ld32(T_dP + lane_addr + c0, v0);
-                tmem_wait_ld();
-                tcgen05_fence_before();
-                mbar_arrive(&bars[V2_DQDONE + h]);
-                if (!masked || i0 + TQ <= n) {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) red_add_f32(base + (size_t)e * HD, __uint_as_float(v0[e]));
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e)
-                        if (ig0 + e < n) red_add_f32(base + (size_t)e * HD, __uint_as_float(v0[e]));
-                }
-            }
-            }
-            ++k;
-        }
-        // ------------------------------------------------------------ epilogue: dV_j, dK_j (32 columns per warpgroup)
-        if (k > 0) {
-            // both halves' last products must have landed, not only this warpgroup's own
-            mbar_wait(&bars[V2_DQ + h], (k - 1) & 1, ab);
-            mbar_wait(&bars[V2_DQ + (h ^ 1)], (k - 1) & 1, ab);
-            tcgen05_fence_after();
-        }
-        {
-            constexpr int HALF = 32;
-            const int cq = (warp / 4) * 32;
-            const int jc = jg < n ? jg : 0;
-            __nv_bfloat16 *pv = a.dV + ((size_t)bh * n + jc) * HD + cq;
-            __nv_bfloat16 *pk = a.dK + ((size_t)bh * n + jc) * HD + cq;
-#pragma unroll
-            for (int c = 0; c < HALF; c += 32) {
-                uint32_t v[32], w[32];
-                if (k > 0) {
-                    tmem_ld32(T_dV + lane_addr + cq + c, v);
-                    tmem_ld32(T_dK + lane_addr + cq + c, w);
-                    tmem_wait_ld();
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) v[e] = w[e] = 0u;
-                }
-                if (jg < n) {
-#pragma unroll
-                    for (int e = 0; e < 32; e += 8) {
-                        uint4 ov, ok;
-                        ov.x = pack_bf16(__uint_as_float(v[e]), __uint_as_float(v[e + 1]));
-                        ov.y = pack_bf16(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
-                        ov.z = pack_bf16(__uint_as_float(v[e + 4]), __uint_as_float(v[e + 5]));
-                        ov.w = pack_bf16(__uint_as_float(v[e + 6]), __uint_as_float(v[e + 7]));
-                        ok.x = pack_bf16(__uint_as_float(w[e]), __uint_as_float(w[e + 1]));
-                        ok.y = pack_bf16(__uint_as_float(w[e + 2]), __uint_as_float(w[e + 3]));
-                        ok.z = pack_bf16(__uint_as_float(w[e + 4]), __uint_as_float(w[e + 5]));
-                        ok.w = pack_bf16(__uint_as_float(w[e + 6]), __uint_as_float(w[e + 7]));
-                        *reinterpret_cast<uint4 *>(pv + c + e) = ov;
-                        *reinterpret_cast<uint4 *>(pk + c + e) = ok;
-                    }
-                }
-            }
-        }
-    }
-    tcgen05_fence_before();
-    __syncthreads();
-    if (warp == 0) tmem_dealloc(tm, 512);
-}
-
 // ---------------------------------------------------------------------------------------
-// d = 128, dK and dV only: the key-stationary half of the path without atomics (dQ comes from the
+// dK and dV only: the key-stationary half of the path without atomics (dQ comes from the
 // query-stationary kernel).  Without the dQ product dS^T never has to be in shared memory: it
 // is written over dP^T in tensor memory as bf16 pairs, exactly as P^T over S^T, and
 // dK += dS^T Q takes it from there.  The 32 KB this frees hold a third Q stage, and Q, dO and
@@ -852,8 +174,9 @@ tc_bwd_kernel_v2(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
 // phase), so loads run up to two tiles ahead.  Products execute on the tensor pipe in issue
 // order, so S^T of tile k+1 is queued right behind dV of tile k, and dP^T of tile k+1 behind
 // dK of tile k, with no wait in between.
-struct DkdvSmem {
-    static constexpr uint32_t kTile = 2 * SLAB;             // one [128][128] bf16 tile
+template <int HD> struct DkdvSmem {
+    static constexpr uint32_t kSlabs = HD / 64;
+    static constexpr uint32_t kTile = kSlabs * SLAB;        // one [128][HD] bf16 tile
     static constexpr uint32_t oK = 0;
     static constexpr uint32_t oV = oK + kTile;
     static constexpr uint32_t oQ = oV + kTile;              // 3 stages
@@ -869,13 +192,13 @@ enum { KD_KV = 0, KD_QFULL = 1, KD_QEMPTY = 4, KD_OFULL = 7, KD_OEMPTY = 9, KD_L
        KD_S = 15, KD_DP = 17, KD_P = 19, KD_DS = 21, KD_DONE = 23 };
 constexpr int kThreadsDkdv = 512 + 64;   // 16 exp/dS warps, MMA issuer warp, TMA producer warp
 
+template <int HD>
 __global__ void __launch_bounds__(kThreadsDkdv, 1)
 tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mK_,
                    const __grid_constant__ CUtensorMap mV, const __grid_constant__ CUtensorMap mdO, const BwdArgs a)
 {
-    constexpr int HD = 128;
     constexpr int kHalfThreads = 256;
-    using L = DkdvSmem;
+    using L = DkdvSmem<HD>;
     extern __shared__ __align__(1024) uint8_t smem[];
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::oBar);
     uint32_t *tmem_base_s = reinterpret_cast<uint32_t *>(smem + L::oMisc);
@@ -924,7 +247,7 @@ tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
         if (lane == 0) {
             mbar_expect_tx(&bars[KD_KV], 2 * L::kTile);
 #pragma unroll
-            for (uint32_t sl = 0; sl < 2; ++sl) {
+            for (uint32_t sl = 0; sl < L::kSlabs; ++sl) {
                 tma_load_3d(smem + L::oK + sl * SLAB, &mK_, &bars[KD_KV], sl * 64, j0, (int)bh);
                 tma_load_3d(smem + L::oV + sl * SLAB, &mV, &bars[KD_KV], sl * 64, j0, (int)bh);
             }
@@ -937,7 +260,7 @@ tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
                 if (k >= 3) mbar_wait(&bars[KD_QEMPTY + sq], ((k / 3) - 1) & 1, ab);
                 mbar_expect_tx(&bars[KD_QFULL + sq], L::kTile);
 #pragma unroll
-                for (uint32_t sl = 0; sl < 2; ++sl)
+                for (uint32_t sl = 0; sl < L::kSlabs; ++sl)
                     tma_load_3d(smem + L::oQ + sq * L::kTile + sl * SLAB, &mQ, &bars[KD_QFULL + sq], sl * 64, i0, (int)bh);
                 if (k >= 2) mbar_wait(&bars[KD_LEMPTY + s2], ((k >> 1) - 1) & 1, ab);
                 mbar_expect_tx(&bars[KD_LFULL + s2], 2 * rows * 4);
@@ -946,7 +269,7 @@ tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
                 if (k >= 2) mbar_wait(&bars[KD_OEMPTY + s2], ((k >> 1) - 1) & 1, ab);
                 mbar_expect_tx(&bars[KD_OFULL + s2], L::kTile);
 #pragma unroll
-                for (uint32_t sl = 0; sl < 2; ++sl)
+                for (uint32_t sl = 0; sl < L::kSlabs; ++sl)
                     tma_load_3d(smem + L::odO + s2 * L::kTile + sl * SLAB, &mdO, &bars[KD_OFULL + s2], sl * 64, i0, (int)bh);
                 ++k;
             }
@@ -1129,12 +452,12 @@ tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
             tcgen05_fence_after();
         }
         {
-            const int cq = (warp / 4) * 32;
+            const int cq = (warp / 4) * 32;       // d = 64: the upper two warpgroups have no columns
             const int jc = jg < n ? jg : 0;
             __nv_bfloat16 *pv = a.dV + ((size_t)bh * n + jc) * HD + cq;
             __nv_bfloat16 *pk = a.dK + ((size_t)bh * n + jc) * HD + cq;
             uint32_t v[32], w[32];
-            if (k > 0) {
+            if (k > 0 && cq < HD) {
                 tmem_ld32(T_dV + lane_addr + cq, v);
                 tmem_ld32(T_dK + lane_addr + cq, w);
                 tmem_wait_ld();
@@ -1142,7 +465,7 @@ tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
 #pragma unroll
                 for (int e = 0; e < 32; ++e) v[e] = w[e] = 0u;
             }
-            if (jg < n) {
+            if (jg < n && cq < HD) {
 #pragma unroll
                 for (int e = 0; e < 32; e += 8) {
                     uint4 ov, ok;
@@ -1166,11 +489,12 @@ tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
 }
 
 // ---------------------------------------------------------------------------------------
-// d = 128, pipelined variant with reducer warps.  As tc_bwd_kernel_v2<true>, plus eight warps
-// (16-23) that do nothing but move finished dQ^T tiles from tensor memory into the fp32
-// accumulator: the red.global.add queue stalls them, not the warps on the tile loop.  To fit
-// 25 warps in the register file the exp/dS warps keep P only as the bf16 pairs they hand to
-// the dV product, and form dS from those.
+// The fused kernel.  Every 128-query tile is handled as two halves of 64 queries (every barrier exists
+// once per half).  Warps 0-7: exp / dS (warpgroup h owns half h); warps 8-15: reducers, which do
+// nothing but move finished dQ^T tiles from tensor memory into the fp32 accumulator, so that the
+// red.global.add queue stalls them and not the warps on the tile loop; warp 16 lane 0 issues every
+// product, warp 17 lane 0 every TMA load.  The exp / dS warps keep P only as the bf16 pairs they
+// hand to the dV product, and form dS from those.
 constexpr int kThreadsV4 = 256 + 256 + 128;  // 8 exp/dS warps, 8 reducer warps, issuer warp, TMA producer warp, 2 idle warps
 // Registers per thread after the warpgroups have traded them (setmaxnreg): the kernel starts with 96 everywhere;
 // the issuer / producer warpgroup and the reducers give up 40 and 16 each, which the exp / dS warpgroups take:
@@ -1505,7 +829,6 @@ tc_bwd_kernel_v4(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
             tcgen05_fence_after();
         }
         {
-            constexpr int HALF = 32;
             const int cq0 = (warp / 4) * (HD / 2);
             const int jc = jg < n ? jg : 0;
 #pragma unroll
@@ -1571,9 +894,6 @@ attn_status launch_bwd(const Problem &p)
     a.scale = p.scale;
     a.status = p.status;
     a.group = p.BH % 8 == 0 ? 8 : p.BH % 4 == 0 ? 4 : p.BH % 2 == 0 ? 2 : 1;
-    auto kernel = tc_bwd_kernel<HD, WITH_DQ>;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::kBytes) != cudaSuccess)
-        return ATTN_ERR_LAUNCH;
     const size_t acc_elems = (size_t)p.BH * p.n * HD;
     if (WITH_DQ && cudaMemsetAsync(p.dQ_acc, 0, acc_elems * sizeof(float), p.stream) != cudaSuccess) return ATTN_ERR_LAUNCH;
     {
@@ -1589,21 +909,15 @@ attn_status launch_bwd(const Problem &p)
     }
     const dim3 grid((unsigned)((p.n + TK - 1) / TK * a.group), (unsigned)(p.BH / a.group));
     launch_begin(WITH_DQ ? "tc_bwd_fused" : "tc_bwd_dkdv", p.stream);
-    if (WITH_DQ && kReducerWarps) {
+    if (WITH_DQ) {
         constexpr uint32_t bytes = HD == 64 ? ((L::kBytes + 1023u) & ~1023u) + SLAB : L::kBytes;
         if (cudaFuncSetAttribute(tc_bwd_kernel_v4<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
             return ATTN_ERR_LAUNCH;
         tc_bwd_kernel_v4<HD><<<grid, kThreadsV4, bytes, p.stream>>>(mQ, mK, mV, mdO, a);
-    } else if (HD == 128 && !WITH_DQ) {
-        if (cudaFuncSetAttribute(tc_bwd_dkdv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DkdvSmem::kBytes) != cudaSuccess)
-            return ATTN_ERR_LAUNCH;
-        tc_bwd_dkdv_kernel<<<grid, kThreadsDkdv, DkdvSmem::kBytes, p.stream>>>(mQ, mK, mV, mdO, a);
-    } else if (HD == 128) {
-        if (cudaFuncSetAttribute(tc_bwd_kernel_v2<WITH_DQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::kBytes) != cudaSuccess)
-            return ATTN_ERR_LAUNCH;
-        tc_bwd_kernel_v2<WITH_DQ><<<grid, kThreadsV2, L::kBytes, p.stream>>>(mQ, mK, mV, mdO, a);
     } else {
-        kernel<<<grid, kThreads, L::kBytes, p.stream>>>(mQ, mK, mV, mdO, a);
+        if (cudaFuncSetAttribute(tc_bwd_dkdv_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DkdvSmem<HD>::kBytes) != cudaSuccess)
+            return ATTN_ERR_LAUNCH;
+        tc_bwd_dkdv_kernel<HD><<<grid, kThreadsDkdv, DkdvSmem<HD>::kBytes, p.stream>>>(mQ, mK, mV, mdO, a);
     }
     launch_end(p.stream);
     if (cudaGetLastError() != cudaSuccess) return ATTN_ERR_LAUNCH;
