@@ -22,7 +22,7 @@
 // converts it to bf16 at the end.  Tensor memory (512 columns): S^T / P^T 128,
 // dP^T then dQ^T 128, dV d, dK d.
 //
-// Two kernels: tc_bwd_kernel_v4 (all five products, the default) and tc_bwd_dkdv_kernel
+// Two kernels: tc_bwd_fused_kernel (all five products, the default) and tc_bwd_dkdv_kernel
 // (without the dQ product; `deterministic = 1` pairs it with the query-stationary dQ kernel of
 // attn_tc_bwd_dq.cu).  Warp roles are described at each kernel.  All waits are bounded
 // (tc_common.cuh).
@@ -490,27 +490,28 @@ tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
 
 // ---------------------------------------------------------------------------------------
 // The fused kernel.  Every 128-query tile is handled as two halves of 64 queries (every barrier exists
-// once per half).  Warps 0-7: exp / dS (warpgroup h owns half h); warps 8-15: reducers, which do
-// nothing but move finished dQ^T tiles from tensor memory into the fp32 accumulator, so that the
-// red.global.add queue stalls them and not the warps on the tile loop; warp 16 lane 0 issues every
-// product, warp 17 lane 0 every TMA load.  The exp / dS warps keep P only as the bf16 pairs they
-// hand to the dV product, and form dS from those.
-constexpr int kThreadsV4 = 256 + 256 + 128;  // 8 exp/dS warps, 8 reducer warps, issuer warp, TMA producer warp, 2 idle warps
-// Registers per thread after the warpgroups have traded them (setmaxnreg): the kernel starts with 96 everywhere;
-// the issuer / producer warpgroup and the reducers give up 40 and 16 each, which the exp / dS warpgroups take:
-// 256 x 128 + 256 x 80 + 128 x 56 = 60,416 of the 61,440 allocated at launch.
-constexpr int kRegsExp = 120, kRegsReduce = 80, kRegsIssue = 72;
+// once per half).  Warps 0-15: exp / dS (warpgroups 2h and 2h+1 own the two 32-query quarters of half
+// h, so each scheduler has four such warps to hide tensor-memory and MUFU latency); warps 16-23:
+// reducers, which do nothing but move finished dQ^T tiles from tensor memory into the fp32
+// accumulator, so that the red.global.add queue stalls them and not the warps on the tile loop;
+// warp 24 lane 0 issues every product, warp 25 lane 0 every TMA load; warps 26-27 only complete
+// that warpgroup.  The exp / dS warps keep P only as the bf16 pairs they hand to the dV product, and
+// form dS from those.  Registers are traded between the warpgroups after launch (setmaxnreg).
 template <int N> __device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+constexpr int kThreadsFused = 512 + 256 + 128;  // 16 exp/dS warps, 8 reducer warps, issuer warp, TMA producer warp, 2 idle warps
+// 72 registers everywhere at launch (896 x 72 = 64,512); the reducers give up 24 each, the exp / dS warps take 8:
+// 512 x 80 + 256 x 48 + 128 x 72 = 62,464.
+constexpr int kRegsExp = 80, kRegsReduce = 48;
 template <int HD>
-__global__ void __launch_bounds__(kThreadsV4, 1)
-tc_bwd_kernel_v4(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mK_,
+__global__ void __launch_bounds__(kThreadsFused, 1)
+tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mK_,
                  const __grid_constant__ CUtensorMap mV, const __grid_constant__ CUtensorMap mdO, const BwdArgs a)
 {
     constexpr bool WITH_DQ = true;
     // d = 64: the dQ^T product needs M = 128, so the K tile's second 64-wide slab of M is an all-zero slab
     constexpr uint32_t oZero = (BwdSmem<HD>::kBytes + 1023u) & ~1023u;
-    constexpr int kHalfThreads = 128;     // exp / dS threads per half
+    constexpr int kHalfThreads = 256;     // exp / dS threads per half
     constexpr int kReduceThreads = 128;   // reducer threads per half
     using L = BwdSmem<HD>;
     static_assert(L::oMisc - L::oBar >= 17 * 8, "barrier area");
@@ -548,7 +549,7 @@ tc_bwd_kernel_v4(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
         prefetch_tensormap(&mQ); prefetch_tensormap(&mK_); prefetch_tensormap(&mV); prefetch_tensormap(&mdO);
     }
     if (HD == 64) {
-        for (uint32_t i = tid; i < SLAB / 16; i += kThreadsV4) reinterpret_cast<uint4 *>(smem + oZero)[i] = make_uint4(0, 0, 0, 0);
+        for (uint32_t i = tid; i < SLAB / 16; i += kThreadsFused) reinterpret_cast<uint4 *>(smem + oZero)[i] = make_uint4(0, 0, 0, 0);
         fence_proxy_async_smem();
     }
     if (warp == 0) tmem_alloc(tmem_base_s, 512);
@@ -561,11 +562,9 @@ tc_bwd_kernel_v4(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
 
     const TileIter iter(a, jt, bh);
 
-    if (warp >= 16) {
-        setmaxnreg_dec<kRegsIssue>();   // whole warpgroup 16-19; warps 18 and 19 exist only to complete it
-    }
-    if (warp >= 18) {
-    } else if (warp == 17) {
+    if (warp >= 26) {
+        // idle: they only complete the issuer's warpgroup, which keeps its 72 registers
+    } else if (warp == 25) {
         // ------------------------------------------------------------ TMA producer: every load, as soon as its stage is free
         if (lane == 0) {
             auto issue_load = [&](int it, int s) {
@@ -597,7 +596,7 @@ tc_bwd_kernel_v4(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
                 ++k;
             }
         }
-    } else if (warp == 16) {
+    } else if (warp == 24) {
         if (lane == 0) {
             constexpr uint32_t idesc_s = idesc_bf16(128, 128, 0, 0);       // S^T, dP^T (both halves at once)
             constexpr uint32_t idesc_dv = idesc_bf16(128, HD, 0, 1);       // dV (A tmem), dK (A K-major smem)
@@ -653,7 +652,7 @@ tc_bwd_kernel_v4(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
                     tcgen05_fence_after();
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
-                        mma_ts_lo(T_dV, T_S + 64 * h + kk * 8, mdO_ + h * kHalf + kk * 128,
+                        mma_ts_lo(T_dV, T_S + 64 * h + (kk < 2 ? kk * 8 : 48 + (kk - 2) * 8), mdO_ + h * kHalf + kk * 128,
                                   idesc_dv, (k > 0) || (h > 0) || (kk > 0));
                 }
                 // T_S is free again: S^T of the next tile runs while this tile's dS is being formed
@@ -680,50 +679,51 @@ tc_bwd_kernel_v4(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
                 idx = nidx;
             }
         }
-    } else if (warp >= 8) {
+    } else if (warp >= 16) {
         setmaxnreg_dec<kRegsReduce>();
         // ------------------------------------------------------------ reducers: dQ_h^T tile -> fp32 accumulator
-        // lanes = head-dimension index c, columns = queries: one warp instruction adds 128 contiguous bytes
-        const int h = (warp - 8) / 4;
+        // lanes = head-dimension index c, columns = queries: one warp instruction adds 128 contiguous bytes.
+        // 32 columns at a time (the reducers run on 48 registers); the half is released after the second load
+        const int h = (warp - 16) / 4;
         const int row = (warp % 4) * 32 + lane;
         const uint32_t lane_addr = (uint32_t)((warp % 4) * 32) << 16;
+        const bool live = (warp % 4) * 32 < HD;   // d = 64: lanes 64..127 of the padded product hold zeros
         int k = 0;
         for (int idx = 0; idx < iter.raw; ++idx) {
             const int it = iter.tile(idx);
             if (it < 0) continue;
             const int ig0 = it * TQ + h * 64;
+            float *base = a.dQ_acc + ((size_t)bh * n + ig0) * HD + row;
             mbar_wait(&bars[V2_DQ + h], k & 1, ab);
             tcgen05_fence_after();
-            uint32_t v0[32], v1[32];
-            const bool live = (warp % 4) * 32 < HD;   // d = 64: lanes 64..127 of the padded product hold zeros
-            if (live) {
-                tmem_ld32(T_dP + lane_addr + h * 64, v0);
-                tmem_ld32(T_dP + lane_addr + h * 64 + 32, v1);
-                tmem_wait_ld();
-            }
-            tcgen05_fence_before();
-            mbar_arrive(&bars[V2_DQDONE + h]);   // T_dP half h is free again; the reductions proceed from registers
-            float *base = a.dQ_acc + ((size_t)bh * n + ig0) * HD + row;
-            if (!live) {
-            } else if (ig0 + 64 <= n) {
 #pragma unroll
-                for (int e = 0; e < 32; ++e) red_add_f32(base + (size_t)e * HD, __uint_as_float(v0[e]));
+            for (int part = 0; part < 2; ++part) {
+                uint32_t v0[32];
+                if (live) {
+                    tmem_ld32(T_dP + lane_addr + h * 64 + part * 32, v0);
+                    tmem_wait_ld();
+                }
+                if (part == 1) {
+                    tcgen05_fence_before();
+                    mbar_arrive(&bars[V2_DQDONE + h]);   // T_dP half h is free again
+                }
+                if (live) {
+                    if (ig0 + 64 <= n) {
 #pragma unroll
-                for (int e = 0; e < 32; ++e) red_add_f32(base + (size_t)(32 + e) * HD, __uint_as_float(v1[e]));
-            } else {
+                        for (int e = 0; e < 32; ++e) red_add_f32(base + (size_t)(part * 32 + e) * HD, __uint_as_float(v0[e]));
+                    } else {
 #pragma unroll
-                for (int e = 0; e < 32; ++e)
-                    if (ig0 + e < n) red_add_f32(base + (size_t)e * HD, __uint_as_float(v0[e]));
-#pragma unroll
-                for (int e = 0; e < 32; ++e)
-                    if (ig0 + 32 + e < n) red_add_f32(base + (size_t)(32 + e) * HD, __uint_as_float(v1[e]));
+                        for (int e = 0; e < 32; ++e)
+                            if (ig0 + part * 32 + e < n) red_add_f32(base + (size_t)(part * 32 + e) * HD, __uint_as_float(v0[e]));
+                    }
+                }
             }
             ++k;
         }
     } else {
-        // ------------------------------------------------------------ warpgroup h owns queries 64 h .. 64 h + 63 of every tile
+        // ------------------------------------------------------------ warps 0-15: exp / dS; warpgroup 2h + qq owns queries 64 h + 32 qq .. + 31
         setmaxnreg_inc<kRegsExp>();
-        const int h = warp / 4;
+        const int h = warp / 8, qq = (warp / 4) & 1;
         const int row = (warp % 4) * 32 + lane;        // tensor-memory lane = key row inside the tile
         const uint32_t lane_addr = (uint32_t)((warp % 4) * 32) << 16;
         const int jg = j0 + row;
@@ -733,24 +733,22 @@ tc_bwd_kernel_v4(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
             const int it = iter.tile(idx);
             if (it < 0) continue;
             const int s = k & 1, i0 = it * TQ;
-            const float4 *sNL = reinterpret_cast<const float4 *>(smem + L::oLSE + s * 512 + h * 256);
-            const float4 *sDs = reinterpret_cast<const float4 *>(smem + L::oD + s * 512 + h * 256);
+            const float4 *sNL = reinterpret_cast<const float4 *>(smem + L::oLSE + s * 512 + h * 256 + qq * 128);
+            const float4 *sDs = reinterpret_cast<const float4 *>(smem + L::oD + s * 512 + h * 256 + qq * 128);
             const bool diag = a.mask_kind == ATTN_MASK_CAUSAL && it == jt;
             const bool masked = diag || i0 + TQ > n || j0 + TK > n;
-            const int ig0 = i0 + h * 64;
-            const uint32_t c0 = h * 64;                // this thread's first column in T_S / T_dP
+            const int ig0 = i0 + h * 64 + qq * 32;
+            const uint32_t c0 = h * 64 + qq * 32;      // this thread's first column in T_S / T_dP
             mbar_wait(&bars[V2_QFULL + s], (k >> 1) & 1, ab);
             mbar_wait(&bars[V2_S + h], k & 1, ab);
             tcgen05_fence_after();
-            uint32_t ppack[32];   // P as bf16 pairs: what dV uses, and what dS is formed from
-            uint32_t svb[2][16];   // two chunks in flight: the load of chunk ch + 1 runs under the arithmetic of chunk ch
-            tmem_ld16(T_S + lane_addr + c0, svb[0]);
+            uint32_t ppack[16];   // P as bf16 pairs: what dV uses, and what dS is formed from
 #pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {   // 16 columns at a time
+            for (int ch = 0; ch < 2; ++ch) {   // 16 columns at a time
                 float p[16];
+                uint32_t sv0[16];
+                tmem_ld16(T_S + lane_addr + c0 + ch * 16, sv0);
                 tmem_wait_ld();
-                if (ch < 3) tmem_ld16(T_S + lane_addr + c0 + (ch + 1) * 16, svb[(ch + 1) & 1]);
-                const uint32_t *sv0 = svb[ch & 1];
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                     const float4 nl = sNL[ch * 4 + q];
@@ -771,9 +769,10 @@ tc_bwd_kernel_v4(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
 #pragma unroll
                 for (int e = 0; e < 8; ++e) ppack[ch * 8 + e] = pack_bf16(p[2 * e], p[2 * e + 1]);
             }
-            // P^T (bf16 pairs) over the first 32 of this half's 64 S^T columns: only this thread's own
-            // lane is read and written, so no cross-thread ordering is needed
-            tmem_st32(T_S + lane_addr + c0, ppack);
+            // P^T (bf16 pairs) goes over columns this very thread has just read -- quarter 0 to columns
+            // 0..15 of the half, quarter 1 to columns 48..63 -- so no thread overwrites S^T entries another
+            // thread still has to read
+            tmem_st16(T_S + lane_addr + h * 64 + qq * 48, ppack);
             tmem_wait_st();
             tcgen05_fence_before();
             mbar_arrive(&bars[V2_P + h]);
@@ -782,13 +781,11 @@ tc_bwd_kernel_v4(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
             tcgen05_fence_after();
             {
                 uint8_t *slab = smem + L::odS + h * SLAB;
-                uint32_t dvb[2][16];
-                tmem_ld16(T_dP + lane_addr + c0, dvb[0]);
 #pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
+                for (int ch = 0; ch < 2; ++ch) {
+                    uint32_t dv[16];
+                    tmem_ld16(T_dP + lane_addr + c0 + ch * 16, dv);
                     tmem_wait_ld();
-                    if (ch < 3) tmem_ld16(T_dP + lane_addr + c0 + (ch + 1) * 16, dvb[(ch + 1) & 1]);
-                    const uint32_t *dv = dvb[ch & 1];
 #pragma unroll
                     for (int g = 0; g < 2; ++g) {    // 8 query columns = one 16-byte chunk
                         float ds[8], p[8];
@@ -811,7 +808,7 @@ tc_bwd_kernel_v4(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
 #pragma unroll
                             for (int e = 0; e < 8; ++e) ds[e] = p[e] != 0.f ? ds[e] : 0.f;
                         }
-                        *reinterpret_cast<uint4 *>(slab + sw128_offset(row, ch * 16 + g * 8)) =
+                        *reinterpret_cast<uint4 *>(slab + sw128_offset(row, qq * 32 + ch * 16 + g * 8)) =
                             make_uint4(pack_bf16(ds[0], ds[1]), pack_bf16(ds[2], ds[3]), pack_bf16(ds[4], ds[5]),
                                        pack_bf16(ds[6], ds[7]));
                     }
@@ -829,10 +826,9 @@ tc_bwd_kernel_v4(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
             tcgen05_fence_after();
         }
         {
-            const int cq0 = (warp / 4) * (HD / 2);
+            const int cq0 = (warp / 4) * 32;       // d = 64: the upper two warpgroups have no columns
             const int jc = jg < n ? jg : 0;
-#pragma unroll
-            for (int cq = cq0; cq < cq0 + HD / 2; cq += 32) {
+            for (int cq = cq0; cq < cq0 + 32 && cq < HD; cq += 32) {
                 __nv_bfloat16 *pv = a.dV + ((size_t)bh * n + jc) * HD + cq;
                 __nv_bfloat16 *pk = a.dK + ((size_t)bh * n + jc) * HD + cq;
                 uint32_t v[32], w[32];
@@ -911,9 +907,9 @@ attn_status launch_bwd(const Problem &p)
     launch_begin(WITH_DQ ? "tc_bwd_fused" : "tc_bwd_dkdv", p.stream);
     if (WITH_DQ) {
         constexpr uint32_t bytes = HD == 64 ? ((L::kBytes + 1023u) & ~1023u) + SLAB : L::kBytes;
-        if (cudaFuncSetAttribute(tc_bwd_kernel_v4<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(tc_bwd_fused_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
             return ATTN_ERR_LAUNCH;
-        tc_bwd_kernel_v4<HD><<<grid, kThreadsV4, bytes, p.stream>>>(mQ, mK, mV, mdO, a);
+        tc_bwd_fused_kernel<HD><<<grid, kThreadsFused, bytes, p.stream>>>(mQ, mK, mV, mdO, a);
     } else {
         if (cudaFuncSetAttribute(tc_bwd_dkdv_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DkdvSmem<HD>::kBytes) != cudaSuccess)
             return ATTN_ERR_LAUNCH;
