@@ -500,9 +500,14 @@ tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
 template <int N> __device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 constexpr int kThreadsFused = 512 + 256 + 128;  // 16 exp/dS warps, 8 reducer warps, issuer warp, TMA producer warp, 2 idle warps
-// 72 registers everywhere at launch (896 x 72 = 64,512); the reducers give up 24 each, the exp / dS warps take 8:
-// 512 x 80 + 256 x 48 + 128 x 72 = 62,464.
-constexpr int kRegsExp = 80, kRegsReduce = 48;
+// 72 registers everywhere at launch (896 x 72 = 64,512).  d = 128: the reducers give up 24 each and work through
+// their 64 columns in two steps, the exp / dS warps take 8: 512 x 80 + 256 x 48 + 128 x 72 = 62,464.  d = 64: only
+// half of the reducer lanes carry data, nothing is traded, and the reducers read their 64 columns at once so that
+// the tensor-memory columns are released before any reduction is issued.
+template <int HD> struct FusedRegs {
+    static constexpr bool kTrade = HD == 128;
+    static constexpr int kExp = 80, kReduce = 48;
+};
 template <int HD>
 __global__ void __launch_bounds__(kThreadsFused, 1)
 tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mK_,
@@ -680,7 +685,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
             }
         }
     } else if (warp >= 16) {
-        setmaxnreg_dec<kRegsReduce>();
+        if (FusedRegs<HD>::kTrade) setmaxnreg_dec<FusedRegs<HD>::kReduce>();
         // ------------------------------------------------------------ reducers: dQ_h^T tile -> fp32 accumulator
         // lanes = head-dimension index c, columns = queries: one warp instruction adds 128 contiguous bytes.
         // 32 columns at a time (the reducers run on 48 registers); the half is released after the second load
@@ -694,35 +699,62 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
             if (it < 0) continue;
             const int ig0 = it * TQ + h * 64;
             float *base = a.dQ_acc + ((size_t)bh * n + ig0) * HD + row;
-            mbar_wait(&bars[V2_DQ + h], k & 1, ab);
-            tcgen05_fence_after();
-#pragma unroll
-            for (int part = 0; part < 2; ++part) {
-                uint32_t v0[32];
+            if (FusedRegs<HD>::kTrade) {
+                mbar_wait(&bars[V2_DQ + h], k & 1, ab);
+                tcgen05_fence_after();
+    #pragma unroll
+                for (int part = 0; part < 2; ++part) {
+                    uint32_t v0[32];
+                    if (live) {
+                        tmem_ld32(T_dP + lane_addr + h * 64 + part * 32, v0);
+                        tmem_wait_ld();
+                    }
+                    if (part == 1) {
+                        tcgen05_fence_before();
+                        mbar_arrive(&bars[V2_DQDONE + h]);   // T_dP half h is free again
+                    }
+                    if (live) {
+                        if (ig0 + 64 <= n) {
+    #pragma unroll
+                            for (int e = 0; e < 32; ++e) red_add_f32(base + (size_t)(part * 32 + e) * HD, __uint_as_float(v0[e]));
+                        } else {
+    #pragma unroll
+                            for (int e = 0; e < 32; ++e)
+                                if (ig0 + part * 32 + e < n) red_add_f32(base + (size_t)(part * 32 + e) * HD, __uint_as_float(v0[e]));
+                        }
+                    }
+                }
+            } else {
+                mbar_wait(&bars[V2_DQ + h], k & 1, ab);
+                tcgen05_fence_after();
+                uint32_t v0[32], v1[32];
                 if (live) {
-                    tmem_ld32(T_dP + lane_addr + h * 64 + part * 32, v0);
+                    tmem_ld32(T_dP + lane_addr + h * 64, v0);
+                    tmem_ld32(T_dP + lane_addr + h * 64 + 32, v1);
                     tmem_wait_ld();
                 }
-                if (part == 1) {
-                    tcgen05_fence_before();
-                    mbar_arrive(&bars[V2_DQDONE + h]);   // T_dP half h is free again
-                }
-                if (live) {
-                    if (ig0 + 64 <= n) {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) red_add_f32(base + (size_t)(part * 32 + e) * HD, __uint_as_float(v0[e]));
-                    } else {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e)
-                            if (ig0 + part * 32 + e < n) red_add_f32(base + (size_t)(part * 32 + e) * HD, __uint_as_float(v0[e]));
-                    }
+                tcgen05_fence_before();
+                mbar_arrive(&bars[V2_DQDONE + h]);   // T_dP half h is free again; the reductions proceed from registers
+                if (!live) {
+                } else if (ig0 + 64 <= n) {
+    #pragma unroll
+                    for (int e = 0; e < 32; ++e) red_add_f32(base + (size_t)e * HD, __uint_as_float(v0[e]));
+    #pragma unroll
+                    for (int e = 0; e < 32; ++e) red_add_f32(base + (size_t)(32 + e) * HD, __uint_as_float(v1[e]));
+                } else {
+    #pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        if (ig0 + e < n) red_add_f32(base + (size_t)e * HD, __uint_as_float(v0[e]));
+    #pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        if (ig0 + 32 + e < n) red_add_f32(base + (size_t)(32 + e) * HD, __uint_as_float(v1[e]));
                 }
             }
             ++k;
         }
     } else {
         // ------------------------------------------------------------ warps 0-15: exp / dS; warpgroup 2h + qq owns queries 64 h + 32 qq .. + 31
-        setmaxnreg_inc<kRegsExp>();
+        if (FusedRegs<HD>::kTrade) setmaxnreg_inc<FusedRegs<HD>::kExp>();
         const int h = warp / 8, qq = (warp / 4) & 1;
         const int row = (warp % 4) * 32 + lane;        // tensor-memory lane = key row inside the tile
         const uint32_t lane_addr = (uint32_t)((warp % 4) * 32) << 16;
