@@ -400,6 +400,8 @@ def main():
     fwd_ms = sum(ev[s][0].elapsed_time(ev[s][1]) for s in range(args.steps))
     bwd_ms = sum(ev[s][1].elapsed_time(ev[s][2]) for s in range(args.steps))
     step_ms = sum(ev[s][0].elapsed_time(ev[s][2]) for s in range(args.steps))
+    bwd_each = sorted(ev[s][1].elapsed_time(ev[s][2]) for s in range(args.steps))
+    fwd_each = sorted(ev[s][0].elapsed_time(ev[s][1]) for s in range(args.steps))
     st = attn.attn_workspace_status(ws_b)
     if st != attn.ATTN_OK or attn.attn_workspace_status(ws_f) != attn.ATTN_OK:
         raise SystemExit("kernel reported a device-side timeout")
@@ -499,6 +501,8 @@ def main():
                    "per_rank_batch": w.batch},
         "fwd_tflops": ff_all * args.steps / (fwd_ms * 1e-3) / 1e12,
         "fwd_ms": fwd_ms / args.steps, "bwd_ms": bwd_ms / args.steps, "wall_ms_per_step": wall_ms / args.steps,
+        "bwd_ms_median": bwd_each[len(bwd_each) // 2], "bwd_ms_min": bwd_each[0],
+        "fwd_ms_median": fwd_each[len(fwd_each) // 2], "fwd_ms_min": fwd_each[0],
         "frac_of_sustained_peak": value / world / peaks["bf16_tflops_sustained"],
         "clocks": clocks, "gpu_launches": int(launches_all),
         "roofline": roofline, "roofline_hbm": roofline_hbm, "io": io,
