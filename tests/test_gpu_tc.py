@@ -156,3 +156,23 @@ def test_deterministic_backward_is_bitwise_repeatable():
     for other in runs[1:]:
         for a, b in zip(runs[0], other):
             assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("b,h", [(1, 3), (3, 2), (3, 4), (1, 8), (5, 1)])
+@pytest.mark.parametrize("deterministic", [0, 1])
+def test_head_group_sizes_and_explicit_scale(b, h, deterministic):
+    """batch * heads = 3, 6, 12, 8, 5: the launch groups heads by 1, 2, 4, 8, 1; the scale is not 1/sqrt(d)."""
+    from paper_2410_09397_b200 import binding as B
+    cfg = B.Cfg(algo=B.ATTN_ALGO_FUSED, deterministic=deterministic)
+    errs = H.run_case(b, h, 392, 128, "bf16", inputs.MASK_CAUSAL, seed=41, cfg=cfg, scale=0.11, check_bwd_only=False)
+    H.assert_within(errs, "bf16")
+
+
+@pytest.mark.parametrize("d", [64, 128])
+def test_deterministic_block_sparse_with_per_head_masks(d):
+    from paper_2410_09397_b200 import binding as B
+    b, h, n, block = 2, 2, 768, 128
+    bm = inputs.block_mask(42, n // block, 0.35, heads=b * h)
+    cfg = B.Cfg(algo=B.ATTN_ALGO_FUSED, deterministic=1)
+    errs = H.run_case(b, h, n, d, "bf16", inputs.MASK_BLOCK_SPARSE, seed=42, block=block, bmask=bm, cfg=cfg)
+    H.assert_within(errs, "bf16")

@@ -149,3 +149,26 @@ def test_weight_kernels_at_headline_size_on_sampled_units():
         a, gg = to_np(A[bi, hi])[None, None], to_np(G[bi, hi])[None, None]
         assert rel_err(to_np(out[bi, hi]), orc.project(a, to_np(W[hi])[None])[0, 0]) <= TOL["bf16"]
         assert rel_err(to_np(g[u]), orc.weight_grad(a, gg, 1)[0]) <= TOL["bf16"]
+
+
+def test_weight_gradients_through_a_block_sparse_mask():
+    """The whole path with the 128 x 128 block mask of the sparse workload's kind (diagonal kept, others with
+    probability 0.3), one weight per head, against the oracle."""
+    import torch
+    import paper_2410_09397_b200 as attn
+    from paper_2410_09397_b200 import binding as B
+    b, h, n, d, block = 1, 2, 640, 128, 128
+    A1, A2, A3, dO = (inputs.normal_tensor(35, t, (b, h, n, d), bf16=True) for t in range(4))
+    X, Y = weights(35, 4, h, d, "bf16"), weights(35, 5, h, d, "bf16")
+    bm = inputs.block_mask(36, n // block, 0.3)
+    ref = orc.attn_weights_bwd(A1, A2, A3, X, Y, dO, mask_kind=orc.MASK_BLOCK, block=block, mask_bits=bm)
+    dev = {k: to_dev(v, "bf16") for k, v in dict(A1=A1, A2=A2, A3=A3, dO=dO, X=X, Y=Y).items()}
+    mask = B.Mask(kind=inputs.MASK_BLOCK_SPARSE, block=block, block_mask=torch.from_numpy(bm).cuda())
+    S, hh = attn.attn_project(dev["A1"], dev["X"]), attn.attn_project(dev["A3"], dev["Y"])
+    O, LSE = attn.attn_fwd(S, dev["A2"], hh, mask=mask)
+    ws = torch.zeros(B.attn_weights_bwd_workspace_bytes(n, d, h, b, mask, B.ATTN_BF16, None), dtype=torch.uint8,
+                     device="cuda")
+    gX, gY = attn.attn_weights_bwd(dev["A1"], dev["A2"], dev["A3"], S, hh, O, dev["dO"], LSE, h, mask=mask, workspace=ws)
+    torch.cuda.synchronize()
+    assert attn.attn_workspace_status(ws) == attn.ATTN_OK
+    assert rel_err(to_np(gX), ref["gX"]) <= TOL["bf16"] and rel_err(to_np(gY), ref["gY"]) <= TOL["bf16"]
