@@ -60,7 +60,7 @@ struct BwdSmem {
     static constexpr uint32_t oLSE = odS + 2 * SLAB;      // 2 stages x 128 floats
     static constexpr uint32_t oD = oLSE + 2 * 128 * 4;
     static constexpr uint32_t oBar = oD + 2 * 128 * 4;    // mbarriers (8 bytes each)
-    static constexpr uint32_t oMisc = oBar + 20 * 8;      // tmem base, abort flag
+    static constexpr uint32_t oMisc = oBar + 24 * 8;      // tmem base, abort flag
     static constexpr uint32_t kBytes = oMisc + 64;
     static_assert(kBytes <= 227 * 1024, "shared memory budget");
 };
@@ -163,7 +163,8 @@ __global__ void __launch_bounds__(256) tc_preprocess_kernel(const __nv_bfloat16 
 }
 
 // barrier indices of the fused kernel: every barrier exists once per 64-query half of a tile
-enum { V2_KV = 0, V2_QFULL = 1, V2_QEMPTY = 3, V2_S = 5, V2_DP = 7, V2_P = 9, V2_DS = 11, V2_DQ = 13, V2_DQDONE = 15 };
+enum { V2_KV = 0, V2_QFULL = 1, V2_QEMPTY = 3, V2_S = 5, V2_DP = 7, V2_P = 9, V2_DS = 11, V2_DQ = 13, V2_DQDONE = 15, V2_SLD = 17,
+       V2_DPLD = 19, V2_DQREL = 21 };
 
 // ---------------------------------------------------------------------------------------
 // dK and dV only: the key-stationary half of the path without atomics (dQ comes from the
@@ -495,31 +496,44 @@ tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
 // reducers, which do nothing but move finished dQ^T tiles from tensor memory into the fp32
 // accumulator, so that the red.global.add queue stalls them and not the warps on the tile loop;
 // warp 24 lane 0 issues every product, warp 25 lane 0 every TMA load; warps 26-27 only complete
-// that warpgroup.  The exp / dS warps keep P only as the bf16 pairs they hand to the dV product, and
-// form dS from those.  Registers are traded between the warpgroups after launch (setmaxnreg).
+// that warpgroup.
+//
+// Tensor memory: region A (128 columns) receives S^T and dP^T in turn, region B (128 columns) holds
+// P^T (bf16 pairs, 32 columns per half) and then dQ^T.  An exp / dS thread copies its 32 columns of
+// S^T (and later of dP^T) into registers at once and releases region A right away, so the next
+// product into A runs while the exponentials (or the dS arithmetic) are still being computed:
+//
+//   issuer:  dP^T(k) -> A | dV += P^T(k) dO   | S^T(k+1) -> A | dQ^T(k) -> B | dK += dS^T(k) Q
+//   waits :  S(k) read    | P(k) written in B | dP(k) read    | dS(k) in shared memory
+//
+// The exp / dS warps keep P only as the bf16 pairs they hand to the dV product, and form dS from
+// those.  Registers are traded between the warpgroups after launch (setmaxnreg).
 template <int N> __device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 constexpr int kThreadsFused = 512 + 256 + 128;  // 16 exp/dS warps, 8 reducer warps, issuer warp, TMA producer warp, 2 idle warps
-// 72 registers everywhere at launch (896 x 72 = 64,512).  d = 128: the reducers give up 24 each and work through
-// their 64 columns in two steps, the exp / dS warps take 8: 512 x 80 + 256 x 48 + 128 x 72 = 62,464.  d = 64: only
-// half of the reducer lanes carry data, nothing is traded, and the reducers read their 64 columns at once so that
-// the tensor-memory columns are released before any reduction is issued.
-template <int HD> struct FusedRegs {
-    static constexpr bool kTrade = HD == 128;
-    static constexpr int kExp = 80, kReduce = 48;
+// 72 registers everywhere at launch (896 x 72 = 64,512).  The reducers give up 24 each and work through their
+// 64 columns in two steps, the issuer's warpgroup gives up 16, the exp / dS warps take 16:
+// 512 x 88 + 256 x 48 + 128 x 56 = 64,512.
+struct FusedRegs {
+    static constexpr int kExp = 88, kReduce = 48, kIssue = 56;
 };
+// one arrival per warp: every lane has finished (and fenced) its part, lane 0 tells the barrier
+__device__ __forceinline__ void warp_arrive(uint64_t *bar, int lane)
+{
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar);
+}
 template <int HD>
 __global__ void __launch_bounds__(kThreadsFused, 1)
 tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mK_,
                  const __grid_constant__ CUtensorMap mV, const __grid_constant__ CUtensorMap mdO, const BwdArgs a)
 {
-    constexpr bool WITH_DQ = true;
     // d = 64: the dQ^T product needs M = 128, so the K tile's second 64-wide slab of M is an all-zero slab
     constexpr uint32_t oZero = (BwdSmem<HD>::kBytes + 1023u) & ~1023u;
-    constexpr int kHalfThreads = 256;     // exp / dS threads per half
-    constexpr int kReduceThreads = 128;   // reducer threads per half
+    constexpr int kHalfWarps = 8;     // exp / dS warps per half
+    constexpr int kReduceWarps = 4;   // reducer warps per half
     using L = BwdSmem<HD>;
-    static_assert(L::oMisc - L::oBar >= 17 * 8, "barrier area");
+    static_assert(L::oMisc - L::oBar >= 23 * 8, "barrier area");
     extern __shared__ __align__(1024) uint8_t smem[];
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::oBar);
     uint32_t *tmem_base_s = reinterpret_cast<uint32_t *>(smem + L::oMisc);
@@ -545,10 +559,13 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
             mbar_init(&bars[V2_QEMPTY + h], 1);
             mbar_init(&bars[V2_S + h], 1);
             mbar_init(&bars[V2_DP + h], 1);
-            mbar_init(&bars[V2_P + h], kHalfThreads);
-            mbar_init(&bars[V2_DS + h], kHalfThreads);
+            mbar_init(&bars[V2_SLD + h], kHalfWarps);
+            mbar_init(&bars[V2_DPLD + h], kHalfWarps);
+            mbar_init(&bars[V2_P + h], kHalfWarps);
+            mbar_init(&bars[V2_DS + h], kHalfWarps);
             mbar_init(&bars[V2_DQ + h], 1);
-            mbar_init(&bars[V2_DQDONE + h], kReduceThreads);
+            mbar_init(&bars[V2_DQDONE + h], kReduceWarps);
+            mbar_init(&bars[V2_DQREL + h], kReduceWarps);
         }
         fence_barrier_init();
         prefetch_tensormap(&mQ); prefetch_tensormap(&mK_); prefetch_tensormap(&mV); prefetch_tensormap(&mdO);
@@ -562,16 +579,15 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
     __syncthreads();
     tcgen05_fence_after();
     const uint32_t tm = *tmem_base_s;
-    const uint32_t T_S = tm, T_dP = tm + 128, T_dV = tm + 256, T_dK = tm + 256 + HD;
+    const uint32_t T_A = tm, T_B = tm + 128, T_dV = tm + 256, T_dK = tm + 256 + HD;
     constexpr uint32_t HALF_ROWS = 64 * 128;   // byte offset of rows 64.. inside a [128][64] slab
 
     const TileIter iter(a, jt, bh);
 
-    if (warp >= 26) {
-        // idle: they only complete the issuer's warpgroup, which keeps its 72 registers
-    } else if (warp == 25) {
-        // ------------------------------------------------------------ TMA producer: every load, as soon as its stage is free
-        if (lane == 0) {
+    if (warp >= 24) {
+        setmaxnreg_dec<FusedRegs::kIssue>();
+        if (warp == 25 && lane == 0) {
+            // ------------------------------------------------------------ TMA producer: every load, as soon as its stage is free
             auto issue_load = [&](int it, int s) {
                 const int i0 = it * TQ;
                 const uint32_t rows = min(TQ, n - i0);
@@ -600,27 +616,21 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
                 issue_load(it, s);
                 ++k;
             }
-        }
-    } else if (warp == 24) {
-        if (lane == 0) {
-            constexpr uint32_t idesc_s = idesc_bf16(128, 128, 0, 0);       // S^T, dP^T (both halves at once)
-            constexpr uint32_t idesc_dv = idesc_bf16(128, HD, 0, 1);       // dV (A tmem), dK (A K-major smem)
-            constexpr uint32_t idesc_dq = idesc_bf16(128, 128, 1, 1);      // dQ^T
+        } else if (warp == 24 && lane == 0) {
+            // ------------------------------------------------------------ MMA issuer A: the products into region A (S^T, dP^T)
+            constexpr uint32_t idesc_s = idesc_bf16(128, 128, 0, 0);
             // low descriptor words (tc_common.cuh): per-step offsets are added as (bytes >> 4)
             const uint32_t kK = desc_lo_kmajor(smem_u32(smem + L::oK)), kV = desc_lo_kmajor(smem_u32(smem + L::oV));
-            const uint32_t mK = desc_lo_mnmajor(smem_u32(smem + L::oK), HD == 64 ? oZero - L::oK : SLAB);
-            const uint32_t kdS = desc_lo_kmajor(smem_u32(smem + L::odS)), mdS = desc_lo_mnmajor(smem_u32(smem + L::odS), SLAB);
-            constexpr uint32_t kHalf = HALF_ROWS >> 4, kSlab = SLAB >> 4;
-            // S^T = K_j Q_i^T for the whole tile in stage s; one commit per half's barrier
+            constexpr uint32_t kSlab = SLAB >> 4;
+            // S^T = K_j Q_i^T for the whole tile in stage s
             auto issue_S = [&](int s) {
                 const uint32_t kQ = desc_lo_kmajor(smem_u32(smem + L::oQ + s * L::kTile));
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk) {
                     const uint32_t off = (kk / 4) * kSlab + (kk % 4) * 2;
-                    mma_ss_lo(T_S, kK + off, kQ + off, idesc_s, kk > 0);
+                    mma_ss_lo(T_A, kK + off, kQ + off, idesc_s, kk > 0);
                 }
                 mma_commit(&bars[V2_S]);
-                mma_commit(&bars[V2_S + 1]);
             };
             int idx = 0, it = -1;
             while (idx < iter.raw && (it = iter.tile(idx)) < 0) ++idx;
@@ -635,57 +645,77 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
                 const int s = k & 1;
                 int nidx = idx + 1, nit = -1;
                 while (nidx < iter.raw && (nit = iter.tile(nidx)) < 0) ++nidx;
-                const uint32_t sQa = smem_u32(smem + L::oQ + s * L::kTile), sdOa = smem_u32(smem + L::odO + s * L::kTile);
-                const uint32_t kdO = desc_lo_kmajor(sdOa), mdO_ = desc_lo_mnmajor(sdOa, SLAB), mQ_ = desc_lo_mnmajor(sQa, SLAB);
-                // dP^T = V_j dO_i^T once both halves of the previous dQ^T have left T_dP
-                if (WITH_DQ && k > 0) {
-                    mbar_wait(&bars[V2_DQDONE], (k - 1) & 1, ab);
-                    mbar_wait(&bars[V2_DQDONE + 1], (k - 1) & 1, ab);
-                    tcgen05_fence_after();
-                }
+                const uint32_t kdO = desc_lo_kmajor(smem_u32(smem + L::odO + s * L::kTile));
+                // dP^T = V_j dO_i^T into region A once every exp / dS warp holds its part of S^T in registers
+                mbar_wait(&bars[V2_SLD], k & 1, ab);
+                mbar_wait(&bars[V2_SLD + 1], k & 1, ab);
+                tcgen05_fence_after();
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk) {
                     const uint32_t off = (kk / 4) * kSlab + (kk % 4) * 2;
-                    mma_ss_lo(T_dP, kV + off, kdO + off, idesc_s, kk > 0);
+                    mma_ss_lo(T_A, kV + off, kdO + off, idesc_s, kk > 0);
                 }
                 mma_commit(&bars[V2_DP]);
-                mma_commit(&bars[V2_DP + 1]);
-                // dV += P_h^T dO_h
+                // S^T of the next tile into region A as soon as dP^T has been read out of it
+                if (nit >= 0) {
+                    mbar_wait(&bars[V2_DPLD], k & 1, ab);
+                    mbar_wait(&bars[V2_DPLD + 1], k & 1, ab);
+                    mbar_wait(&bars[V2_QFULL + (s ^ 1)], ((k + 1) >> 1) & 1, ab);
+                    tcgen05_fence_after();
+                    issue_S(s ^ 1);
+                }
+                ++k;
+                idx = nidx;
+            }
+        } else if (warp == 26 && lane == 0) {
+            // ------------------------------------------------------------ MMA issuer B: the products that read P^T and dS^T
+            // (dV, dQ^T into region B, dK).  Two issuing threads, because a thread that waits on a barrier or commits
+            // cannot keep the short queue of the tensor pipe filled; everything that orders A's products against B's
+            // goes through the exp / dS warps' barriers.
+            constexpr uint32_t idesc_dv = idesc_bf16(128, HD, 0, 1);       // dV (A tmem), dK (A K-major smem)
+            constexpr uint32_t idesc_dq = idesc_bf16(128, 128, 1, 1);      // dQ^T
+            const uint32_t mK = desc_lo_mnmajor(smem_u32(smem + L::oK), HD == 64 ? oZero - L::oK : SLAB);
+            const uint32_t kdS = desc_lo_kmajor(smem_u32(smem + L::odS)), mdS = desc_lo_mnmajor(smem_u32(smem + L::odS), SLAB);
+            constexpr uint32_t kHalf = HALF_ROWS >> 4, kSlab = SLAB >> 4;
+            int k = 0;
+            for (int idx = 0; idx < iter.raw; ++idx) {
+                if (iter.tile(idx) < 0) continue;
+                const int s = k & 1;
+                const uint32_t mdO_ = desc_lo_mnmajor(smem_u32(smem + L::odO + s * L::kTile), SLAB);
+                const uint32_t mQ_ = desc_lo_mnmajor(smem_u32(smem + L::oQ + s * L::kTile), SLAB);
+                if (k == 0) mbar_wait(&bars[V2_KV], 0, ab);
+                mbar_wait(&bars[V2_QFULL + s], (k >> 1) & 1, ab);
+                // dV += P_h^T dO_h, P_h^T in columns 64 h .. 64 h + 31 of region B
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
                     mbar_wait(&bars[V2_P + h], k & 1, ab);
                     tcgen05_fence_after();
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
-                        mma_ts_lo(T_dV, T_S + 64 * h + (kk < 2 ? kk * 8 : 48 + (kk - 2) * 8), mdO_ + h * kHalf + kk * 128,
-                                  idesc_dv, (k > 0) || (h > 0) || (kk > 0));
+                        mma_ts_lo(T_dV, T_B + 64 * h + kk * 8, mdO_ + h * kHalf + kk * 128, idesc_dv, (k > 0) || (h > 0) || (kk > 0));
                 }
-                // T_S is free again: S^T of the next tile runs while this tile's dS is being formed
-                if (nit >= 0) {
-                    mbar_wait(&bars[V2_QFULL + (s ^ 1)], ((k + 1) >> 1) & 1, ab);
-                    tcgen05_fence_after();
-                    issue_S(s ^ 1);
-                }
-                // dQ^T = K_j^T dS^T first (into T_dP, whose dP^T both halves have consumed): the reducer warps
-                // read it out while dK += dS^T Q_i runs, so dP^T of the next tile is not held up by dK
+                // dQ^T = K_j^T dS^T into region B (this thread's products execute in issue order, so dV has
+                // consumed P^T by then); the reducer warps read it out while dK += dS^T Q_i runs
                 mbar_wait(&bars[V2_DS], k & 1, ab);
                 mbar_wait(&bars[V2_DS + 1], k & 1, ab);
+                if (k > 0) {   // the reducers have read all of the previous dQ^T
+                    mbar_wait(&bars[V2_DQDONE], (k - 1) & 1, ab);
+                    mbar_wait(&bars[V2_DQDONE + 1], (k - 1) & 1, ab);
+                }
                 tcgen05_fence_after();
 #pragma unroll
                 for (int kk = 0; kk < TK / 16; ++kk)
-                    mma_ss_lo(T_dP, mK + kk * 128, mdS + kk * 128, idesc_dq, kk > 0);
+                    mma_ss_lo(T_B, mK + kk * 128, mdS + kk * 128, idesc_dq, kk > 0);
                 mma_commit(&bars[V2_DQ]);
-                mma_commit(&bars[V2_DQ + 1]);
 #pragma unroll
                 for (int kk = 0; kk < TQ / 16; ++kk)
                     mma_ss_lo(T_dK, kdS + (kk / 4) * kSlab + (kk % 4) * 2, mQ_ + kk * 128, idesc_dv, (k > 0) || (kk > 0));
                 mma_commit(&bars[V2_QEMPTY + s]);
                 ++k;
-                idx = nidx;
             }
         }
     } else if (warp >= 16) {
-        if (FusedRegs<HD>::kTrade) setmaxnreg_dec<FusedRegs<HD>::kReduce>();
+        setmaxnreg_dec<FusedRegs::kReduce>();
         // ------------------------------------------------------------ reducers: dQ_h^T tile -> fp32 accumulator
         // lanes = head-dimension index c, columns = queries: one warp instruction adds 128 contiguous bytes.
         // 32 columns at a time (the reducers run on 48 registers); the half is released after the second load
@@ -699,67 +729,41 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
             if (it < 0) continue;
             const int ig0 = it * TQ + h * 64;
             float *base = a.dQ_acc + ((size_t)bh * n + ig0) * HD + row;
-            if (FusedRegs<HD>::kTrade) {
-                mbar_wait(&bars[V2_DQ + h], k & 1, ab);
-                tcgen05_fence_after();
-    #pragma unroll
-                for (int part = 0; part < 2; ++part) {
-                    uint32_t v0[32];
-                    if (live) {
-                        tmem_ld32(T_dP + lane_addr + h * 64 + part * 32, v0);
-                        tmem_wait_ld();
-                    }
-                    if (part == 1) {
-                        tcgen05_fence_before();
-                        mbar_arrive(&bars[V2_DQDONE + h]);   // T_dP half h is free again
-                    }
-                    if (live) {
-                        if (ig0 + 64 <= n) {
-    #pragma unroll
-                            for (int e = 0; e < 32; ++e) red_add_f32(base + (size_t)(part * 32 + e) * HD, __uint_as_float(v0[e]));
-                        } else {
-    #pragma unroll
-                            for (int e = 0; e < 32; ++e)
-                                if (ig0 + part * 32 + e < n) red_add_f32(base + (size_t)(part * 32 + e) * HD, __uint_as_float(v0[e]));
-                        }
-                    }
-                }
-            } else {
-                mbar_wait(&bars[V2_DQ + h], k & 1, ab);
-                tcgen05_fence_after();
-                uint32_t v0[32], v1[32];
+            mbar_wait(&bars[V2_DQ], k & 1, ab);
+            tcgen05_fence_after();
+#pragma unroll
+            for (int part = 0; part < 2; ++part) {
+                uint32_t v0[32];
                 if (live) {
-                    tmem_ld32(T_dP + lane_addr + h * 64, v0);
-                    tmem_ld32(T_dP + lane_addr + h * 64 + 32, v1);
+                    tmem_ld32(T_B + lane_addr + h * 64 + part * 32, v0);
                     tmem_wait_ld();
                 }
                 tcgen05_fence_before();
-                mbar_arrive(&bars[V2_DQDONE + h]);   // T_dP half h is free again; the reductions proceed from registers
-                if (!live) {
-                } else if (ig0 + 64 <= n) {
-    #pragma unroll
-                    for (int e = 0; e < 32; ++e) red_add_f32(base + (size_t)e * HD, __uint_as_float(v0[e]));
-    #pragma unroll
-                    for (int e = 0; e < 32; ++e) red_add_f32(base + (size_t)(32 + e) * HD, __uint_as_float(v1[e]));
-                } else {
-    #pragma unroll
-                    for (int e = 0; e < 32; ++e)
-                        if (ig0 + e < n) red_add_f32(base + (size_t)e * HD, __uint_as_float(v0[e]));
-    #pragma unroll
-                    for (int e = 0; e < 32; ++e)
-                        if (ig0 + 32 + e < n) red_add_f32(base + (size_t)(32 + e) * HD, __uint_as_float(v1[e]));
+                // part 0: the 32 columns that take P^T of the next tile are free; part 1: the whole half is
+                warp_arrive(&bars[(part == 0 ? V2_DQREL : V2_DQDONE) + h], lane);
+                if (live) {
+                    if (ig0 + 64 <= n) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) red_add_f32(base + (size_t)(part * 32 + e) * HD, __uint_as_float(v0[e]));
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if (ig0 + part * 32 + e < n) red_add_f32(base + (size_t)(part * 32 + e) * HD, __uint_as_float(v0[e]));
+                    }
                 }
             }
             ++k;
         }
     } else {
         // ------------------------------------------------------------ warps 0-15: exp / dS; warpgroup 2h + qq owns queries 64 h + 32 qq .. + 31
-        if (FusedRegs<HD>::kTrade) setmaxnreg_inc<FusedRegs<HD>::kExp>();
+        setmaxnreg_inc<FusedRegs::kExp>();
         const int h = warp / 8, qq = (warp / 4) & 1;
         const int row = (warp % 4) * 32 + lane;        // tensor-memory lane = key row inside the tile
         const uint32_t lane_addr = (uint32_t)((warp % 4) * 32) << 16;
         const int jg = j0 + row;
         const float sl2 = a.scale * 1.4426950408889634f;
+        const uint32_t c0 = h * 64 + qq * 32;          // this thread's first column of S^T / dP^T in region A
+        const uint32_t cP = h * 64 + qq * 16;          // and of its bf16 pairs of P^T in region B
         int k = 0;
         for (int idx = 0; idx < iter.raw; ++idx) {
             const int it = iter.tile(idx);
@@ -770,85 +774,85 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
             const bool diag = a.mask_kind == ATTN_MASK_CAUSAL && it == jt;
             const bool masked = diag || i0 + TQ > n || j0 + TK > n;
             const int ig0 = i0 + h * 64 + qq * 32;
-            const uint32_t c0 = h * 64 + qq * 32;      // this thread's first column in T_S / T_dP
             mbar_wait(&bars[V2_QFULL + s], (k >> 1) & 1, ab);
-            mbar_wait(&bars[V2_S + h], k & 1, ab);
+            mbar_wait(&bars[V2_S], k & 1, ab);
             tcgen05_fence_after();
             uint32_t ppack[16];   // P as bf16 pairs: what dV uses, and what dS is formed from
-#pragma unroll
-            for (int ch = 0; ch < 2; ++ch) {   // 16 columns at a time
-                float p[16];
-                uint32_t sv0[16];
-                tmem_ld16(T_S + lane_addr + c0 + ch * 16, sv0);
+            {
+                uint32_t sv[32];
+                tmem_ld32(T_A + lane_addr + c0, sv);
                 tmem_wait_ld();
+                tcgen05_fence_before();
+                warp_arrive(&bars[V2_SLD + h], lane);   // region A may take dP^T
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const float4 nl = sNL[ch * 4 + q];
-                    const uint32_t *sv = &sv0[q * 4];
-                    p[q * 4 + 0] = ex2_approx(fmaf(__uint_as_float(sv[0]), sl2, nl.x));
-                    p[q * 4 + 1] = ex2_approx(fmaf(__uint_as_float(sv[1]), sl2, nl.y));
-                    p[q * 4 + 2] = ex2_approx(fmaf(__uint_as_float(sv[2]), sl2, nl.z));
-                    p[q * 4 + 3] = ex2_approx(fmaf(__uint_as_float(sv[3]), sl2, nl.w));
-                }
-                if (masked) {
+                for (int q = 0; q < 8; ++q) {
+                    const float4 nl = sNL[q];
+                    float p[4];
+                    p[0] = ex2_approx(fmaf(__uint_as_float(sv[q * 4 + 0]), sl2, nl.x));
+                    p[1] = ex2_approx(fmaf(__uint_as_float(sv[q * 4 + 1]), sl2, nl.y));
+                    p[2] = ex2_approx(fmaf(__uint_as_float(sv[q * 4 + 2]), sl2, nl.z));
+                    p[3] = ex2_approx(fmaf(__uint_as_float(sv[q * 4 + 3]), sl2, nl.w));
+                    if (masked) {
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        const int ig = ig0 + ch * 16 + e;
-                        const bool ok = ig < n && jg < n && (!diag || jg <= ig);
-                        p[e] = ok ? p[e] : 0.f;
+                        for (int e = 0; e < 4; ++e) {
+                            const int ig = ig0 + q * 4 + e;
+                            const bool ok = ig < n && jg < n && (!diag || jg <= ig);
+                            p[e] = ok ? p[e] : 0.f;
+                        }
                     }
+                    ppack[q * 2 + 0] = pack_bf16(p[0], p[1]);
+                    ppack[q * 2 + 1] = pack_bf16(p[2], p[3]);
                 }
-#pragma unroll
-                for (int e = 0; e < 8; ++e) ppack[ch * 8 + e] = pack_bf16(p[2 * e], p[2 * e + 1]);
             }
-            // P^T (bf16 pairs) goes over columns this very thread has just read -- quarter 0 to columns
-            // 0..15 of the half, quarter 1 to columns 48..63 -- so no thread overwrites S^T entries another
-            // thread still has to read
-            tmem_st16(T_S + lane_addr + h * 64 + qq * 48, ppack);
+            // P^T goes into the first 32 columns of half h of region B, which the reducers must have emptied
+            // of the previous dQ^T
+            if (k > 0) {
+                mbar_wait(&bars[V2_DQREL + h], (k - 1) & 1, ab);
+                tcgen05_fence_after();
+            }
+            tmem_st16(T_B + lane_addr + cP, ppack);
             tmem_wait_st();
             tcgen05_fence_before();
-            mbar_arrive(&bars[V2_P + h]);
+            warp_arrive(&bars[V2_P + h], lane);
 
-            mbar_wait(&bars[V2_DP + h], k & 1, ab);
+            mbar_wait(&bars[V2_DP], k & 1, ab);
             tcgen05_fence_after();
             {
                 uint8_t *slab = smem + L::odS + h * SLAB;
+                uint32_t dv[32];
+                tmem_ld32(T_A + lane_addr + c0, dv);
+                tmem_wait_ld();
+                tcgen05_fence_before();
+                warp_arrive(&bars[V2_DPLD + h], lane);   // region A may take the next S^T
 #pragma unroll
-                for (int ch = 0; ch < 2; ++ch) {
-                    uint32_t dv[16];
-                    tmem_ld16(T_dP + lane_addr + c0 + ch * 16, dv);
-                    tmem_wait_ld();
+                for (int g = 0; g < 4; ++g) {    // 8 query columns = one 16-byte chunk
+                    float ds[8], p[8];
 #pragma unroll
-                    for (int g = 0; g < 2; ++g) {    // 8 query columns = one 16-byte chunk
-                        float ds[8], p[8];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const uint32_t pk = ppack[ch * 8 + g * 4 + e];   // bf16 -> fp32 is a 16-bit shift
-                            p[2 * e] = __uint_as_float(pk << 16);
-                            p[2 * e + 1] = __uint_as_float(pk & 0xffff0000u);
-                        }
-#pragma unroll
-                        for (int u = 0; u < 2; ++u) {
-                            const float4 dsc = sDs[ch * 4 + g * 2 + u];
-                            const uint32_t *d4 = &dv[g * 8 + u * 4];
-                            ds[u * 4 + 0] = p[u * 4 + 0] * fmaf(__uint_as_float(d4[0]), a.scale, -dsc.x);
-                            ds[u * 4 + 1] = p[u * 4 + 1] * fmaf(__uint_as_float(d4[1]), a.scale, -dsc.y);
-                            ds[u * 4 + 2] = p[u * 4 + 2] * fmaf(__uint_as_float(d4[2]), a.scale, -dsc.z);
-                            ds[u * 4 + 3] = p[u * 4 + 3] * fmaf(__uint_as_float(d4[3]), a.scale, -dsc.w);
-                        }
-                        if (masked) {   // stale tail entries of the row vectors may be anything: select, do not multiply
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) ds[e] = p[e] != 0.f ? ds[e] : 0.f;
-                        }
-                        *reinterpret_cast<uint4 *>(slab + sw128_offset(row, qq * 32 + ch * 16 + g * 8)) =
-                            make_uint4(pack_bf16(ds[0], ds[1]), pack_bf16(ds[2], ds[3]), pack_bf16(ds[4], ds[5]),
-                                       pack_bf16(ds[6], ds[7]));
+                    for (int e = 0; e < 4; ++e) {
+                        const uint32_t pk = ppack[g * 4 + e];   // bf16 -> fp32 is a 16-bit shift
+                        p[2 * e] = __uint_as_float(pk << 16);
+                        p[2 * e + 1] = __uint_as_float(pk & 0xffff0000u);
                     }
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        const float4 dsc = sDs[g * 2 + u];
+                        const uint32_t *d4 = &dv[g * 8 + u * 4];
+                        ds[u * 4 + 0] = p[u * 4 + 0] * fmaf(__uint_as_float(d4[0]), a.scale, -dsc.x);
+                        ds[u * 4 + 1] = p[u * 4 + 1] * fmaf(__uint_as_float(d4[1]), a.scale, -dsc.y);
+                        ds[u * 4 + 2] = p[u * 4 + 2] * fmaf(__uint_as_float(d4[2]), a.scale, -dsc.z);
+                        ds[u * 4 + 3] = p[u * 4 + 3] * fmaf(__uint_as_float(d4[3]), a.scale, -dsc.w);
+                    }
+                    if (masked) {   // stale tail entries of the row vectors may be anything: select, do not multiply
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) ds[e] = p[e] != 0.f ? ds[e] : 0.f;
+                    }
+                    *reinterpret_cast<uint4 *>(slab + sw128_offset(row, qq * 32 + g * 8)) =
+                        make_uint4(pack_bf16(ds[0], ds[1]), pack_bf16(ds[2], ds[3]), pack_bf16(ds[4], ds[5]),
+                                   pack_bf16(ds[6], ds[7]));
                 }
             }
             fence_proxy_async_smem();
-            tcgen05_fence_before();
-            mbar_arrive(&bars[V2_DS + h]);
+            warp_arrive(&bars[V2_DS + h], lane);
             ++k;
         }
         // ------------------------------------------------------------ epilogue: dV_j, dK_j (32 columns per warpgroup)
@@ -863,28 +867,25 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
             for (int cq = cq0; cq < cq0 + 32 && cq < HD; cq += 32) {
                 __nv_bfloat16 *pv = a.dV + ((size_t)bh * n + jc) * HD + cq;
                 __nv_bfloat16 *pk = a.dK + ((size_t)bh * n + jc) * HD + cq;
-                uint32_t v[32], w[32];
-                if (k > 0) {
-                    tmem_ld32(T_dV + lane_addr + cq, v);
-                    tmem_ld32(T_dK + lane_addr + cq, w);
-                    tmem_wait_ld();
-                } else {
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) v[e] = w[e] = 0u;
-                }
-                if (jg < n) {
+                for (int which = 0; which < 2; ++which) {
+                    uint32_t v[32];
+                    if (k > 0) {
+                        tmem_ld32((which == 0 ? T_dV : T_dK) + lane_addr + cq, v);
+                        tmem_wait_ld();
+                    } else {
 #pragma unroll
-                    for (int e = 0; e < 32; e += 8) {
-                        *reinterpret_cast<uint4 *>(pv + e) =
-                            make_uint4(pack_bf16(__uint_as_float(v[e]), __uint_as_float(v[e + 1])),
-                                       pack_bf16(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3])),
-                                       pack_bf16(__uint_as_float(v[e + 4]), __uint_as_float(v[e + 5])),
-                                       pack_bf16(__uint_as_float(v[e + 6]), __uint_as_float(v[e + 7])));
-                        *reinterpret_cast<uint4 *>(pk + e) =
-                            make_uint4(pack_bf16(__uint_as_float(w[e]), __uint_as_float(w[e + 1])),
-                                       pack_bf16(__uint_as_float(w[e + 2]), __uint_as_float(w[e + 3])),
-                                       pack_bf16(__uint_as_float(w[e + 4]), __uint_as_float(w[e + 5])),
-                                       pack_bf16(__uint_as_float(w[e + 6]), __uint_as_float(w[e + 7])));
+                        for (int e = 0; e < 32; ++e) v[e] = 0u;
+                    }
+                    __nv_bfloat16 *po = which == 0 ? pv : pk;
+                    if (jg < n) {
+#pragma unroll
+                        for (int e = 0; e < 32; e += 8)
+                            *reinterpret_cast<uint4 *>(po + e) =
+                                make_uint4(pack_bf16(__uint_as_float(v[e]), __uint_as_float(v[e + 1])),
+                                           pack_bf16(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3])),
+                                           pack_bf16(__uint_as_float(v[e + 4]), __uint_as_float(v[e + 5])),
+                                           pack_bf16(__uint_as_float(v[e + 6]), __uint_as_float(v[e + 7])));
                     }
                 }
             }
