@@ -19,8 +19,9 @@
 //
 // dQ partial tiles are added into an fp32 accumulator in the workspace with
 // red.global.add (the one place where summation order is not fixed); a small kernel
-// converts it to bf16 at the end.  Tensor memory (512 columns): S^T / P^T 128,
-// dP^T then dQ^T 128, dV d, dK d.
+// converts it to bf16 at the end.  Tensor memory (512 columns): 128 shared by S^T and
+// dP^T (fused kernel; S^T / P^T in the dK/dV kernel), 128 by P^T and dQ^T (dP^T / dS^T
+// in the dK/dV kernel), dV d, dK d.
 //
 // Two kernels: tc_bwd_fused_kernel (all five products, the default) and tc_bwd_dkdv_kernel
 // (without the dQ product; `deterministic = 1` pairs it with the query-stationary dQ kernel of
@@ -495,22 +496,23 @@ tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
 // h, so each scheduler has four such warps to hide tensor-memory and MUFU latency); warps 16-23:
 // reducers, which do nothing but move finished dQ^T tiles from tensor memory into the fp32
 // accumulator, so that the red.global.add queue stalls them and not the warps on the tile loop;
-// warp 24 lane 0 issues every product, warp 25 lane 0 every TMA load; warps 26-27 only complete
-// that warpgroup.
+// warp 24 lane 0 issues the products into region A (S^T, dP^T), warp 26 lane 0 the products that read
+// P^T and dS^T (dV, dQ^T, dK), warp 25 lane 0 every TMA load; warp 27 only completes that warpgroup.
 //
 // Tensor memory: region A (128 columns) receives S^T and dP^T in turn, region B (128 columns) holds
 // P^T (bf16 pairs, 32 columns per half) and then dQ^T.  An exp / dS thread copies its 32 columns of
 // S^T (and later of dP^T) into registers at once and releases region A right away, so the next
 // product into A runs while the exponentials (or the dS arithmetic) are still being computed:
 //
-//   issuer:  dP^T(k) -> A | dV += P^T(k) dO   | S^T(k+1) -> A | dQ^T(k) -> B | dK += dS^T(k) Q
-//   waits :  S(k) read    | P(k) written in B | dP(k) read    | dS(k) in shared memory
+//   issuer A:  dP^T(k) -> A  (once S^T(k) has been copied out)  |  S^T(k+1) -> A  (once dP^T(k) has been)
+//   issuer B:  dV += P^T(k) dO  (P^T(k) written in B)  |  dQ^T(k) -> B, dK += dS^T(k) Q  (dS^T(k) in shared
+//              memory, the reducers done with dQ^T(k-1))
 //
 // The exp / dS warps keep P only as the bf16 pairs they hand to the dV product, and form dS from
 // those.  Registers are traded between the warpgroups after launch (setmaxnreg).
 template <int N> __device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 template <int N> __device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
-constexpr int kThreadsFused = 512 + 256 + 128;  // 16 exp/dS warps, 8 reducer warps, issuer warp, TMA producer warp, 2 idle warps
+constexpr int kThreadsFused = 512 + 256 + 128;  // 16 exp/dS warps, 8 reducer warps, two issuer warps, TMA producer warp, 1 idle warp
 // 72 registers everywhere at launch (896 x 72 = 64,512).  The reducers give up 24 each and work through their
 // 64 columns in two steps, the issuer's warpgroup gives up 16, the exp / dS warps take 16:
 // 512 x 88 + 256 x 48 + 128 x 56 = 64,512.
