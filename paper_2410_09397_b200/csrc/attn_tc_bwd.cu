@@ -561,13 +561,13 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
             mbar_init(&bars[V2_QEMPTY + h], 1);
             mbar_init(&bars[V2_S + h], 1);
             mbar_init(&bars[V2_DP + h], 1);
-            mbar_init(&bars[V2_SLD + h], kHalfWarps);
-            mbar_init(&bars[V2_DPLD + h], kHalfWarps);
+            mbar_init(&bars[V2_SLD + h], 2 * kHalfWarps);     // SLD, DPLD, DS, DQDONE, DQREL: index 0 serves both halves
+            mbar_init(&bars[V2_DPLD + h], 2 * kHalfWarps);
             mbar_init(&bars[V2_P + h], kHalfWarps);
-            mbar_init(&bars[V2_DS + h], kHalfWarps);
+            mbar_init(&bars[V2_DS + h], 2 * kHalfWarps);
             mbar_init(&bars[V2_DQ + h], 1);
-            mbar_init(&bars[V2_DQDONE + h], kReduceWarps);
-            mbar_init(&bars[V2_DQREL + h], kReduceWarps);
+            mbar_init(&bars[V2_DQDONE + h], 2 * kReduceWarps);
+            mbar_init(&bars[V2_DQREL + h], 2 * kReduceWarps);
         }
         fence_barrier_init();
         prefetch_tensormap(&mQ); prefetch_tensormap(&mK_); prefetch_tensormap(&mV); prefetch_tensormap(&mdO);
@@ -649,8 +649,10 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
                 while (nidx < iter.raw && (nit = iter.tile(nidx)) < 0) ++nidx;
                 const uint32_t kdO = desc_lo_kmajor(smem_u32(smem + L::odO + s * L::kTile));
                 // dP^T = V_j dO_i^T into region A once every exp / dS warp holds its part of S^T in registers
+                if (k > 0) {   // see the exp / dS warps: P^T of this tile is stored once dP^T has been seen
+                    mbar_wait(&bars[V2_DQREL], (k - 1) & 1, ab);
+                }
                 mbar_wait(&bars[V2_SLD], k & 1, ab);
-                mbar_wait(&bars[V2_SLD + 1], k & 1, ab);
                 tcgen05_fence_after();
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk) {
@@ -661,7 +663,6 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
                 // S^T of the next tile into region A as soon as dP^T has been read out of it
                 if (nit >= 0) {
                     mbar_wait(&bars[V2_DPLD], k & 1, ab);
-                    mbar_wait(&bars[V2_DPLD + 1], k & 1, ab);
                     mbar_wait(&bars[V2_QFULL + (s ^ 1)], ((k + 1) >> 1) & 1, ab);
                     tcgen05_fence_after();
                     issue_S(s ^ 1);
@@ -699,10 +700,8 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
                 // dQ^T = K_j^T dS^T into region B (this thread's products execute in issue order, so dV has
                 // consumed P^T by then); the reducer warps read it out while dK += dS^T Q_i runs
                 mbar_wait(&bars[V2_DS], k & 1, ab);
-                mbar_wait(&bars[V2_DS + 1], k & 1, ab);
                 if (k > 0) {   // the reducers have read all of the previous dQ^T
                     mbar_wait(&bars[V2_DQDONE], (k - 1) & 1, ab);
-                    mbar_wait(&bars[V2_DQDONE + 1], (k - 1) & 1, ab);
                 }
                 tcgen05_fence_after();
 #pragma unroll
@@ -742,7 +741,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
                 }
                 tcgen05_fence_before();
                 // part 0: the 32 columns that take P^T of the next tile are free; part 1: the whole half is
-                warp_arrive(&bars[(part == 0 ? V2_DQREL : V2_DQDONE) + h], lane);
+                warp_arrive(&bars[part == 0 ? V2_DQREL : V2_DQDONE], lane);
                 if (live) {
                     if (ig0 + 64 <= n) {
 #pragma unroll
@@ -785,7 +784,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
                 tmem_ld32(T_A + lane_addr + c0, sv);
                 tmem_wait_ld();
                 tcgen05_fence_before();
-                warp_arrive(&bars[V2_SLD + h], lane);   // region A may take dP^T
+                warp_arrive(&bars[V2_SLD], lane);   // region A may take dP^T
 #pragma unroll
                 for (int q = 0; q < 8; ++q) {
                     const float4 nl = sNL[q];
@@ -806,17 +805,8 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
                     ppack[q * 2 + 1] = pack_bf16(p[2], p[3]);
                 }
             }
-            // P^T goes into the first 32 columns of half h of region B, which the reducers must have emptied
-            // of the previous dQ^T
-            if (k > 0) {
-                mbar_wait(&bars[V2_DQREL + h], (k - 1) & 1, ab);
-                tcgen05_fence_after();
-            }
-            tmem_st16(T_B + lane_addr + cP, ppack);
-            tmem_wait_st();
-            tcgen05_fence_before();
-            warp_arrive(&bars[V2_P + h], lane);
-
+            // dP^T first: copying it out lets S^T of the next tile start.  Its issuer has also seen the reducers
+            // take the previous dQ^T out of the first 32 columns of both halves of region B, where P^T goes
             mbar_wait(&bars[V2_DP], k & 1, ab);
             tcgen05_fence_after();
             {
@@ -825,7 +815,11 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
                 tmem_ld32(T_A + lane_addr + c0, dv);
                 tmem_wait_ld();
                 tcgen05_fence_before();
-                warp_arrive(&bars[V2_DPLD + h], lane);   // region A may take the next S^T
+                warp_arrive(&bars[V2_DPLD], lane);   // region A may take the next S^T
+                tmem_st16(T_B + lane_addr + cP, ppack);
+                tmem_wait_st();
+                tcgen05_fence_before();
+                warp_arrive(&bars[V2_P + h], lane);
 #pragma unroll
                 for (int g = 0; g < 4; ++g) {    // 8 query columns = one 16-byte chunk
                     float ds[8], p[8];
@@ -854,7 +848,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
                 }
             }
             fence_proxy_async_smem();
-            warp_arrive(&bars[V2_DS + h], lane);
+            warp_arrive(&bars[V2_DS], lane);
             ++k;
         }
         // ------------------------------------------------------------ epilogue: dV_j, dK_j (32 columns per warpgroup)
