@@ -97,6 +97,35 @@ def test_large_scores_trigger_rescale():
     assert H.rel_err(H.to_np(LSE), LSE_ref) <= 2e-2
 
 
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("n", [384, 1152])
+@pytest.mark.parametrize("mask_kind", [inputs.MASK_NONE, inputs.MASK_CAUSAL])
+@pytest.mark.parametrize("big", ["odd", "even", "rising"])
+def test_forward_merges_partial_softmaxes_with_unequal_maxima(n, d, mask_kind, big):
+    """The two softmax warpgroups own alternate 128-key tiles and are merged at the end: make the scores of one
+    family of tiles (or of the late tiles) far larger than the others', so that the merge weights differ by
+    many orders of magnitude and the running maxima have to move."""
+    import torch
+    import paper_2410_09397_b200 as attn
+    from oracle import oracle as orc
+    x = H.make_inputs(41, 1, 2, n, d, "bf16")
+    tile = np.arange(n) // 128
+    if big == "rising":
+        shift = np.linspace(0.0, 5.0, n, dtype=np.float32)
+    else:
+        shift = np.where(tile % 2 == (1 if big == "odd" else 0), 4.0, 0.0).astype(np.float32)
+    x["Q"] = inputs.round_to_bf16(np.abs(x["Q"]).astype(np.float32))                       # positive queries:
+    x["K"] = inputs.round_to_bf16((x["K"] * 0.2 + shift[None, None, :, None]).astype(np.float32))   # score ~ shift * |q|_1
+    O_ref, LSE_ref = orc.attn_fwd(x["Q"], x["K"], x["V"], mask_kind=mask_kind)
+    dev = {k: H.to_dev(v, "bf16") for k, v in x.items()}
+    mask = attn.Mask(kind=mask_kind) if mask_kind else None
+    O, LSE = attn.attn_fwd(dev["Q"], dev["K"], dev["V"], mask=mask, cfg=fused())
+    torch.cuda.synchronize()
+    # forward only: with a common offset of 4 on the keys dQ = scale * dS K is a difference of large terms, and
+    # the bf16 rounding of dS (part of the method's storage format) then dominates a tolerance relative to max|dQ|
+    H.assert_within({"O": H.rel_err(H.to_np(O), O_ref), "LSE": H.rel_err(H.to_np(LSE), LSE_ref)}, "bf16")
+
+
 def materialized(tile_k=0):
     from paper_2410_09397_b200 import binding as B
     return B.Cfg(tile_k=tile_k, algo=B.ATTN_ALGO_MATERIALIZED)
