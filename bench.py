@@ -292,6 +292,8 @@ def main():
     ap.add_argument("--deterministic", type=int, default=0)
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling on a smaller case)")
     ap.add_argument("--heads", type=int, default=0, help="override the workload's heads")
+    ap.add_argument("--keep-prob", type=float, default=0.0,
+                    help="override the off-diagonal keep probability of a block-sparse workload (density sweep)")
     ap.add_argument("--profile", action="store_true",
                     help="for runs under ncu: allow fewer than 3 warm-up steps, skip e2e and the CPU baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -311,6 +313,8 @@ def main():
     if args.batch or args.heads:
         w = inputs.Workload(**{**w.__dict__, "batch": args.batch or w.batch, "heads": args.heads or w.heads,
                                "name": w.name + "-reduced"})
+    if args.keep_prob and w.mask == inputs.MASK_BLOCK_SPARSE:
+        w = inputs.Workload(**{**w.__dict__, "keep_prob": args.keep_prob, "name": w.name + "-density"})
     bmask = w.block_mask()
 
     if args.impl == "reference":
@@ -488,6 +492,9 @@ def main():
         bound_el = attn.attn_io_bound_elems(w.n, w.d, M, True) * (0.5 if w.mask == inputs.MASK_CAUSAL else 1.0) if M else None
     comp = (8 * w.n * w.d * elem + 2 * 4 * w.n) * w.batch * w.heads
     io = {"backward_compulsory_bytes": comp, "onchip_elems_M": M,
+          # Theorem 1.2: Z_input^2 / Z_QK is the cache size at which the two terms of the sparse bound meet
+          "sparse_dividing_M": (float(w.n * w.d) ** 2 / kept_entries(w, bmask)) if w.mask == inputs.MASK_BLOCK_SPARSE else None,
+          "kept_entries_per_head": kept_entries(w, bmask),
           "paper_bound_bytes_at_M": bound_el * elem * w.batch * w.heads if bound_el else None,
           "dram_bytes_measured_dominant_kernel": TRAFFIC.get((max(tot, key=tot.get), w.name)) if tot else None}
     line = {

@@ -918,7 +918,15 @@ attn_status launch_bwd(const Problem &p)
     a.col_ptr = p.col_ptr; a.row_idx = p.row_idx;
     a.scale = p.scale;
     a.status = p.status;
-    a.group = p.BH % 8 == 0 ? 8 : p.BH % 4 == 0 ? 4 : p.BH % 2 == 0 ? 2 : 1;
+    // Heads are launched in groups (key tile major inside a group).  The fp32 dQ accumulators of the heads that
+    // run at the same time should stay in L2 between the reductions of one key tile and the next: otherwise every
+    // reduced sector is fetched from and written back to device memory (measured on the block-sparse workload with
+    // n = 32768: 13 times the compulsory traffic with 8 heads in flight).  So the group is the largest of 8, 4, 2,
+    // 1 that divides the head count and whose accumulators take at most kAccBudget bytes.
+    constexpr size_t kAccBudget = 40u << 20;
+    a.group = 1;
+    for (int g = 8; g > 1; g >>= 1)
+        if (p.BH % g == 0 && (size_t)g * p.n * HD * sizeof(float) <= kAccBudget) { a.group = g; break; }
     const size_t acc_elems = (size_t)p.BH * p.n * HD;
     if (WITH_DQ && cudaMemsetAsync(p.dQ_acc, 0, acc_elems * sizeof(float), p.stream) != cudaSuccess) return ATTN_ERR_LAUNCH;
     {
