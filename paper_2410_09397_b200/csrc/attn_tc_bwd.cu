@@ -167,15 +167,24 @@ __global__ void __launch_bounds__(256) tc_preprocess_kernel(const __nv_bfloat16 
 enum { V2_KV = 0, V2_QFULL = 1, V2_QEMPTY = 3, V2_S = 5, V2_DP = 7, V2_P = 9, V2_DS = 11, V2_DQ = 13, V2_DQDONE = 15, V2_SLD = 17,
        V2_DPLD = 19, V2_DQREL = 21 };
 
+// one arrival per warp: every lane has finished (and fenced) its part, lane 0 tells the barrier
+__device__ __forceinline__ void warp_arrive(uint64_t *bar, int lane)
+{
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar);
+}
+
 // ---------------------------------------------------------------------------------------
 // dK and dV only: the key-stationary half of the path without atomics (dQ comes from the
-// query-stationary kernel).  Without the dQ product dS^T never has to be in shared memory: it
-// is written over dP^T in tensor memory as bf16 pairs, exactly as P^T over S^T, and
-// dK += dS^T Q takes it from there.  The 32 KB this frees hold a third Q stage, and Q, dO and
-// the row statistics are released separately (dO after dV, Q after dK, LSE / D after the dS
-// phase), so loads run up to two tiles ahead.  Products execute on the tensor pipe in issue
-// order, so S^T of tile k+1 is queued right behind dV of tile k, and dP^T of tile k+1 behind
-// dK of tile k, with no wait in between.
+// query-stationary kernel).  Without the dQ product dS^T never has to be in shared memory.
+// Tensor memory: region A (128 columns) receives S^T and dP^T in turn; an exp / dS thread copies its
+// 32 columns into registers with one load and releases the region at once.  Region B (128 columns)
+// holds P^T and dS^T as bf16 pairs (per 64-query half: P^T in columns 64 h .. 64 h + 31, dS^T in
+// 64 h + 32 .. 64 h + 63), from where dV += P^T dO and dK += dS^T Q take them as their A operand.
+// Two MMA-issuing threads: A issues dP^T(k) (once S^T(k) has been copied out and dK(k-1) has left
+// dS^T(k-1)) and S^T(k+1) (once dP^T(k) has been copied out); B issues dV(k) and dK(k).  The 32 KB that
+// dS^T does not take in shared memory hold a third Q stage; Q, dO and the row statistics are released
+// separately (dO after dV, Q after dK, LSE / D after the dS phase).
 template <int HD> struct DkdvSmem {
     static constexpr uint32_t kSlabs = HD / 64;
     static constexpr uint32_t kTile = kSlabs * SLAB;        // one [128][HD] bf16 tile
@@ -191,15 +200,15 @@ template <int HD> struct DkdvSmem {
     static_assert(kBytes <= 227 * 1024, "shared memory budget");
 };
 enum { KD_KV = 0, KD_QFULL = 1, KD_QEMPTY = 4, KD_OFULL = 7, KD_OEMPTY = 9, KD_LFULL = 11, KD_LEMPTY = 13,
-       KD_S = 15, KD_DP = 17, KD_P = 19, KD_DS = 21, KD_DONE = 23 };
-constexpr int kThreadsDkdv = 512 + 64;   // 16 exp/dS warps, MMA issuer warp, TMA producer warp
+       KD_S = 15, KD_DP = 16, KD_SLD = 17, KD_DPLD = 18, KD_P = 19, KD_DS = 21, KD_DONE = 22 };
+constexpr int kThreadsDkdv = 512 + 128;   // 16 exp/dS warps, issuer A, TMA producer, issuer B, one idle warp
 
 template <int HD>
 __global__ void __launch_bounds__(kThreadsDkdv, 1)
 tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mK_,
                    const __grid_constant__ CUtensorMap mV, const __grid_constant__ CUtensorMap mdO, const BwdArgs a)
 {
-    constexpr int kHalfThreads = 256;
+    constexpr int kExpWarps = 16, kHalfWarps = 8;
     using L = DkdvSmem<HD>;
     extern __shared__ __align__(1024) uint8_t smem[];
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::oBar);
@@ -224,12 +233,14 @@ tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
             mbar_init(&bars[KD_OFULL + s], 1);
             mbar_init(&bars[KD_OEMPTY + s], 1);
             mbar_init(&bars[KD_LFULL + s], 1);
-            mbar_init(&bars[KD_LEMPTY + s], 2 * kHalfThreads);
-            mbar_init(&bars[KD_S + s], 1);
-            mbar_init(&bars[KD_DP + s], 1);
-            mbar_init(&bars[KD_P + s], kHalfThreads);
-            mbar_init(&bars[KD_DS + s], kHalfThreads);
+            mbar_init(&bars[KD_LEMPTY + s], kExpWarps);
+            mbar_init(&bars[KD_P + s], kHalfWarps);
         }
+        mbar_init(&bars[KD_S], 1);
+        mbar_init(&bars[KD_DP], 1);
+        mbar_init(&bars[KD_SLD], kExpWarps);
+        mbar_init(&bars[KD_DPLD], kExpWarps);
+        mbar_init(&bars[KD_DS], kExpWarps);
         mbar_init(&bars[KD_DONE], 1);
         fence_barrier_init();
         prefetch_tensormap(&mQ); prefetch_tensormap(&mK_); prefetch_tensormap(&mV); prefetch_tensormap(&mdO);
@@ -239,7 +250,7 @@ tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
     __syncthreads();
     tcgen05_fence_after();
     const uint32_t tm = *tmem_base_s;
-    const uint32_t T_S = tm, T_dP = tm + 128, T_dV = tm + 256, T_dK = tm + 256 + HD;
+    const uint32_t T_A = tm, T_B = tm + 128, T_dV = tm + 256, T_dK = tm + 256 + HD;
     constexpr uint32_t HALF_ROWS = 64 * 128;   // byte offset of rows 64.. inside a [128][64] slab
 
     const TileIter iter(a, jt, bh);
@@ -277,31 +288,19 @@ tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
             }
         }
     } else if (warp == 16) {
-        // ------------------------------------------------------------ MMA issuer
+        // ------------------------------------------------------------ MMA issuer A: the products into region A
         if (lane == 0) {
             constexpr uint32_t idesc_s = idesc_bf16(128, 128, 0, 0);       // S^T, dP^T
-            constexpr uint32_t idesc_dv = idesc_bf16(128, HD, 0, 1);       // dV, dK: A in tensor memory, B MN-major
             const uint32_t kK = desc_lo_kmajor(smem_u32(smem + L::oK)), kV = desc_lo_kmajor(smem_u32(smem + L::oV));
-            constexpr uint32_t kHalf = HALF_ROWS >> 4, kSlab = SLAB >> 4;
+            constexpr uint32_t kSlab = SLAB >> 4;
             auto issue_S = [&](int k) {
                 const uint32_t kQ = desc_lo_kmajor(smem_u32(smem + L::oQ + (k % 3) * L::kTile));
 #pragma unroll
                 for (int kk = 0; kk < HD / 16; ++kk) {
                     const uint32_t off = (kk / 4) * kSlab + (kk % 4) * 2;
-                    mma_ss_lo(T_S, kK + off, kQ + off, idesc_s, kk > 0);
+                    mma_ss_lo(T_A, kK + off, kQ + off, idesc_s, kk > 0);
                 }
                 mma_commit(&bars[KD_S]);
-                mma_commit(&bars[KD_S + 1]);
-            };
-            auto issue_dP = [&](int k) {
-                const uint32_t kdO = desc_lo_kmajor(smem_u32(smem + L::odO + (k & 1) * L::kTile));
-#pragma unroll
-                for (int kk = 0; kk < HD / 16; ++kk) {
-                    const uint32_t off = (kk / 4) * kSlab + (kk % 4) * 2;
-                    mma_ss_lo(T_dP, kV + off, kdO + off, idesc_s, kk > 0);
-                }
-                mma_commit(&bars[KD_DP]);
-                mma_commit(&bars[KD_DP + 1]);
             };
             int idx = 0, it = -1;
             while (idx < iter.raw && (it = iter.tile(idx)) < 0) ++idx;
@@ -310,60 +309,78 @@ tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
                 mbar_wait(&bars[KD_QFULL], 0, ab);
                 tcgen05_fence_after();
                 issue_S(0);
-                mbar_wait(&bars[KD_OFULL], 0, ab);
-                tcgen05_fence_after();
-                issue_dP(0);
             }
             int k = 0;
             while (idx < iter.raw) {
                 int nidx = idx + 1, nit = -1;
                 while (nidx < iter.raw && (nit = iter.tile(nidx)) < 0) ++nidx;
+                // dP^T(k) into region A: S^T(k) copied out, dO(k) landed, and -- because the exp / dS warps store
+                // dS^T(k) as soon as they have seen dP^T(k) -- the dK product of tile k-1 done with dS^T(k-1)
+                mbar_wait(&bars[KD_OFULL + (k & 1)], (k >> 1) & 1, ab);
+                if (k > 0) mbar_wait(&bars[KD_QEMPTY + (k - 1) % 3], ((k - 1) / 3) & 1, ab);
+                mbar_wait(&bars[KD_SLD], k & 1, ab);
+                tcgen05_fence_after();
+                {
+                    const uint32_t kdO = desc_lo_kmajor(smem_u32(smem + L::odO + (k & 1) * L::kTile));
+#pragma unroll
+                    for (int kk = 0; kk < HD / 16; ++kk) {
+                        const uint32_t off = (kk / 4) * kSlab + (kk % 4) * 2;
+                        mma_ss_lo(T_A, kV + off, kdO + off, idesc_s, kk > 0);
+                    }
+                    mma_commit(&bars[KD_DP]);
+                }
+                if (nit >= 0) {   // S^T(k+1) as soon as dP^T(k) has been copied out
+                    mbar_wait(&bars[KD_QFULL + (k + 1) % 3], ((k + 1) / 3) & 1, ab);
+                    mbar_wait(&bars[KD_DPLD], k & 1, ab);
+                    tcgen05_fence_after();
+                    issue_S(k + 1);
+                }
+                ++k;
+                idx = nidx;
+            }
+        }
+    } else if (warp == 18) {
+        // ------------------------------------------------------------ MMA issuer B: dV += P^T dO, dK += dS^T Q
+        if (lane == 0) {
+            constexpr uint32_t idesc_dv = idesc_bf16(128, HD, 0, 1);       // A in tensor memory, B MN-major
+            constexpr uint32_t kHalf = HALF_ROWS >> 4;
+            int k = 0;
+            for (int idx = 0; idx < iter.raw; ++idx) {
+                if (iter.tile(idx) < 0) continue;
                 const uint32_t mdO_ = desc_lo_mnmajor(smem_u32(smem + L::odO + (k & 1) * L::kTile), SLAB);
                 const uint32_t mQ_ = desc_lo_mnmajor(smem_u32(smem + L::oQ + (k % 3) * L::kTile), SLAB);
-                // dV += P_h^T dO_h
+                mbar_wait(&bars[KD_OFULL + (k & 1)], (k >> 1) & 1, ab);
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
                     mbar_wait(&bars[KD_P + h], k & 1, ab);
                     tcgen05_fence_after();
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
-                        mma_ts_lo(T_dV, T_S + 64 * h + (kk < 2 ? kk * 8 : 48 + (kk - 2) * 8), mdO_ + h * kHalf + kk * 128,
-                                  idesc_dv, (k > 0) || (h > 0) || (kk > 0));
+                        mma_ts_lo(T_dV, T_B + 64 * h + kk * 8, mdO_ + h * kHalf + kk * 128, idesc_dv, (k > 0) || (h > 0) || (kk > 0));
                 }
                 mma_commit(&bars[KD_OEMPTY + (k & 1)]);
-                if (nit >= 0) {
-                    mbar_wait(&bars[KD_QFULL + (k + 1) % 3], ((k + 1) / 3) & 1, ab);
-                    tcgen05_fence_after();
-                    issue_S(k + 1);
-                }
-                // dK += dS_h^T Q_h
+                mbar_wait(&bars[KD_QFULL + k % 3], (k / 3) & 1, ab);
+                mbar_wait(&bars[KD_DS], k & 1, ab);
+                tcgen05_fence_after();
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    mbar_wait(&bars[KD_DS + h], k & 1, ab);
-                    tcgen05_fence_after();
+                for (int h = 0; h < 2; ++h)
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
-                        mma_ts_lo(T_dK, T_dP + 64 * h + (kk < 2 ? kk * 8 : 48 + (kk - 2) * 8), mQ_ + h * kHalf + kk * 128,
-                                  idesc_dv, (k > 0) || (h > 0) || (kk > 0));
-                }
+                        mma_ts_lo(T_dK, T_B + 64 * h + 32 + kk * 8, mQ_ + h * kHalf + kk * 128, idesc_dv, (k > 0) || (h > 0) || (kk > 0));
                 mma_commit(&bars[KD_QEMPTY + k % 3]);
-                if (nit >= 0) {
-                    mbar_wait(&bars[KD_OFULL + ((k + 1) & 1)], ((k + 1) >> 1) & 1, ab);
-                    tcgen05_fence_after();
-                    issue_dP(k + 1);
-                }
                 ++k;
-                idx = nidx;
             }
             mma_commit(&bars[KD_DONE]);
         }
-    } else {
+    } else if (warp < 16) {
         // ------------------------------------------------------------ warpgroup 2h + qq owns queries 64 h + 32 qq .. + 31
         const int h = warp / 8, qq = (warp / 4) & 1;
         const int row = (warp % 4) * 32 + lane;        // tensor-memory lane = key row inside the tile
         const uint32_t lane_addr = (uint32_t)((warp % 4) * 32) << 16;
         const int jg = j0 + row;
         const float sl2 = a.scale * 1.4426950408889634f;
+        const uint32_t c0 = h * 64 + qq * 32;          // this thread's first column of S^T / dP^T in region A
+        const uint32_t cP = h * 64 + qq * 16;          // of its bf16 pairs of P^T in region B; dS^T 32 columns further
         int k = 0;
         for (int idx = 0; idx < iter.raw; ++idx) {
             const int it = iter.tile(idx);
@@ -374,78 +391,78 @@ tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
             const bool diag = a.mask_kind == ATTN_MASK_CAUSAL && it == jt;
             const bool masked = diag || i0 + TQ > n || j0 + TK > n;
             const int ig0 = i0 + h * 64 + qq * 32;
-            const uint32_t c0 = h * 64 + qq * 32;      // this thread's first column in T_S / T_dP
-            // bf16 pairs go over columns this very thread has just read -- quarter 0 to columns
-            // 0..15 of the half, quarter 1 to columns 48..63 -- so no thread overwrites entries
-            // another thread still has to read
-            const uint32_t cpack = h * 64 + qq * 48;
-            mbar_wait(&bars[KD_LFULL + s2], (k >> 1) & 1, ab);
-            mbar_wait(&bars[KD_S + h], k & 1, ab);
+            mbar_wait(&bars[KD_S], k & 1, ab);
             tcgen05_fence_after();
-            float p[32];
+            uint32_t ppack[16];
             {
-                uint32_t sv0[32];
-                tmem_ld32(T_S + lane_addr + c0, sv0);
+                uint32_t sv[32];
+                tmem_ld32(T_A + lane_addr + c0, sv);
                 tmem_wait_ld();
+                tcgen05_fence_before();
+                warp_arrive(&bars[KD_SLD], lane);   // region A may take dP^T
+                mbar_wait(&bars[KD_LFULL + s2], (k >> 1) & 1, ab);
 #pragma unroll
                 for (int q = 0; q < 8; ++q) {
                     const float4 nl = sNL[q];
-                    const uint32_t *sv = &sv0[q * 4];
-                    p[q * 4 + 0] = ex2_approx(fmaf(__uint_as_float(sv[0]), sl2, nl.x));
-                    p[q * 4 + 1] = ex2_approx(fmaf(__uint_as_float(sv[1]), sl2, nl.y));
-                    p[q * 4 + 2] = ex2_approx(fmaf(__uint_as_float(sv[2]), sl2, nl.z));
-                    p[q * 4 + 3] = ex2_approx(fmaf(__uint_as_float(sv[3]), sl2, nl.w));
+                    float p[4];
+                    p[0] = ex2_approx(fmaf(__uint_as_float(sv[q * 4 + 0]), sl2, nl.x));
+                    p[1] = ex2_approx(fmaf(__uint_as_float(sv[q * 4 + 1]), sl2, nl.y));
+                    p[2] = ex2_approx(fmaf(__uint_as_float(sv[q * 4 + 2]), sl2, nl.z));
+                    p[3] = ex2_approx(fmaf(__uint_as_float(sv[q * 4 + 3]), sl2, nl.w));
+                    if (masked) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int ig = ig0 + q * 4 + e;
+                            const bool ok = ig < n && jg < n && (!diag || jg <= ig);
+                            p[e] = ok ? p[e] : 0.f;
+                        }
+                    }
+                    ppack[q * 2 + 0] = pack_bf16(p[0], p[1]);
+                    ppack[q * 2 + 1] = pack_bf16(p[2], p[3]);
                 }
             }
-            if (masked) {
-#pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    const int ig = ig0 + e;
-                    const bool ok = ig < n && jg < n && (!diag || jg <= ig);
-                    p[e] = ok ? p[e] : 0.f;
-                }
-            }
-            {
-                uint32_t ppack[16];
-#pragma unroll
-                for (int e = 0; e < 16; ++e) ppack[e] = pack_bf16(p[2 * e], p[2 * e + 1]);
-                tmem_st16(T_S + lane_addr + cpack, ppack);
-                tmem_wait_st();
-            }
-            tcgen05_fence_before();
-            mbar_arrive(&bars[KD_P + h]);
-
-            mbar_wait(&bars[KD_DP + h], k & 1, ab);
+            mbar_wait(&bars[KD_DP], k & 1, ab);
             tcgen05_fence_after();
+            uint32_t dv[32];
+            tmem_ld32(T_A + lane_addr + c0, dv);
+            tmem_wait_ld();
+            tcgen05_fence_before();
+            warp_arrive(&bars[KD_DPLD], lane);   // region A may take the next S^T
+            // P^T(k) over P^T(k-1): the dV product of the previous tile must have consumed it
+            if (k > 0) {
+                mbar_wait(&bars[KD_OEMPTY + ((k - 1) & 1)], ((k - 1) >> 1) & 1, ab);
+                tcgen05_fence_after();
+            }
+            tmem_st16(T_B + lane_addr + cP, ppack);
+            tmem_wait_st();
+            tcgen05_fence_before();
+            warp_arrive(&bars[KD_P + h], lane);
             {
-                uint32_t dv0[32], dpack[16];
-                tmem_ld32(T_dP + lane_addr + c0, dv0);
-                tmem_wait_ld();
+                uint32_t dpack[16];
 #pragma unroll
                 for (int q = 0; q < 8; ++q) {
                     const float4 dsc = sDs[q];
-                    const uint32_t *dv = &dv0[q * 4];
-                    // a masked entry has p = 0 and a finite dP, so its dS is an exact zero
-                    const float d0 = p[q * 4 + 0] * fmaf(__uint_as_float(dv[0]), a.scale, -dsc.x);
-                    const float d1 = p[q * 4 + 1] * fmaf(__uint_as_float(dv[1]), a.scale, -dsc.y);
-                    const float d2 = p[q * 4 + 2] * fmaf(__uint_as_float(dv[2]), a.scale, -dsc.z);
-                    const float d3 = p[q * 4 + 3] * fmaf(__uint_as_float(dv[3]), a.scale, -dsc.w);
+                    // bf16 -> fp32 is a 16-bit shift; a masked entry has p = 0 and a finite dP, so its dS is an exact zero
+                    const float p0 = __uint_as_float(ppack[q * 2] << 16), p1 = __uint_as_float(ppack[q * 2] & 0xffff0000u);
+                    const float p2 = __uint_as_float(ppack[q * 2 + 1] << 16), p3 = __uint_as_float(ppack[q * 2 + 1] & 0xffff0000u);
+                    float d0 = p0 * fmaf(__uint_as_float(dv[q * 4 + 0]), a.scale, -dsc.x);
+                    float d1 = p1 * fmaf(__uint_as_float(dv[q * 4 + 1]), a.scale, -dsc.y);
+                    float d2 = p2 * fmaf(__uint_as_float(dv[q * 4 + 2]), a.scale, -dsc.z);
+                    float d3 = p3 * fmaf(__uint_as_float(dv[q * 4 + 3]), a.scale, -dsc.w);
+                    if (masked) {   // stale tail entries of the row vectors may be anything: select, do not multiply
+                        d0 = p0 != 0.f ? d0 : 0.f; d1 = p1 != 0.f ? d1 : 0.f;
+                        d2 = p2 != 0.f ? d2 : 0.f; d3 = p3 != 0.f ? d3 : 0.f;
+                    }
                     dpack[q * 2 + 0] = pack_bf16(d0, d1);
                     dpack[q * 2 + 1] = pack_bf16(d2, d3);
                 }
-                if (masked) {
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        if (p[2 * e] == 0.f) dpack[e] &= 0xffff0000u;
-                        if (p[2 * e + 1] == 0.f) dpack[e] &= 0x0000ffffu;
-                    }
-                }
-                tmem_st16(T_dP + lane_addr + cpack, dpack);
+                // dS^T(k) over dS^T(k-1): the issuer of dP^T(k) has seen the dK product of tile k-1 complete
+                tmem_st16(T_B + lane_addr + 32 + cP, dpack);
                 tmem_wait_st();
             }
             tcgen05_fence_before();
-            mbar_arrive(&bars[KD_DS + h]);
-            mbar_arrive(&bars[KD_LEMPTY + s2]);
+            warp_arrive(&bars[KD_DS], lane);
+            warp_arrive(&bars[KD_LEMPTY + s2], lane);
             ++k;
         }
         // ------------------------------------------------------------ epilogue: dV_j, dK_j (32 columns per warpgroup)
@@ -456,31 +473,27 @@ tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
         {
             const int cq = (warp / 4) * 32;       // d = 64: the upper two warpgroups have no columns
             const int jc = jg < n ? jg : 0;
-            __nv_bfloat16 *pv = a.dV + ((size_t)bh * n + jc) * HD + cq;
-            __nv_bfloat16 *pk = a.dK + ((size_t)bh * n + jc) * HD + cq;
-            uint32_t v[32], w[32];
-            if (k > 0 && cq < HD) {
-                tmem_ld32(T_dV + lane_addr + cq, v);
-                tmem_ld32(T_dK + lane_addr + cq, w);
-                tmem_wait_ld();
-            } else {
+            if (cq < HD) {
 #pragma unroll
-                for (int e = 0; e < 32; ++e) v[e] = w[e] = 0u;
-            }
-            if (jg < n && cq < HD) {
+                for (int which = 0; which < 2; ++which) {
+                    __nv_bfloat16 *po = (which == 0 ? a.dV : a.dK) + ((size_t)bh * n + jc) * HD + cq;
+                    uint32_t v[32];
+                    if (k > 0) {
+                        tmem_ld32((which == 0 ? T_dV : T_dK) + lane_addr + cq, v);
+                        tmem_wait_ld();
+                    } else {
 #pragma unroll
-                for (int e = 0; e < 32; e += 8) {
-                    uint4 ov, ok;
-                    ov.x = pack_bf16(__uint_as_float(v[e]), __uint_as_float(v[e + 1]));
-                    ov.y = pack_bf16(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
-                    ov.z = pack_bf16(__uint_as_float(v[e + 4]), __uint_as_float(v[e + 5]));
-                    ov.w = pack_bf16(__uint_as_float(v[e + 6]), __uint_as_float(v[e + 7]));
-                    ok.x = pack_bf16(__uint_as_float(w[e]), __uint_as_float(w[e + 1]));
-                    ok.y = pack_bf16(__uint_as_float(w[e + 2]), __uint_as_float(w[e + 3]));
-                    ok.z = pack_bf16(__uint_as_float(w[e + 4]), __uint_as_float(w[e + 5]));
-                    ok.w = pack_bf16(__uint_as_float(w[e + 6]), __uint_as_float(w[e + 7]));
-                    *reinterpret_cast<uint4 *>(pv + e) = ov;
-                    *reinterpret_cast<uint4 *>(pk + e) = ok;
+                        for (int e = 0; e < 32; ++e) v[e] = 0u;
+                    }
+                    if (jg < n) {
+#pragma unroll
+                        for (int e = 0; e < 32; e += 8)
+                            *reinterpret_cast<uint4 *>(po + e) =
+                                make_uint4(pack_bf16(__uint_as_float(v[e]), __uint_as_float(v[e + 1])),
+                                           pack_bf16(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3])),
+                                           pack_bf16(__uint_as_float(v[e + 4]), __uint_as_float(v[e + 5])),
+                                           pack_bf16(__uint_as_float(v[e + 6]), __uint_as_float(v[e + 7])));
+                    }
                 }
             }
         }
@@ -519,12 +532,6 @@ constexpr int kThreadsFused = 512 + 256 + 128;  // 16 exp/dS warps, 8 reducer wa
 struct FusedRegs {
     static constexpr int kExp = 88, kReduce = 48, kIssue = 56;
 };
-// one arrival per warp: every lane has finished (and fenced) its part, lane 0 tells the barrier
-__device__ __forceinline__ void warp_arrive(uint64_t *bar, int lane)
-{
-    __syncwarp();
-    if (lane == 0) mbar_arrive(bar);
-}
 template <int HD>
 __global__ void __launch_bounds__(kThreadsFused, 1)
 tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mK_,

@@ -14,7 +14,7 @@
 // the price of summing dQ in a fixed order: 7 products instead of 5 per tile pair.
 // Roles: warps 0-15 = four warpgroups, warpgroup g owning key columns 32 g .. 32 g + 31 of every
 // tile (no barrier couples them, so their exp, dS and tensor-memory phases interleave freely);
-// warp 16 lane 0 issues MMAs, warp 17 lane 0 runs TMA.  Tensor memory: S0 128, S1 128, dP 128, dQ d columns.
+// warp 16 lane 0 issues S and dP, warp 17 lane 0 issues dQ, warp 18 lane 0 runs TMA.  Tensor memory: S0 128, S1 128, dP 128, dQ d columns.
 #include "attn_internal.h"
 #include "tc_common.cuh"
 
@@ -25,7 +25,7 @@ using namespace tc;
 
 constexpr int TQ = 128, TKD = 128;
 constexpr int kSoftmaxThreads = 512;
-constexpr int kThreads = kSoftmaxThreads + 64;
+constexpr int kThreads = kSoftmaxThreads + 96;   // + two MMA-issuing warps and the TMA warp
 constexpr uint32_t SLAB = 128 * 128;
 
 struct DqArgs {
@@ -116,9 +116,9 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
         mbar_init(&bars[DB_Q], 1);
         for (int s = 0; s < NSTK; ++s) { mbar_init(&bars[DB_KFULL + s], 1); mbar_init(&bars[DB_KEMPTY + s], 1); }
         for (int s = 0; s < NSTV; ++s) { mbar_init(&bars[DB_VFULL + s], 1); mbar_init(&bars[DB_VEMPTY + s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&bars[DB_S + b], 1); mbar_init(&bars[DB_DS + b], kSoftmaxThreads); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&bars[DB_S + b], 1); mbar_init(&bars[DB_DS + b], kSoftmaxThreads / 32); }   // one arrival per warp
         mbar_init(&bars[DB_DP], 1);
-        mbar_init(&bars[DB_DPFREE], kSoftmaxThreads);
+        mbar_init(&bars[DB_DPFREE], kSoftmaxThreads / 32);
         mbar_init(&bars[DB_DQ], 1);
         fence_barrier_init();
         prefetch_tensormap(&mQ); prefetch_tensormap(&mK); prefetch_tensormap(&mV); prefetch_tensormap(&mdO);
@@ -133,7 +133,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
     int niter = 0;
     for (int idx = 0; idx < iter.raw; ++idx) niter += iter.tile(idx) >= 0;
 
-    if (warp == 17) {
+    if (warp == 18) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             mbar_expect_tx(&bars[DB_Q], 2 * L::kTile);
@@ -162,15 +162,18 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
             if (niter == 0) mbar_wait(&bars[DB_Q], 0, ab);   // let the Q / dO load land before exit
         }
     } else if (warp == 16) {
-        // ------------------------------------------------------------ MMA issuer
+        // ------------------------------------------------------------ MMA issuer A: the products the warps wait for, S and dP,
+        // one tile ahead.  (Two issuing threads: a thread that waits on a barrier or commits cannot keep the short
+        // queue of the tensor pipe filled; B's dQ products are ordered against A's through barriers only.)
         if (lane == 0 && niter > 0) {
             constexpr uint32_t idesc_s = idesc_bf16(128, 128, 0, 0);
-            constexpr uint32_t idesc_dq = idesc_bf16(128, HD, 0, 1);
             constexpr uint32_t kSlab = SLAB >> 4;
             const uint32_t kQ = desc_lo_kmajor(smem_u32(smem + L::oQ)), kdO = desc_lo_kmajor(smem_u32(smem + L::odO));
             auto issue_S = [&](int k) {
                 const int s = k % NSTK;
                 mbar_wait(&bars[DB_KFULL + s], (k / NSTK) & 1, ab);
+                // the buffer of S(k) held dS(k-2): the dQ product of tile k-2 (other thread) must have consumed it
+                if (k >= 2) mbar_wait(&bars[DB_KEMPTY + (k - 2) % NSTK], ((k - 2) / NSTK) & 1, ab);
                 tcgen05_fence_after();
                 const uint32_t kK = desc_lo_kmajor(smem_u32(smem + L::oK + s * L::kTile));
 #pragma unroll
@@ -192,21 +195,24 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
                 mma_commit(&bars[DB_DP]);
                 mma_commit(&bars[DB_VEMPTY + k % NSTV]);
             };
-            // Queue order: S(k+1) and dP(k+1) are issued while the warps still work on tile k, so that
-            // neither is waited for; only dQ(k) needs the warps' result.
             mbar_wait(&bars[DB_Q], 0, ab);
             issue_S(0);
             issue_dP(0);
+            for (int k = 0; k + 1 < niter; ++k) {
+                issue_S(k + 1);
+                // dP(k+1) once every thread has read dP(k) out of tensor memory
+                mbar_wait(&bars[DB_DPFREE], k & 1, ab);
+                tcgen05_fence_after();
+                issue_dP(k + 1);
+            }
+        }
+    } else if (warp == 17) {
+        // ------------------------------------------------------------ MMA issuer B: dQ_i += dS K_j
+        if (lane == 0 && niter > 0) {
+            constexpr uint32_t idesc_dq = idesc_bf16(128, HD, 0, 1);
             for (int k = 0; k < niter; ++k) {
                 const int s = k % NSTK, b = k & 1;
-                if (k + 1 < niter) {
-                    issue_S(k + 1);   // its buffer held dS(k-1), which the dQ product queued last iteration has consumed
-                    // dP(k+1) once every thread has read dP(k) out of tensor memory
-                    mbar_wait(&bars[DB_DPFREE], k & 1, ab);
-                    tcgen05_fence_after();
-                    issue_dP(k + 1);
-                }
-                // dQ_i += dS K_j
+                mbar_wait(&bars[DB_KFULL + s], (k / NSTK) & 1, ab);
                 mbar_wait(&bars[DB_DS + b], (k >> 1) & 1, ab);
                 tcgen05_fence_after();
                 const uint32_t mK_ = desc_lo_mnmajor(smem_u32(smem + L::oK + s * L::kTile), SLAB);
@@ -260,7 +266,8 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
                 tmem_ld32(T_dP + lane_addr + wg * 32, dv0);
                 tmem_wait_ld();
                 tcgen05_fence_before();
-                mbar_arrive(&bars[DB_DPFREE]);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars[DB_DPFREE]);
 #pragma unroll
                 for (int e = 0; e < 32; e += 2)
                     dpack[e / 2] = pack_bf16(p[e] * fmaf(__uint_as_float(dv0[e]), a.scale, -dsi),
@@ -270,7 +277,8 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
             tmem_st16(T_S + lane_addr + wg * 32, dpack);
             tmem_wait_st();
             tcgen05_fence_before();
-            mbar_arrive(&bars[DB_DS + b]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars[DB_DS + b]);
             ++k;
         }
         // ------------------------------------------------------------ epilogue: dQ_i (dS carried the scale)
