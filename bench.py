@@ -541,6 +541,8 @@ def main():
             elem = 2 if w.bf16 else 4
             rows = w.batch * w.heads * w.n
             by = rows * (2 * w.d * elem + (12 if name != "bwd_preprocess_D" else 4))
+            if name == "tc_bwd_preprocess" and "tc_bwd_fused" in kernel_ms:
+                by += rows * w.d * 4   # the same pass clears the fp32 dQ accumulator of the fused backward
             avg = sum(kernel_ms[name]) / len(kernel_ms[name])
             gbs = by / (avg * 1e-3) / 1e9
             roofline_hbm = {"bound": "hbm", "kernel": name, "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",

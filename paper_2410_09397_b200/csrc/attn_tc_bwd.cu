@@ -116,12 +116,15 @@ __device__ __forceinline__ float ex2_approx(float x)
 
 // D pre-pass of the fused backward: Ds_i = scale * sum_c dO_ic O_ic and
 // nlse2_i = -LSE_i * log2(e) (minus infinity for a row with no kept entry, so that its
-// probabilities come out as exactly zero).  16-byte loads, HD/8 lanes share a row.
+// probabilities come out as exactly zero).  16-byte loads, HD/8 lanes share a row.  The same
+// pass clears the fp32 dQ accumulator of the fused backward (`acc`, `acc16` 16-byte words; null =
+// nothing to clear), so that its writes overlap the reads of O and dO.
 template <int HD>
 __global__ void __launch_bounds__(256) tc_preprocess_kernel(const __nv_bfloat16 *__restrict__ O,
                                                             const __nv_bfloat16 *__restrict__ dO,
                                                             const float *__restrict__ LSE, float *__restrict__ Ds,
-                                                            float *__restrict__ nlse2, size_t rows, float scale)
+                                                            float *__restrict__ nlse2, size_t rows, float scale,
+                                                            uint4 *__restrict__ acc, size_t acc16)
 {
     constexpr int LPR = HD / 8;   // lanes per row
     constexpr int RPW = 32 / LPR; // rows per warp
@@ -129,6 +132,10 @@ __global__ void __launch_bounds__(256) tc_preprocess_kernel(const __nv_bfloat16 
     const int lane = threadIdx.x % 32, sub = lane / LPR, lr = lane % LPR;
     const size_t warp = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) / 32;
     const size_t nwarps = (size_t)gridDim.x * blockDim.x / 32;
+    if (acc != nullptr) {
+        for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < acc16; i += (size_t)gridDim.x * blockDim.x)
+            __stcs(acc + i, make_uint4(0u, 0u, 0u, 0u));
+    }
     for (size_t base = warp * RPW * U; base < rows; base += nwarps * RPW * U) {
         uint4 xo[U], xg[U];
 #pragma unroll
@@ -935,7 +942,6 @@ attn_status launch_bwd(const Problem &p)
     for (int g = 8; g > 1; g >>= 1)
         if (p.BH % g == 0 && (size_t)g * p.n * HD * sizeof(float) <= kAccBudget) { a.group = g; break; }
     const size_t acc_elems = (size_t)p.BH * p.n * HD;
-    if (WITH_DQ && cudaMemsetAsync(p.dQ_acc, 0, acc_elems * sizeof(float), p.stream) != cudaSuccess) return ATTN_ERR_LAUNCH;
     {
         const size_t rows = (size_t)p.BH * p.n;
         constexpr size_t rpw = 32 / (HD / 8);
@@ -943,7 +949,8 @@ attn_status launch_bwd(const Problem &p)
         if (blocks > 148 * 8) blocks = 148 * 8;
         launch_begin("tc_bwd_preprocess", p.stream);
         tc_preprocess_kernel<HD><<<(unsigned)blocks, 256, 0, p.stream>>>((const __nv_bfloat16 *)p.O, (const __nv_bfloat16 *)p.dO,
-                                                                         p.LSE, p.D, p.nLSE2, rows, p.scale);
+                                                                         p.LSE, p.D, p.nLSE2, rows, p.scale,
+                                                                         WITH_DQ ? (uint4 *)p.dQ_acc : nullptr, acc_elems / 4);
         launch_end(p.stream);
         if (cudaGetLastError() != cudaSuccess) return ATTN_ERR_LAUNCH;
     }
