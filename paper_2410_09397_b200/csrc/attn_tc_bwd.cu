@@ -542,7 +542,8 @@ struct FusedRegs {
 template <int HD>
 __global__ void __launch_bounds__(kThreadsFused, 1)
 tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mK_,
-                 const __grid_constant__ CUtensorMap mV, const __grid_constant__ CUtensorMap mdO, const BwdArgs a)
+                 const __grid_constant__ CUtensorMap mV, const __grid_constant__ CUtensorMap mdO,
+                 const __grid_constant__ CUtensorMap mdK, const __grid_constant__ CUtensorMap mdV, const BwdArgs a)
 {
     // d = 64: the dQ^T product needs M = 128, so the K tile's second 64-wide slab of M is an all-zero slab
     constexpr uint32_t oZero = (BwdSmem<HD>::kBytes + 1023u) & ~1023u;
@@ -872,11 +873,11 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
             tcgen05_fence_after();
         }
         {
-            const int cq0 = (warp / 4) * 32;       // d = 64: the upper two warpgroups have no columns
-            const int jc = jg < n ? jg : 0;
-            for (int cq = cq0; cq < cq0 + 32 && cq < HD; cq += 32) {
-                __nv_bfloat16 *pv = a.dV + ((size_t)bh * n + jc) * HD + cq;
-                __nv_bfloat16 *pk = a.dK + ((size_t)bh * n + jc) * HD + cq;
+            // dV_j and dK_j go out through shared memory and TMA stores (coalesced; rows beyond n are clipped): the
+            // first Q and dO stages are free by now -- every product that read them has completed.  Each thread packs
+            // 32 columns of its key row into the swizzled slab layout the store expects.
+            const int cq = (warp / 4) * 32;        // d = 64: the upper two warpgroups have no columns
+            if (cq < HD) {
 #pragma unroll
                 for (int which = 0; which < 2; ++which) {
                     uint32_t v[32];
@@ -887,17 +888,26 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
 #pragma unroll
                         for (int e = 0; e < 32; ++e) v[e] = 0u;
                     }
-                    __nv_bfloat16 *po = which == 0 ? pv : pk;
-                    if (jg < n) {
+                    uint8_t *slab = smem + (which == 0 ? L::oQ : L::odO) + (cq / 64) * SLAB;
 #pragma unroll
-                        for (int e = 0; e < 32; e += 8)
-                            *reinterpret_cast<uint4 *>(po + e) =
-                                make_uint4(pack_bf16(__uint_as_float(v[e]), __uint_as_float(v[e + 1])),
-                                           pack_bf16(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3])),
-                                           pack_bf16(__uint_as_float(v[e + 4]), __uint_as_float(v[e + 5])),
-                                           pack_bf16(__uint_as_float(v[e + 6]), __uint_as_float(v[e + 7])));
-                    }
+                    for (int e = 0; e < 32; e += 8)
+                        *reinterpret_cast<uint4 *>(slab + sw128_offset(row, (cq % 64) + e)) =
+                            make_uint4(pack_bf16(__uint_as_float(v[e]), __uint_as_float(v[e + 1])),
+                                       pack_bf16(__uint_as_float(v[e + 2]), __uint_as_float(v[e + 3])),
+                                       pack_bf16(__uint_as_float(v[e + 4]), __uint_as_float(v[e + 5])),
+                                       pack_bf16(__uint_as_float(v[e + 6]), __uint_as_float(v[e + 7])));
                 }
+            }
+            fence_proxy_async_smem();
+            asm volatile("bar.sync 1, 512;" ::: "memory");   // the sixteen exp / dS warps
+            if (tid == 0) {
+#pragma unroll
+                for (uint32_t sl = 0; sl < L::kSlabs; ++sl) {
+                    tma_store_3d(&mdV, smem + L::oQ + sl * SLAB, sl * 64, j0, (int)bh);
+                    tma_store_3d(&mdK, smem + L::odO + sl * SLAB, sl * 64, j0, (int)bh);
+                }
+                tma_store_commit();
+                tma_store_wait_read();   // the slabs have been read; the writes complete with the grid
             }
         }
     }
@@ -960,7 +970,9 @@ attn_status launch_bwd(const Problem &p)
         constexpr uint32_t bytes = HD == 64 ? ((L::kBytes + 1023u) & ~1023u) + SLAB : L::kBytes;
         if (cudaFuncSetAttribute(tc_bwd_fused_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
             return ATTN_ERR_LAUNCH;
-        tc_bwd_fused_kernel<HD><<<grid, kThreadsFused, bytes, p.stream>>>(mQ, mK, mV, mdO, a);
+        CUtensorMap mdK, mdV;
+        if (!make_tmap_bf16_3d(&mdK, p.dK, HD, p.n, BH, 128) || !make_tmap_bf16_3d(&mdV, p.dV, HD, p.n, BH, 128)) return ATTN_ERR_LAUNCH;
+        tc_bwd_fused_kernel<HD><<<grid, kThreadsFused, bytes, p.stream>>>(mQ, mK, mV, mdO, mdK, mdV, a);
     } else {
         if (cudaFuncSetAttribute(tc_bwd_dkdv_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DkdvSmem<HD>::kBytes) != cudaSuccess)
             return ATTN_ERR_LAUNCH;
