@@ -165,7 +165,7 @@ size_t attn_weights_bwd_workspace_bytes(int n, int d, int heads, int batch, cons
  *
  * Who needs it: code that is handed Q, K, V, O, dO, LSE and the output tensors but has
  * no allocator it may call at that moment -- a plug-in inside a framework whose memory
- * pool is frozen, a host callback, a real-time loop that must not call cudaMalloc.
+ * pool is frozen, a real-time loop that must not call cudaMalloc.
  * Such a caller cannot provide attn_bwd's `workspace`.  This entry point uses instead a
  * fixed scratch array of attn_noalloc_scratch_bytes() = 8 MiB that is part of the
  * library image (every GPU that loads the library holds these 8 MiB until the process
@@ -180,13 +180,15 @@ size_t attn_weights_bwd_workspace_bytes(int n, int d, int heads, int batch, cons
  *  - All calls on a device share the one array and it keeps the previous call's
  *    contents; the parts that must start at zero are cleared by every call.  Two calls
  *    that overlap on the GPU (different streams, no ordering) race on it: serialise them.
- *  - Device-side errors land in the array's first word; there is no way to read it from
- *    outside, so use attn_bwd when you need attn_workspace_status(). */
+ *  - Device-side errors (a bounded wait that ran out) land in the array's first word:
+ *    attn_noalloc_status() synchronises `cuda_stream` and returns it, like
+ *    attn_workspace_status() does for a caller-owned workspace; it allocates nothing either. */
 attn_status attn_bwd_noalloc(const void *Q, const void *K, const void *V, const void *O, const void *dO,
                              const float *LSE, void *dQ, void *dK, void *dV,
                              int n, int d, int heads, int batch, const attn_mask *mask,
                              int dt, float scale, const attn_cfg *cfg, void *cuda_stream);
 size_t attn_noalloc_scratch_bytes(void);
+attn_status attn_noalloc_status(void *cuda_stream);
 
 /* Workspace sizes in bytes for the same arguments (0 on invalid arguments). */
 size_t attn_fwd_workspace_bytes(int n, int d, int heads, int batch, const attn_mask *mask, int dt,
@@ -229,6 +231,17 @@ const char *attn_status_str(int status);
 unsigned long long attn_kernel_launches(void);
 attn_status attn_timing_enable(int on);
 int attn_timing_collect(float *ms /* host */, const char **names /* host */, int max);
+
+/* Self-test of the bounded waits (no counterpart in the paper): every wait inside the
+ * tensor-core kernels gives up after a time limit, sets the workspace status word to
+ * ATTN_ERR_DEVICE_TIMEOUT and lets the kernel run to its normal end.  This call enqueues
+ * one warp that waits, for at most `limit_us` microseconds (1 .. 100000), on a barrier
+ * nothing arrives at; afterwards attn_workspace_status(workspace) is
+ * ATTN_ERR_DEVICE_TIMEOUT and the context is as usable as before.  workspace: device,
+ * at least 256 bytes; its first two words are overwritten (word 1: bit 0 / bit 1 set if
+ * the first / second wait wrongly reported success). */
+attn_status attn_selftest_wait_timeout(void *workspace, size_t workspace_bytes, unsigned limit_us,
+                                       void *cuda_stream);
 
 #ifdef __cplusplus
 }

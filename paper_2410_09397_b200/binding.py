@@ -27,7 +27,8 @@ EXPORTS = (
     "attn_fwd", "attn_bwd", "attn_bwd_preprocess", "attn_fwd_workspace_bytes", "attn_bwd_workspace_bytes",
     "attn_workspace_status", "attn_supported_cfgs", "attn_cfg_onchip_elems", "attn_io_bound_elems",
     "attn_io_bound_sparse_elems", "attn_status_str", "attn_kernel_launches", "attn_timing_enable",
-    "attn_timing_collect", "attn_bwd_noalloc", "attn_noalloc_scratch_bytes",
+    "attn_timing_collect", "attn_bwd_noalloc", "attn_noalloc_scratch_bytes", "attn_noalloc_status",
+    "attn_selftest_wait_timeout",
     "attn_project", "attn_weight_grad", "attn_weights_bwd", "attn_weights_bwd_workspace_bytes",
 )
 
@@ -97,6 +98,10 @@ def lib() -> ctypes.CDLL:
     L.attn_bwd_noalloc.argtypes = [vp] * 9 + [ci, ci, ci, ci, ctypes.POINTER(CMask), ci, cf, ctypes.POINTER(CCfg), vp]
     L.attn_noalloc_scratch_bytes.restype = sz
     L.attn_noalloc_scratch_bytes.argtypes = []
+    L.attn_noalloc_status.restype = ci
+    L.attn_noalloc_status.argtypes = [vp]
+    L.attn_selftest_wait_timeout.restype = ci
+    L.attn_selftest_wait_timeout.argtypes = [vp, sz, ctypes.c_uint, vp]
     L.attn_bwd_preprocess.restype = ci
     L.attn_bwd_preprocess.argtypes = [vp, vp, vp, sz, ci, ci, vp]
     for f in (L.attn_fwd_workspace_bytes, L.attn_bwd_workspace_bytes):
@@ -332,6 +337,19 @@ def attn_timing_collect(max_entries: int = 256) -> list[tuple[str, float]]:
 
 def attn_noalloc_scratch_bytes() -> int:
     return int(lib().attn_noalloc_scratch_bytes())
+
+
+def attn_noalloc_status() -> int:
+    """Synchronises the current stream; status word of the last ``attn_bwd_noalloc`` on this device."""
+    return int(lib().attn_noalloc_status(_stream()))
+
+
+def attn_selftest_wait_timeout(workspace, limit_us: int = 2000) -> None:
+    """Enqueues the bounded-wait self-test: afterwards ``attn_workspace_status(workspace)`` is
+    ``ATTN_ERR_DEVICE_TIMEOUT``.  ``workspace``: CUDA uint8 tensor of at least 256 bytes."""
+    st = lib().attn_selftest_wait_timeout(workspace.data_ptr(), workspace.numel(), limit_us, _stream())
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_selftest_wait_timeout")
 
 
 def attn_bwd_noalloc(Q, K, V, O, dO, LSE, dQ, dK, dV, *, mask: Mask | None = None, scale: float = 0.0,

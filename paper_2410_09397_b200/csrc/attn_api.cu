@@ -134,6 +134,19 @@ attn_status check_arch()
     return major == 10 ? ATTN_OK : ATTN_ERR_ARCH;
 }
 
+}  // namespace
+
+int sm_count()
+{
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        return 1;
+    return sms;
+}
+
+namespace {
+
 attn_status fill_problem(Problem &p, const Args &a, int backward, float scale, void *workspace, size_t workspace_bytes,
                          void *stream)
 {

@@ -45,6 +45,9 @@ void launch_end(cudaStream_t s);
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Streaming multiprocessors of the current device (grid sizing of the grid-stride and persistent kernels).
+int sm_count();
+
 // SIMT fp32 path (attn_simt.cu)
 attn_status simt_fwd(const Problem &p);
 attn_status simt_bwd(const Problem &p);

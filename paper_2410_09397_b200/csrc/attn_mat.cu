@@ -276,7 +276,8 @@ attn_status run_chunk(const Problem &p, size_t h0, int mh)
     // phase 3: dS = scale P o (dP - D)
     {
         const size_t nvec = (size_t)mh * n * n / 8;
-        const unsigned blocks = (unsigned)((nvec + 255) / 256 < 148 * 16 ? (nvec + 255) / 256 : 148 * 16);
+        const size_t cap = (size_t)sm_count() * 16;
+        const unsigned blocks = (unsigned)((nvec + 255) / 256 < cap ? (nvec + 255) / 256 : cap);
         launch_begin("mat_phase3_dS", p.stream);
         mat_ds_kernel<<<blocks, 256, 0, p.stream>>>((const uint4 *)p.matP, (const uint4 *)p.matdP, (uint4 *)p.matdS,
                                                     p.D + h0 * n, nvec, n, p.scale);
@@ -339,7 +340,7 @@ attn_status mat_bwd(const Problem &p)
     if (p.mask_kind == ATTN_MASK_BLOCK_SPARSE) return ATTN_ERR_MASK;
     const size_t rows = (size_t)p.BH * p.n;
     size_t blocks = (rows + 7) / 8;
-    if (blocks > 148 * 8) blocks = 148 * 8;
+    if (blocks > (size_t)sm_count() * 8) blocks = (size_t)sm_count() * 8;
     launch_begin("mat_preprocess", p.stream);
     mat_preprocess_kernel<<<(unsigned)blocks, 256, 0, p.stream>>>((const __nv_bfloat16 *)p.O, (const __nv_bfloat16 *)p.dO,
                                                                   p.LSE, p.D, p.nLSE2, rows, p.d, p.scale);

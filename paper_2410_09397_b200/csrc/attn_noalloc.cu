@@ -3,8 +3,8 @@
 // attn_bwd needs scratch memory (the status word, D = rowsum(dO o O) and, for the fused
 // algorithm, the fp32 dQ accumulator) and asks its caller to pass it in.  Some callers
 // have no way to get such a buffer at the moment of the call: code running inside a
-// region where cudaMalloc is forbidden (a memory pool that has been frozen, a host
-// callback, a plug-in that was handed tensors but no allocator).  For them the scratch
+// region where cudaMalloc is forbidden (a memory pool that has been frozen, a real-time
+// loop, a plug-in that was handed tensors but no allocator).  For them the scratch
 // lives here, in a fixed array that is part of the library image.
 #include "attn_internal.h"
 
@@ -38,6 +38,16 @@ attn_status scratch_for_current_device(void **out)
 extern "C" {
 
 size_t attn_noalloc_scratch_bytes(void) { return kScratchBytes; }
+
+// The status word of the last attn_bwd_noalloc call on the current device is the first word of the
+// array: copied out with a plain device-to-host copy (no allocation), after `cuda_stream` has drained.
+attn_status attn_noalloc_status(void *cuda_stream)
+{
+    void *scratch = nullptr;
+    const attn_status st = scratch_for_current_device(&scratch);
+    if (st != ATTN_OK) return st;
+    return attn_workspace_status(scratch, cuda_stream);
+}
 
 attn_status attn_bwd_noalloc(const void *Q, const void *K, const void *V, const void *O, const void *dO,
                              const float *LSE, void *dQ, void *dK, void *dV, int n, int d, int heads, int batch,

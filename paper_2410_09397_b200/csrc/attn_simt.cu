@@ -570,7 +570,7 @@ attn_status preprocess_D(const void *O, const void *dO, float *D, size_t rows, i
     const size_t rows_per_warp = 32 / lanes;
     const size_t warps = (rows + rows_per_warp - 1) / rows_per_warp;
     size_t blocks = (warps + 7) / 8;
-    const size_t cap = 148 * 8;      // eight resident CTAs of 256 threads per SM, grid-stride beyond that
+    const size_t cap = (size_t)sm_count() * 8;      // eight resident CTAs of 256 threads per SM, grid-stride beyond that
     if (blocks > cap) blocks = cap;
     launch_begin("bwd_preprocess_D", s);
     if (dt == ATTN_F32)

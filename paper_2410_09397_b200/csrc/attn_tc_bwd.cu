@@ -293,6 +293,9 @@ tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
                     tma_load_3d(smem + L::odO + s2 * L::kTile + sl * SLAB, &mdO, &bars[KD_OFULL + s2], sl * 64, i0, (int)bh);
                 ++k;
             }
+            // a key tile without a single query tile (an empty block column): nobody else waits for K_j and V_j, and
+            // the CTA must not exit with their bulk loads still in flight into its shared memory
+            if (k == 0) mbar_wait(&bars[KD_KV], 0, ab);
         }
     } else if (warp == 16) {
         // ------------------------------------------------------------ MMA issuer A: the products into region A
@@ -525,8 +528,8 @@ tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
 // product into A runs while the exponentials (or the dS arithmetic) are still being computed:
 //
 //   issuer A:  dP^T(k) -> A  (once S^T(k) has been copied out)  |  S^T(k+1) -> A  (once dP^T(k) has been)
-//   issuer B:  dV += P^T(k) dO  (P^T(k) written in B)  |  dQ^T(k) -> B, dK += dS^T(k) Q  (dS^T(k) in shared
-//              memory, the reducers done with dQ^T(k-1))
+//   issuer B:  dV += P^T(k) dO  (P^T(k) written in B)  |  dK += dS^T(k) Q, dQ^T(k) -> B  (dS^T(k) in shared
+//              memory, the reducers done with dQ^T(k-1)); dK goes first because it releases the Q / dO stage
 //
 // The exp / dS warps keep P only as the bf16 pairs they hand to the dV product, and form dS from
 // those.  Registers are traded between the warpgroups after launch (setmaxnreg).
@@ -633,6 +636,9 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
                 issue_load(it, s);
                 ++k;
             }
+            // a key tile without a single query tile (an empty block column): nobody else waits for K_j and V_j, and
+            // the CTA must not exit with their bulk loads still in flight into its shared memory
+            if (k == 0) mbar_wait(&bars[V2_KV], 0, ab);
         } else if (warp == 24 && lane == 0) {
             // ------------------------------------------------------------ MMA issuer A: the products into region A (S^T, dP^T)
             constexpr uint32_t idesc_s = idesc_bf16(128, 128, 0, 0);
@@ -664,9 +670,6 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
                 while (nidx < iter.raw && (nit = iter.tile(nidx)) < 0) ++nidx;
                 const uint32_t kdO = desc_lo_kmajor(smem_u32(smem + L::odO + s * L::kTile));
                 // dP^T = V_j dO_i^T into region A once every exp / dS warp holds its part of S^T in registers
-                if (k > 0) {   // see the exp / dS warps: P^T of this tile is stored once dP^T has been seen
-                    mbar_wait(&bars[V2_DQREL], (k - 1) & 1, ab);
-                }
                 mbar_wait(&bars[V2_SLD], k & 1, ab);
                 tcgen05_fence_after();
 #pragma unroll
@@ -712,21 +715,22 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
                     for (int kk = 0; kk < 4; ++kk)
                         mma_ts_lo(T_dV, T_B + 64 * h + kk * 8, mdO_ + h * kHalf + kk * 128, idesc_dv, (k > 0) || (h > 0) || (kk > 0));
                 }
-                // dQ^T = K_j^T dS^T into region B (this thread's products execute in issue order, so dV has
-                // consumed P^T by then); the reducer warps read it out while dK += dS^T Q_i runs
+                // dK += dS^T Q_i first: its completion releases the Q / dO stage, and the load of the tile after next --
+                // two stages only -- is what the next S^T product ends up waiting for.  Then dQ^T = K_j^T dS^T into
+                // region B (this thread's products execute in issue order, so dV has consumed P^T by then)
                 mbar_wait(&bars[V2_DS], k & 1, ab);
                 if (k > 0) {   // the reducers have read all of the previous dQ^T
                     mbar_wait(&bars[V2_DQDONE], (k - 1) & 1, ab);
                 }
                 tcgen05_fence_after();
 #pragma unroll
-                for (int kk = 0; kk < TK / 16; ++kk)
-                    mma_ss_lo(T_B, mK + kk * 128, mdS + kk * 128, idesc_dq, kk > 0);
-                mma_commit(&bars[V2_DQ]);
-#pragma unroll
                 for (int kk = 0; kk < TQ / 16; ++kk)
                     mma_ss_lo(T_dK, kdS + (kk / 4) * kSlab + (kk % 4) * 2, mQ_ + kk * 128, idesc_dv, (k > 0) || (kk > 0));
                 mma_commit(&bars[V2_QEMPTY + s]);
+#pragma unroll
+                for (int kk = 0; kk < TK / 16; ++kk)
+                    mma_ss_lo(T_B, mK + kk * 128, mdS + kk * 128, idesc_dq, kk > 0);
+                mma_commit(&bars[V2_DQ]);
                 ++k;
             }
         }
@@ -791,6 +795,11 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
             const bool masked = diag || i0 + TQ > n || j0 + TK > n;
             const int ig0 = i0 + h * 64 + qq * 32;
             mbar_wait(&bars[V2_QFULL + s], (k >> 1) & 1, ab);
+            // the 32 row statistics of this thread's query columns go into registers before the wait for S^T: while the
+            // products stream their operands, a shared-memory load inside the arithmetic below waits a few hundred cycles
+            float4 nlr[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) nlr[q] = sNL[q];
             mbar_wait(&bars[V2_S], k & 1, ab);
             tcgen05_fence_after();
             uint32_t ppack[16];   // P as bf16 pairs: what dV uses, and what dS is formed from
@@ -802,7 +811,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
                 warp_arrive(&bars[V2_SLD], lane);   // region A may take dP^T
 #pragma unroll
                 for (int q = 0; q < 8; ++q) {
-                    const float4 nl = sNL[q];
+                    const float4 nl = nlr[q];
                     float p[4];
                     p[0] = ex2_approx(fmaf(__uint_as_float(sv[q * 4 + 0]), sl2, nl.x));
                     p[1] = ex2_approx(fmaf(__uint_as_float(sv[q * 4 + 1]), sl2, nl.y));
@@ -820,8 +829,17 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
                     ppack[q * 2 + 1] = pack_bf16(p[2], p[3]);
                 }
             }
-            // dP^T first: copying it out lets S^T of the next tile start.  Its issuer has also seen the reducers
-            // take the previous dQ^T out of the first 32 columns of both halves of region B, where P^T goes
+            float4 dsr[8];   // scale * D of the same columns, again ahead of the wait
+#pragma unroll
+            for (int q = 0; q < 8; ++q) dsr[q] = sDs[q];
+            // P^T goes into region B before dP^T is awaited: a tensor-memory store issued while products run takes
+            // several hundred cycles, which now pass during that wait.  Its first 32 columns per half held dQ^T of the
+            // previous tile; the reducers release them after their first load
+            if (k > 0) {
+                mbar_wait(&bars[V2_DQREL], (k - 1) & 1, ab);
+                tcgen05_fence_after();
+            }
+            tmem_st16(T_B + lane_addr + cP, ppack);
             mbar_wait(&bars[V2_DP], k & 1, ab);
             tcgen05_fence_after();
             {
@@ -831,10 +849,12 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
                 tmem_wait_ld();
                 tcgen05_fence_before();
                 warp_arrive(&bars[V2_DPLD], lane);   // region A may take the next S^T
-                tmem_st16(T_B + lane_addr + cP, ppack);
                 tmem_wait_st();
                 tcgen05_fence_before();
                 warp_arrive(&bars[V2_P + h], lane);
+                // dS^T(k) goes over dS^T(k-1), which the dK and dQ^T products of tile k-1 read from shared memory.  Both
+                // have completed: the reducers release their columns (awaited above) only after dQ^T(k-1), the later of
+                // the two in the other thread's issue order, has landed
 #pragma unroll
                 for (int g = 0; g < 4; ++g) {    // 8 query columns = one 16-byte chunk
                     float ds[8], p[8];
@@ -846,7 +866,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
                     }
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {
-                        const float4 dsc = sDs[g * 2 + u];
+                        const float4 dsc = dsr[g * 2 + u];
                         const uint32_t *d4 = &dv[g * 8 + u * 4];
                         ds[u * 4 + 0] = p[u * 4 + 0] * fmaf(__uint_as_float(d4[0]), a.scale, -dsc.x);
                         ds[u * 4 + 1] = p[u * 4 + 1] * fmaf(__uint_as_float(d4[1]), a.scale, -dsc.y);
@@ -868,7 +888,8 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
         }
         // ------------------------------------------------------------ epilogue: dV_j, dK_j (32 columns per warpgroup)
         if (k > 0) {
-            // the last tile's dK product is the last thing the issuer queued before this commit
+            // dV and dK of the last tile have completed when its stage is released (dQ^T, queued after them, is the
+            // reducers' business and reads neither accumulator nor the stages reused below)
             mbar_wait(&bars[V2_QEMPTY + ((k - 1) & 1)], ((k - 1) >> 1) & 1, ab);
             tcgen05_fence_after();
         }
@@ -956,7 +977,7 @@ attn_status launch_bwd(const Problem &p)
         const size_t rows = (size_t)p.BH * p.n;
         constexpr size_t rpw = 32 / (HD / 8);
         size_t blocks = ((rows + rpw - 1) / rpw + 7) / 8;
-        if (blocks > 148 * 8) blocks = 148 * 8;
+        if (blocks > (size_t)sm_count() * 8) blocks = (size_t)sm_count() * 8;
         launch_begin("tc_bwd_preprocess", p.stream);
         tc_preprocess_kernel<HD><<<(unsigned)blocks, 256, 0, p.stream>>>((const __nv_bfloat16 *)p.O, (const __nv_bfloat16 *)p.dO,
                                                                          p.LSE, p.D, p.nLSE2, rows, p.scale,
@@ -982,7 +1003,8 @@ attn_status launch_bwd(const Problem &p)
     if (cudaGetLastError() != cudaSuccess) return ATTN_ERR_LAUNCH;
     if (!WITH_DQ) return tc_bwd_dq(p);   // deterministic path: dQ without atomics, from its own kernel
     const size_t n4 = acc_elems / 4;
-    const unsigned blocks = (unsigned)((n4 + 255) / 256 < 148 * 16 ? (n4 + 255) / 256 : 148 * 16);
+    const size_t cap = (size_t)sm_count() * 16;
+    const unsigned blocks = (unsigned)((n4 + 255) / 256 < cap ? (n4 + 255) / 256 : cap);
     launch_begin("bwd_dq_convert", p.stream);
     dq_convert_kernel<<<blocks, 256, 0, p.stream>>>((const float4 *)p.dQ_acc, (uint2 *)p.dQ, n4);
     launch_end(p.stream);

@@ -1,22 +1,24 @@
 // Fused forward for bf16 on the 5th-generation tensor cores: O = softmax(scale Q K^T) V
 // and LSE, never writing a score tile to device memory (Definition 3.1; large-cache
-// tiling: row block of 128 queries stays on chip, key/value blocks stream through).
+// tiling: a row block of 128 queries stays on chip, key/value blocks stream through).
 //
-// A CTA owns one tile of 128 queries (tensor-memory lane = query row) and walks the
-// kept key tiles j of TKF keys (128 for d <= 128, 64 for d = 256):
+// A CTA owns one tile of 128 queries (tensor-memory lane = query row) and walks the kept
+// key tiles j:
 //
-//   S   = Q_i K_j^T                 tcgen05.mma, operands K-major in shared memory,
-//                                   two S buffers in tensor memory so that S(j+1) is
-//                                   computed while the softmax of S(j) runs
+//   S   = Q_i K_j^T                  tcgen05.mma, operands K-major in shared memory
 //   m, l running row maximum / row sum in the exp2 domain; the reference maximum is
 //       only moved (and O rescaled in tensor memory) when the tile maximum exceeds it
 //       by more than 2^8 -- the final LSE does not depend on which reference was used
 //   P   = exp2(S * scale*log2e - m)  -> bf16, written over S in tensor memory
 //   O  += P V_j                      A = P from tensor memory, B = V_j MN-major
 //
-// Roles: warps 0-7 = two warpgroups that split the key columns of every tile (row
-// maxima are exchanged through shared memory), warp 8 lane 0 = MMA issuer, warp 9
-// lane 0 = TMA producer.  Tensor memory: S0 128, S1 128, O d columns.
+// Two kernels.  tc_fwd_rows_kernel (d = 64, 128; key tiles of 128): the two softmax
+// warpgroups take alternate key tiles, each with an S buffer and a partial accumulator of
+// its own, a thread holds a whole row of scores, and the two partial softmaxes are merged
+// in the epilogue.  tc_fwd_kernel (d = 256; key tiles of 64): both warpgroups split the
+// columns of every tile and exchange row maxima through shared memory, one accumulator of
+// 256 columns.  Each has one MMA-issuing thread and one TMA-producing thread; the roles and
+// the tensor-memory layout are described at each kernel.
 #include "attn_internal.h"
 #include "tc_common.cuh"
 
@@ -610,8 +612,9 @@ attn_status launch_fwd(const Problem &p)
     a.row_ptr = p.row_ptr; a.col_idx = p.col_idx;
     a.scale = p.scale;
     a.status = p.status;
-    auto kernel = tc_fwd_kernel<HD>;
-    if constexpr (HD != 256) kernel = tc_fwd_rows_kernel<HD>;
+    void (*kernel)(CUtensorMap, CUtensorMap, CUtensorMap, FwdArgs);
+    if constexpr (HD == 256) kernel = tc_fwd_kernel<HD>;
+    else kernel = tc_fwd_rows_kernel<HD>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kBytes) != cudaSuccess)
         return ATTN_ERR_LAUNCH;
     const dim3 grid((p.n + TQ - 1) / TQ, (unsigned)p.BH);

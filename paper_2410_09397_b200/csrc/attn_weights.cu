@@ -524,14 +524,6 @@ attn_status check_arch()
     return major == 10 ? ATTN_OK : ATTN_ERR_ARCH;
 }
 
-int sm_count()
-{
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-        return 148;
-    return sms > 0 ? sms : 148;
-}
-
 attn_status check_common(int n, int d, int heads, int batch, int weight_units, int dt, const void *workspace,
                          size_t workspace_bytes)
 {
@@ -619,7 +611,7 @@ attn_status launch_simt_project(const void *A, const void *W, void *out, int n, 
 {
     const size_t total = (size_t)BH * n * d;
     size_t blocks = (total + 255) / 256;
-    if (blocks > 148 * 16) blocks = 148 * 16;
+    if (blocks > (size_t)sm_count() * 16) blocks = (size_t)sm_count() * 16;
     launch_begin("wproj_simt", s);
     simt_project_kernel<T><<<(unsigned)blocks, 256, 0, s>>>((const T *)A, (const T *)W, (T *)out, total, n, d, wu);
     launch_end(s);

@@ -2,7 +2,7 @@
 // waits, TMA tile loads, tensor-memory (TMEM) allocation and access, tcgen05.mma issue,
 // and the shared-memory / instruction descriptors.  Inline PTX only.
 //
-// Waiting never blocks for ever: every wait polls for at most kWaitNs nanoseconds, then
+// Waiting never blocks for ever: every wait polls for at most Abort::limit_ns (kWaitNs) nanoseconds, then
 // raises the CTA's abort flag and the global status word and returns false.  After an
 // abort all later waits of the CTA return at once, the kernel runs to its normal end
 // (its results are then meaningless, and the caller sees ATTN_ERR_DEVICE_TIMEOUT), TMEM
@@ -57,10 +57,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
     return ok != 0;
 }
 
-// Per-CTA abort state: `flag` lives in shared memory, `status` is the workspace word.
+// Per-CTA abort state: `flag` lives in shared memory, `status` is the workspace word, `limit_ns` is how
+// long one wait may poll (the kernels of the library leave it at kWaitNs).
 struct Abort {
     volatile uint32_t *flag;
     uint32_t *status;
+    unsigned long long limit_ns = kWaitNs;
 };
 
 // Returns true when the phase with the given parity has completed.
@@ -73,7 +75,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, const 
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 63u) == 0) {
             if (*ab.flag) return false;
-            if (globaltimer() - t0 > kWaitNs) {
+            if (globaltimer() - t0 > ab.limit_ns) {
                 *ab.flag = 1u;
                 atomicExch(ab.status, 10u);   // ATTN_ERR_DEVICE_TIMEOUT
                 return false;
