@@ -520,13 +520,13 @@ def main():
         share = {k: round(v / sum(tot.values()), 4) for k, v in tot.items()}
         # FLOPs one launch of each kernel executes, as a share of the forward (F) / backward (B) algorithmic
         # count: the backward's five products are 0.2 B each; the split kernels recompute S and dP
-        own = {"tc_fwd": ("F", 1.0), "simt_fwd": ("F", 1.0), "tc_bwd_fused": ("B", 1.0),
+        own = {"tc_fwd": ("F", 1.0), "simt_fwd": ("F", 1.0), "tc_bwd_fused": ("B", 1.0), "tc_bwd_fused64": ("B", 1.0),
                "tc_bwd_dkdv": ("B", 0.8), "tc_bwd_dq": ("B", 0.6), "simt_bwd_dkdv": ("B", 0.8), "simt_bwd_dq": ("B", 0.6),
                "mat_phase1_P": ("B", 0.2), "mat_phase2_dP": ("B", 0.2), "mat_phase4_dV": ("B", 0.2),
                "mat_phase4_dK": ("B", 0.2), "mat_phase4_dQ": ("B", 0.2)}
         which, share_ = own.get(top, ("B", 1.0))
         alg = (ff if which == "F" else fb) * share_
-        note = ("algorithmic FLOPs of the five backward products" if top == "tc_bwd_fused" else
+        note = ("algorithmic FLOPs of the five backward products" if top in ("tc_bwd_fused", "tc_bwd_fused64") else
                 f"this kernel's own products: {share_:g} x the {'forward' if which == 'F' else 'backward'} count")
         ach = alg / (avg_ms * 1e-3) / 1e12
         roofline = {"bound": "tensor", "kernel": top, "achieved": ach, "peak": peaks["bf16_tflops_sustained"],

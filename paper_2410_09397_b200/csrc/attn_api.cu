@@ -39,6 +39,11 @@ attn_status resolve_cfg(const Args &a, int backward, attn_cfg *out)
         c.algo = ATTN_ALGO_FUSED;
         c.tile_q = c.tile_k = c.tile_d = 0;
     }
+    // a configuration that names a backward tile shape may be handed to the forward as well (one cfg for a
+    // forward / backward pair): the forward then runs with its own tiles
+    if (c.algo == ATTN_ALGO_FUSED && !backward && a.dt == ATTN_BF16 && !tc_cfg_supported(a.d, c, 0) &&
+        tc_cfg_supported(a.d, c, 1))
+        c.tile_q = c.tile_k = c.tile_d = 0;
     if (c.algo == ATTN_ALGO_SIMT) {
         if ((c.tile_q && c.tile_q != 64) || (c.tile_k && c.tile_k != 64) || (c.tile_d && c.tile_d != 64))
             return ATTN_ERR_TILE;
@@ -55,6 +60,9 @@ attn_status resolve_cfg(const Args &a, int backward, attn_cfg *out)
         const int cnt = attn_supported_cfgs(a.d, a.dt, list, 32);
         for (int i = 0; i < cnt; ++i) {
             if (list[i].algo != c.algo) continue;
+            attn_cfg cand = list[i];
+            cand.deterministic = c.deterministic;
+            if (!tc_cfg_supported(a.d, cand, backward)) continue;
             if ((c.tile_q == 0 || c.tile_q == list[i].tile_q) && (c.tile_k == 0 || c.tile_k == list[i].tile_k) &&
                 (c.tile_d == 0 || c.tile_d == list[i].tile_d)) {
                 c.tile_q = list[i].tile_q; c.tile_k = list[i].tile_k; c.tile_d = list[i].tile_d;
@@ -312,6 +320,7 @@ int attn_supported_cfgs(int d, int dt, attn_cfg *out, int max_out)
         const int tiles[][4] = {
             {128, 128, 0, ATTN_ALGO_FUSED},
             {128, 64, 0, ATTN_ALGO_FUSED},
+            {64, 128, 0, ATTN_ALGO_FUSED},
             {128, 128, 64, ATTN_ALGO_MATERIALIZED},
             {128, 64, 64, ATTN_ALGO_MATERIALIZED},
             {128, 32, 64, ATTN_ALGO_MATERIALIZED},

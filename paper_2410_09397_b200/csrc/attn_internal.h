@@ -63,6 +63,8 @@ bool tc_cfg_supported(int d, const attn_cfg &cfg, int backward);
 size_t tc_cfg_onchip_bytes(int d, const attn_cfg &cfg, int backward);
 size_t fwd_smem_bytes(int d);
 size_t bwd_smem_bytes(int d);
+size_t bwd64_smem_bytes(int d);            // fused backward with 64-query tiles
+attn_status tc_bwd64(const Problem &p);
 bool mat_cfg_supported(int d, const attn_cfg &cfg);
 size_t mat_onchip_bytes(int d, const attn_cfg &cfg);
 

@@ -27,28 +27,15 @@
 // (without the dQ product; `deterministic = 1` pairs it with the query-stationary dQ kernel of
 // attn_tc_bwd_dq.cu).  Warp roles are described at each kernel.  All waits are bounded
 // (tc_common.cuh).
-#include "attn_internal.h"
-#include "tc_common.cuh"
+#include "tc_bwd_common.cuh"
 
 namespace attn {
 namespace {
 
 using namespace tc;
+using namespace bwdk;
 
-constexpr int TQ = 128, TK = 128;
-constexpr uint32_t SLAB = 128 * 128;   // bytes of one [128 rows][64 bf16] slab
-struct BwdArgs {
-    const float *nLSE2, *Ds;   // -LSE log2(e) and scale * D per row (workspace)
-    float *dQ_acc;
-    __nv_bfloat16 *dK, *dV;
-    int n, BH;
-    int mask_kind, block, nb, mask_heads;
-    const int *col_ptr, *row_idx;   // block-CSC of the mask
-    float scale;
-    int group;                 // heads per launch group (divides BH)
-    uint32_t *status;
-};
-
+constexpr int TQ = 128;
 template <int HD>
 struct BwdSmem {
     static constexpr uint32_t kSlabs = HD / 64;
@@ -67,119 +54,12 @@ struct BwdSmem {
 };
 
 
-struct TileIter {
-    // Enumerates the query tiles a key tile jt has to visit.
-    int kind, n, jt, sub, raw;
-    const int *rows;   // block rows kept in this block column
-    __device__ TileIter(const BwdArgs &a, int jt_, long bh) : kind(a.mask_kind), n(a.n), jt(jt_), sub(1), raw(0), rows(nullptr)
-    {
-        const int nt = (n + TQ - 1) / TQ;
-        if (kind == ATTN_MASK_NONE) raw = nt;
-        else if (kind == ATTN_MASK_CAUSAL) raw = nt - jt;
-        else {
-            sub = a.block / TQ;
-            const int J = jt / sub;
-            const long mh = a.mask_heads == 1 ? 0 : bh;
-            const int *cp = a.col_ptr + mh * 2 * a.nb + 2 * J;
-            rows = a.row_idx + mh * (long)a.nb * a.nb + cp[0];
-            raw = (cp[1] - cp[0]) * sub;
-        }
-    }
-    // query tile of raw index idx, or -1 if that tile lies beyond n
-    __device__ int tile(int idx) const
-    {
-        int it;
-        if (kind == ATTN_MASK_NONE) it = idx;
-        else if (kind == ATTN_MASK_CAUSAL) it = jt + idx;
-        else it = rows[idx / sub] * sub + idx % sub;
-        return it * TQ < n ? it : -1;
-    }
-};
-
-__device__ __forceinline__ void bulk_load_1d(void *dst, const void *src, uint32_t bytes, uint64_t *bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(smem_u32(bar))
-                 : "memory");
-}
-__device__ __forceinline__ void red_add_f32(float *p, float v)
-{
-    asm volatile("red.global.add.f32 [%0], %1;" ::"l"(p), "f"(v) : "memory");
-}
-
-__device__ __forceinline__ float ex2_approx(float x)
-{
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-// D pre-pass of the fused backward: Ds_i = scale * sum_c dO_ic O_ic and
-// nlse2_i = -LSE_i * log2(e) (minus infinity for a row with no kept entry, so that its
-// probabilities come out as exactly zero).  16-byte loads, HD/8 lanes share a row.  The same
-// pass clears the fp32 dQ accumulator of the fused backward (`acc`, `acc16` 16-byte words; null =
-// nothing to clear), so that its writes overlap the reads of O and dO.
-template <int HD>
-__global__ void __launch_bounds__(256) tc_preprocess_kernel(const __nv_bfloat16 *__restrict__ O,
-                                                            const __nv_bfloat16 *__restrict__ dO,
-                                                            const float *__restrict__ LSE, float *__restrict__ Ds,
-                                                            float *__restrict__ nlse2, size_t rows, float scale,
-                                                            uint4 *__restrict__ acc, size_t acc16)
-{
-    constexpr int LPR = HD / 8;   // lanes per row
-    constexpr int RPW = 32 / LPR; // rows per warp
-    constexpr int U = 4;          // row groups per step: eight 16-byte loads in flight per lane
-    const int lane = threadIdx.x % 32, sub = lane / LPR, lr = lane % LPR;
-    const size_t warp = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) / 32;
-    const size_t nwarps = (size_t)gridDim.x * blockDim.x / 32;
-    if (acc != nullptr) {
-        for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < acc16; i += (size_t)gridDim.x * blockDim.x)
-            __stcs(acc + i, make_uint4(0u, 0u, 0u, 0u));
-    }
-    for (size_t base = warp * RPW * U; base < rows; base += nwarps * RPW * U) {
-        uint4 xo[U], xg[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const size_t row = base + (size_t)u * RPW + sub;
-            xo[u] = xg[u] = make_uint4(0u, 0u, 0u, 0u);
-            if (row < rows) {
-                xo[u] = __ldcs(reinterpret_cast<const uint4 *>(O + row * HD) + lr);
-                xg[u] = __ldcs(reinterpret_cast<const uint4 *>(dO + row * HD) + lr);
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const size_t row = base + (size_t)u * RPW + sub;
-            const __nv_bfloat162 *eo = reinterpret_cast<const __nv_bfloat162 *>(&xo[u]);
-            const __nv_bfloat162 *eg = reinterpret_cast<const __nv_bfloat162 *>(&xg[u]);
-            float acc = 0.f;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float2 fo = __bfloat1622float2(eo[e]), fg = __bfloat1622float2(eg[e]);
-                acc = fmaf(fo.x, fg.x, acc);
-                acc = fmaf(fo.y, fg.y, acc);
-            }
-#pragma unroll
-            for (int o = LPR / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-            if (row < rows && lr == 0) {
-                Ds[row] = acc * scale;
-                const float l = LSE[row];
-                nlse2[row] = l == -INFINITY ? -INFINITY : -l * 1.4426950408889634f;
-            }
-        }
-    }
-}
+using TileIter = TileIterT<TQ>;
 
 // barrier indices of the fused kernel: every barrier exists once per 64-query half of a tile
 enum { V2_KV = 0, V2_QFULL = 1, V2_QEMPTY = 3, V2_S = 5, V2_DP = 7, V2_P = 9, V2_DS = 11, V2_DQ = 13, V2_DQDONE = 15, V2_SLD = 17,
        V2_DPLD = 19, V2_DQREL = 21 };
 
-// one arrival per warp: every lane has finished (and fenced) its part, lane 0 tells the barrier
-__device__ __forceinline__ void warp_arrive(uint64_t *bar, int lane)
-{
-    __syncwarp();
-    if (lane == 0) mbar_arrive(bar);
-}
 
 // ---------------------------------------------------------------------------------------
 // dK and dV only: the key-stationary half of the path without atomics (dQ comes from the
@@ -963,28 +843,8 @@ attn_status launch_bwd(const Problem &p)
     a.col_ptr = p.col_ptr; a.row_idx = p.row_idx;
     a.scale = p.scale;
     a.status = p.status;
-    // Heads are launched in groups (key tile major inside a group).  The fp32 dQ accumulators of the heads that
-    // run at the same time should stay in L2 between the reductions of one key tile and the next: otherwise every
-    // reduced sector is fetched from and written back to device memory (measured on the block-sparse workload with
-    // n = 32768: 13 times the compulsory traffic with 8 heads in flight).  So the group is the largest of 8, 4, 2,
-    // 1 that divides the head count and whose accumulators take at most kAccBudget bytes.
-    constexpr size_t kAccBudget = 40u << 20;
-    a.group = 1;
-    for (int g = 8; g > 1; g >>= 1)
-        if (p.BH % g == 0 && (size_t)g * p.n * HD * sizeof(float) <= kAccBudget) { a.group = g; break; }
-    const size_t acc_elems = (size_t)p.BH * p.n * HD;
-    {
-        const size_t rows = (size_t)p.BH * p.n;
-        constexpr size_t rpw = 32 / (HD / 8);
-        size_t blocks = ((rows + rpw - 1) / rpw + 7) / 8;
-        if (blocks > (size_t)sm_count() * 8) blocks = (size_t)sm_count() * 8;
-        launch_begin("tc_bwd_preprocess", p.stream);
-        tc_preprocess_kernel<HD><<<(unsigned)blocks, 256, 0, p.stream>>>((const __nv_bfloat16 *)p.O, (const __nv_bfloat16 *)p.dO,
-                                                                         p.LSE, p.D, p.nLSE2, rows, p.scale,
-                                                                         WITH_DQ ? (uint4 *)p.dQ_acc : nullptr, acc_elems / 4);
-        launch_end(p.stream);
-        if (cudaGetLastError() != cudaSuccess) return ATTN_ERR_LAUNCH;
-    }
+    a.group = bwd_head_group(p);
+    if (bwd_preprocess_launch(p, WITH_DQ) != ATTN_OK) return ATTN_ERR_LAUNCH;
     const dim3 grid((unsigned)((p.n + TK - 1) / TK * a.group), (unsigned)(p.BH / a.group));
     launch_begin(WITH_DQ ? "tc_bwd_fused" : "tc_bwd_dkdv", p.stream);
     if (WITH_DQ) {
@@ -1002,7 +862,52 @@ attn_status launch_bwd(const Problem &p)
     launch_end(p.stream);
     if (cudaGetLastError() != cudaSuccess) return ATTN_ERR_LAUNCH;
     if (!WITH_DQ) return tc_bwd_dq(p);   // deterministic path: dQ without atomics, from its own kernel
-    const size_t n4 = acc_elems / 4;
+    return bwd_dq_convert_launch(p);
+}
+
+}  // namespace
+
+// Heads are launched in groups (key tile major inside a group).  The fp32 dQ accumulators of the heads that run
+// at the same time should stay in L2 between the reductions of one key tile and the next: otherwise every reduced
+// sector is fetched from and written back to device memory (measured on the block-sparse workload with n = 32768:
+// 13 times the compulsory traffic with 8 heads in flight).  So the group is the largest of 8, 4, 2, 1 that divides
+// the head count and whose accumulators take at most kAccBudget bytes.
+int bwd_head_group(const Problem &p)
+{
+    constexpr size_t kAccBudget = 40u << 20;
+    for (int g = 8; g > 1; g >>= 1)
+        if (p.BH % g == 0 && (size_t)g * p.n * p.d * sizeof(float) <= kAccBudget) return g;
+    return 1;
+}
+
+namespace {
+template <int HD>
+attn_status preprocess_launch_t(const Problem &p, bool clear_acc)
+{
+    const size_t rows = (size_t)p.BH * p.n, acc_elems = rows * HD;
+    constexpr size_t rpw = 32 / (HD / 8);
+    size_t blocks = ((rows + rpw - 1) / rpw + 7) / 8;
+    if (blocks > (size_t)sm_count() * 8) blocks = (size_t)sm_count() * 8;
+    launch_begin("tc_bwd_preprocess", p.stream);
+    tc_preprocess_kernel<HD><<<(unsigned)blocks, 256, 0, p.stream>>>((const __nv_bfloat16 *)p.O, (const __nv_bfloat16 *)p.dO,
+                                                                     p.LSE, p.D, p.nLSE2, rows, p.scale,
+                                                                     clear_acc ? (uint4 *)p.dQ_acc : nullptr, acc_elems / 4);
+    launch_end(p.stream);
+    return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_LAUNCH;
+}
+}  // namespace
+
+attn_status bwd_preprocess_launch(const Problem &p, bool clear_acc)
+{
+    if (p.d == 64) return preprocess_launch_t<64>(p, clear_acc);
+    if (p.d == 128) return preprocess_launch_t<128>(p, clear_acc);
+    if (p.d == 256) return preprocess_launch_t<256>(p, clear_acc);
+    return ATTN_ERR_TILE;
+}
+
+attn_status bwd_dq_convert_launch(const Problem &p)
+{
+    const size_t n4 = (size_t)p.BH * p.n * p.d / 4;
     const size_t cap = (size_t)sm_count() * 16;
     const unsigned blocks = (unsigned)((n4 + 255) / 256 < cap ? (n4 + 255) / 256 : cap);
     launch_begin("bwd_dq_convert", p.stream);
@@ -1011,12 +916,11 @@ attn_status launch_bwd(const Problem &p)
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_LAUNCH;
 }
 
-}  // namespace
-
 size_t bwd_smem_bytes(int d) { return d == 64 ? BwdSmem<64>::kBytes : d == 128 ? BwdSmem<128>::kBytes : 0; }
 
 attn_status tc_bwd(const Problem &p)
 {
+    if (p.cfg.tile_q == 64 || p.d == 256) return tc_bwd64(p);
     if (p.d == 64) return p.cfg.deterministic ? launch_bwd<64, false>(p) : launch_bwd<64, true>(p);
     if (p.d == 128) return p.cfg.deterministic ? launch_bwd<128, false>(p) : launch_bwd<128, true>(p);
     return ATTN_ERR_TILE;

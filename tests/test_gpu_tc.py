@@ -140,7 +140,7 @@ def test_materialized_backward(n, d, tile_k, mask_kind):
     H.assert_within(errs, "bf16")
 
 
-def test_materialized_rejects_block_sparse_and_auto_picks_it_for_d256():
+def test_materialized_rejects_block_sparse_and_runs_its_own_phases():
     import torch
     import paper_2410_09397_b200 as attn
     from paper_2410_09397_b200 import binding as B
@@ -149,7 +149,7 @@ def test_materialized_rejects_block_sparse_and_auto_picks_it_for_d256():
     assert attn.attn_bwd_workspace_bytes(256, 256, 1, 1, mask, attn.ATTN_BF16, materialized()) == 0
     attn.attn_timing_enable(True)
     attn.attn_timing_collect()
-    errs = H.run_case(1, 1, 256, 256, "bf16", inputs.MASK_NONE, seed=39, check_bwd_only=False)
+    errs = H.run_case(1, 1, 256, 256, "bf16", inputs.MASK_NONE, seed=39, check_bwd_only=False, cfg=materialized())
     names = [k for k, _ in attn.attn_timing_collect()]
     attn.attn_timing_enable(False)
     H.assert_within(errs, "bf16")
