@@ -216,6 +216,19 @@ double attn_io_bound_elems(double n, double d, double M, int backward);
 /* min{Z_input^2/M, Z_input sqrt(Z_QK)/sqrt(M)} (Theorem 1.2). */
 double attn_io_bound_sparse_elems(double z_input, double z_qk, double M);
 
+/* I/O of the library's own tilings in the same model (Section 3.3: a cache of M items in front of
+ * a large memory; here the cache is one CTA's shared + tensor memory).  Replays on the host the loop
+ * nest of the kernels that `cfg` selects for one head of n x d with the given mask (ATTN_MASK_NONE
+ * or ATTN_MASK_CAUSAL) and counts the elements that cross the SM boundary: operand tiles loaded,
+ * results stored, and fp32 partial sums added into memory (the fused backward's dQ).  Passes that
+ * belong to the call are included (D pre-pass, accumulator clear and conversion, the materialised
+ * path's P, dP, dS round trips).  The sum is what Theorem 1.1 bounds from below at
+ * M = attn_cfg_onchip_elems(); comparing the two shows how close a tile shape is to the bound and
+ * how the I/O falls as the tile -- the cache -- grows (Figure 1 of the introduction).  Host only. */
+typedef struct { double loads, stores, reductions; } attn_io_count; /* elements, per head */
+attn_status attn_io_replay(int n, int d, int mask_kind, int dt, const attn_cfg *cfg, int backward,
+                           attn_io_count *out /* host */);
+
 const char *attn_status_str(int status);
 
 /* ---- diagnostics (process-wide state; not thread-safe; off by default) ----

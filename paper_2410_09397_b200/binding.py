@@ -26,7 +26,7 @@ ATTN_ALGO_AUTO, ATTN_ALGO_FUSED, ATTN_ALGO_MATERIALIZED, ATTN_ALGO_SIMT = 0, 1, 
 EXPORTS = (
     "attn_fwd", "attn_bwd", "attn_bwd_preprocess", "attn_fwd_workspace_bytes", "attn_bwd_workspace_bytes",
     "attn_workspace_status", "attn_supported_cfgs", "attn_cfg_onchip_elems", "attn_io_bound_elems",
-    "attn_io_bound_sparse_elems", "attn_status_str", "attn_kernel_launches", "attn_timing_enable",
+    "attn_io_bound_sparse_elems", "attn_io_replay", "attn_status_str", "attn_kernel_launches", "attn_timing_enable",
     "attn_timing_collect", "attn_bwd_noalloc", "attn_noalloc_scratch_bytes", "attn_noalloc_status",
     "attn_selftest_wait_timeout",
     "attn_project", "attn_weight_grad", "attn_weights_bwd", "attn_weights_bwd_workspace_bytes",
@@ -47,6 +47,10 @@ class CMask(ctypes.Structure):
 class CCfg(ctypes.Structure):
     _fields_ = [("tile_q", ctypes.c_int), ("tile_k", ctypes.c_int), ("tile_d", ctypes.c_int),
                 ("algo", ctypes.c_int), ("deterministic", ctypes.c_int)]
+
+
+class CIoCount(ctypes.Structure):
+    _fields_ = [("loads", ctypes.c_double), ("stores", ctypes.c_double), ("reductions", ctypes.c_double)]
 
 
 @dataclass
@@ -126,6 +130,8 @@ def lib() -> ctypes.CDLL:
     L.attn_io_bound_elems.argtypes = [ctypes.c_double] * 3 + [ci]
     L.attn_io_bound_sparse_elems.restype = ctypes.c_double
     L.attn_io_bound_sparse_elems.argtypes = [ctypes.c_double] * 3
+    L.attn_io_replay.restype = ci
+    L.attn_io_replay.argtypes = [ci, ci, ci, ci, ctypes.POINTER(CCfg), ci, ctypes.POINTER(CIoCount)]
     L.attn_kernel_launches.restype = ctypes.c_ulonglong
     L.attn_kernel_launches.argtypes = []
     L.attn_timing_enable.restype = ci
@@ -307,6 +313,16 @@ def attn_supported_cfgs(d: int, dt: int) -> list[Cfg]:
 
 def attn_cfg_onchip_elems(d: int, dt: int, cfg: Cfg | None, backward: bool) -> int:
     return int(lib().attn_cfg_onchip_elems(d, dt, _ref(cfg.c() if cfg else None), int(backward)))
+
+
+def attn_io_replay(n: int, d: int, mask_kind: int, dt: int, cfg: Cfg | None, backward: bool) -> dict:
+    """Elements one head moves across the SM boundary under ``cfg``: {"loads", "stores", "reductions", "total"}."""
+    out = CIoCount()
+    st = lib().attn_io_replay(n, d, mask_kind, dt, _ref(cfg.c() if cfg else None), int(backward), ctypes.byref(out))
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_io_replay")
+    return {"loads": out.loads, "stores": out.stores, "reductions": out.reductions,
+            "total": out.loads + out.stores + out.reductions}
 
 
 def attn_io_bound_elems(n, d, M, backward: bool) -> float:

@@ -108,4 +108,5 @@ def test_config4_full_small_cache_regime_tile_sweep(tile_k):
 
 
 def test_config4_full_default_cfg():
-    run_full("C4", [3])
+    """d = 256 with the default configuration: fused forward and the fused backward with 64-query tiles."""
+    run_full("C4", [0, 3, 7])
