@@ -56,12 +56,12 @@
 #include <omp.h>
 #endif
 
-enum { MASK_NONE = 0, MASK_CAUSAL = 1, MASK_BLOCK = 2, MASK_ELEMENT = 3 };
+enum { MASK_NONE = 0, MASK_CAUSAL = 1, MASK_BLOCK = 2, MASK_ELEMENT = 3, MASK_BLOCK_CAUSAL = 4 };
 
 typedef struct {
     int kind;            /* MASK_* */
-    int block;           /* block edge for MASK_BLOCK */
-    const uint8_t *bits; /* MASK_BLOCK: [mask_heads][nb][nb]; MASK_ELEMENT: [mask_heads][n][n]; 1 = keep */
+    int block;           /* block edge for MASK_BLOCK, MASK_BLOCK_CAUSAL */
+    const uint8_t *bits; /* MASK_BLOCK(_CAUSAL): [mask_heads][nb][nb]; MASK_ELEMENT: [mask_heads][n][n]; 1 = keep */
     int mask_heads;      /* 1: shared by every (batch, head); else batch*heads */
 } mask_t;
 
@@ -72,9 +72,11 @@ static int kept(const mask_t *m, int n, long bh, int i, int j)
         return 1;
     case MASK_CAUSAL:
         return j <= i;
-    case MASK_BLOCK: {
+    case MASK_BLOCK:
+    case MASK_BLOCK_CAUSAL: {   /* the latter: kept by the block mask AND j <= i */
         int nb = (n + m->block - 1) / m->block;
         long mh = m->mask_heads == 1 ? 0 : bh;
+        if (m->kind == MASK_BLOCK_CAUSAL && j > i) return 0;
         return m->bits[(mh * nb + i / m->block) * nb + j / m->block] != 0;
     }
     case MASK_ELEMENT: {

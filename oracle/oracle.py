@@ -28,7 +28,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "attn_oracle.c")
 _LIB = os.path.join(_HERE, "liboracle.so")
 
-MASK_NONE, MASK_CAUSAL, MASK_BLOCK, MASK_ELEMENT = 0, 1, 2, 3
+MASK_NONE, MASK_CAUSAL, MASK_BLOCK, MASK_ELEMENT, MASK_BLOCK_CAUSAL = 0, 1, 2, 3, 4
 
 
 def build(force: bool = False) -> str:
@@ -64,7 +64,7 @@ def _f64(a):
 
 
 def _mask_args(mask_kind, block, mask_bits):
-    if mask_kind in (MASK_BLOCK, MASK_ELEMENT):
+    if mask_kind in (MASK_BLOCK, MASK_ELEMENT, MASK_BLOCK_CAUSAL):
         mask_bits = np.ascontiguousarray(mask_bits, dtype=np.uint8)
         assert mask_bits.ndim == 3
         return mask_bits, int(mask_bits.shape[0])
@@ -105,7 +105,7 @@ def attn_dense(Q, K, V, dO, *, mask_kind=MASK_NONE, block=128, mask_bits=None, s
     n, d = Q.shape
     scale = 1.0 / math.sqrt(d) if scale is None else float(scale)
     bits = None
-    if mask_kind in (MASK_BLOCK, MASK_ELEMENT):
+    if mask_kind in (MASK_BLOCK, MASK_ELEMENT, MASK_BLOCK_CAUSAL):
         bits = np.ascontiguousarray(mask_bits, dtype=np.uint8)
     out = {"l": np.empty(n), "f": np.empty((n, n)), "q": np.empty((n, n)), "p": np.empty((n, n)),
            "v_fq": np.empty(n)}

@@ -28,6 +28,8 @@ def masks_for(n, block=2, seed=11):
         dict(mask_kind=orc.MASK_NONE),
         dict(mask_kind=orc.MASK_CAUSAL),
         dict(mask_kind=orc.MASK_BLOCK, block=block, mask_bits=bm),
+        # block mask AND causal; the diagonal blocks are kept so that every row keeps its own key
+        dict(mask_kind=orc.MASK_BLOCK_CAUSAL, block=block, mask_bits=bm | np.eye(nb, dtype=bm.dtype)[None]),
     ]
 
 
@@ -108,7 +110,8 @@ def keep_matrix(n, mk):
     if kind == orc.MASK_CAUSAL:
         return np.tril(np.ones((n, n), bool))
     blk = mk["block"]
-    return np.kron(mk["mask_bits"][0].astype(bool), np.ones((blk, blk), bool))[:n, :n]
+    keep = np.kron(mk["mask_bits"][0].astype(bool), np.ones((blk, blk), bool))[:n, :n]
+    return keep & np.tril(np.ones((n, n), bool)) if kind == orc.MASK_BLOCK_CAUSAL else keep
 
 
 @pytest.mark.parametrize("n,d", [(6, 4), (12, 8), (33, 16)])
