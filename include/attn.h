@@ -60,7 +60,8 @@ typedef enum {
 
 typedef enum { ATTN_F32 = 0, ATTN_BF16 = 1 } attn_dtype;
 
-typedef enum { ATTN_MASK_NONE = 0, ATTN_MASK_CAUSAL = 1, ATTN_MASK_BLOCK_SPARSE = 2 } attn_mask_kind;
+typedef enum { ATTN_MASK_NONE = 0, ATTN_MASK_CAUSAL = 1, ATTN_MASK_BLOCK_SPARSE = 2,
+               ATTN_MASK_BLOCK_SPARSE_CAUSAL = 3 } attn_mask_kind;
 
 /* Which (i, j) score entries are kept.  NULL means ATTN_MASK_NONE.
  *   CAUSAL:       keep j <= i (one n for queries and keys).
@@ -68,6 +69,8 @@ typedef enum { ATTN_MASK_NONE = 0, ATTN_MASK_CAUSAL = 1, ATTN_MASK_BLOCK_SPARSE 
  *                 block_mask is DEVICE uint8 [mask_heads][nb][nb], nb = ceil(n / block);
  *                 mask_heads is 1 (shared by every batch and head) or batch * heads.
  *                 The tensor-core algorithms need block to be a multiple of 128.
+ *   BLOCK_SPARSE_CAUSAL: both at once -- keep (i, j) iff its block is kept and j <= i
+ *                 (same fields as BLOCK_SPARSE; blocks above the diagonal are never visited).
  * This is the sparse setting of Section 4.1 with Z_QK = the number of kept entries;
  * a masked score is minus infinity, not a stored zero. */
 typedef struct {

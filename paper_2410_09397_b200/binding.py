@@ -19,7 +19,7 @@ ATTN_OK = 0
 (ATTN_ERR_NULL, ATTN_ERR_SHAPE, ATTN_ERR_DTYPE, ATTN_ERR_ALIGN, ATTN_ERR_TILE, ATTN_ERR_MASK, ATTN_ERR_WORKSPACE,
  ATTN_ERR_ARCH, ATTN_ERR_LAUNCH, ATTN_ERR_DEVICE_TIMEOUT) = range(1, 11)
 ATTN_F32, ATTN_BF16 = 0, 1
-ATTN_MASK_NONE, ATTN_MASK_CAUSAL, ATTN_MASK_BLOCK_SPARSE = 0, 1, 2
+ATTN_MASK_NONE, ATTN_MASK_CAUSAL, ATTN_MASK_BLOCK_SPARSE, ATTN_MASK_BLOCK_SPARSE_CAUSAL = 0, 1, 2, 3
 ATTN_ALGO_AUTO, ATTN_ALGO_FUSED, ATTN_ALGO_MATERIALIZED, ATTN_ALGO_SIMT = 0, 1, 2, 3
 
 # every symbol include/attn.h declares
@@ -61,7 +61,7 @@ class Mask:
     block_mask: object = None
 
     def c(self) -> CMask | None:
-        if self.kind == ATTN_MASK_BLOCK_SPARSE:
+        if self.kind in (ATTN_MASK_BLOCK_SPARSE, ATTN_MASK_BLOCK_SPARSE_CAUSAL):
             bm = self.block_mask
             return CMask(self.kind, self.block, bm.data_ptr() if bm is not None else None,
                          int(bm.shape[0]) if bm is not None else 1)

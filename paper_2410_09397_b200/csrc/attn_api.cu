@@ -27,12 +27,12 @@ attn_status resolve_cfg(const Args &a, int backward, attn_cfg *out)
         attn_cfg probe = c;
         probe.algo = ATTN_ALGO_FUSED;
         const bool tc_ok = a.dt == ATTN_BF16 && (a.n % 8) == 0 && tc_cfg_supported(a.d, probe, backward) &&
-                           !(a.mask && a.mask->kind == ATTN_MASK_BLOCK_SPARSE && a.mask->block % 128 != 0);
+                           !(a.mask && mask_is_block(a.mask->kind) && a.mask->block % 128 != 0);
         c.algo = tc_ok ? ATTN_ALGO_FUSED : ATTN_ALGO_SIMT;
         // d = 256 backward: the fused tile set does not fit on chip; the small-cache algorithm takes it
         probe.algo = ATTN_ALGO_MATERIALIZED;
         if (!tc_ok && backward && a.dt == ATTN_BF16 && a.d == 256 && (a.n % 8) == 0 &&
-            !(a.mask && a.mask->kind == ATTN_MASK_BLOCK_SPARSE) && tc_cfg_supported(a.d, probe, backward))
+            !(a.mask && mask_is_block(a.mask->kind)) && tc_cfg_supported(a.d, probe, backward))
             c.algo = ATTN_ALGO_MATERIALIZED;
     }
     if (c.algo == ATTN_ALGO_MATERIALIZED && !backward) {   // its forward is the fused one, with that kernel's own tiles
@@ -52,8 +52,8 @@ attn_status resolve_cfg(const Args &a, int backward, attn_cfg *out)
         if (a.dt != ATTN_BF16) return ATTN_ERR_DTYPE;
         if (a.d != 64 && a.d != 128 && a.d != 256) return ATTN_ERR_SHAPE;
         if (a.n % 8 != 0) return ATTN_ERR_SHAPE;
-        if (a.mask && a.mask->kind == ATTN_MASK_BLOCK_SPARSE && a.mask->block % 128 != 0) return ATTN_ERR_MASK;
-        if (c.algo == ATTN_ALGO_MATERIALIZED && a.mask && a.mask->kind == ATTN_MASK_BLOCK_SPARSE) return ATTN_ERR_MASK;
+        if (a.mask && mask_is_block(a.mask->kind) && a.mask->block % 128 != 0) return ATTN_ERR_MASK;
+        if (c.algo == ATTN_ALGO_MATERIALIZED && a.mask && mask_is_block(a.mask->kind)) return ATTN_ERR_MASK;
         if (!tc_cfg_supported(a.d, c, backward)) return ATTN_ERR_TILE;
         // fill defaults the way the kernels resolve them
         attn_cfg list[32];
@@ -83,8 +83,8 @@ attn_status check_shape(const Args &a)
     if ((double)a.batch * a.heads * a.n * a.d > 1.7e10) return ATTN_ERR_SHAPE;
     if (a.mask) {
         const attn_mask &m = *a.mask;
-        if (m.kind < ATTN_MASK_NONE || m.kind > ATTN_MASK_BLOCK_SPARSE) return ATTN_ERR_MASK;
-        if (m.kind == ATTN_MASK_BLOCK_SPARSE) {
+        if (m.kind < ATTN_MASK_NONE || m.kind > ATTN_MASK_BLOCK_SPARSE_CAUSAL) return ATTN_ERR_MASK;
+        if (mask_is_block(m.kind)) {
             if (m.block < 1) return ATTN_ERR_MASK;
             if (m.mask_heads != 1 && m.mask_heads != a.batch * a.heads) return ATTN_ERR_MASK;
         }
@@ -105,7 +105,7 @@ attn_status layout(const Args &a, int backward, attn_cfg *cfg_out, WorkspaceLayo
     L->status = off; off += 256;
     const size_t BH = (size_t)a.batch * a.heads;
     if (backward) { L->D = off; off += align_up(BH * a.n * sizeof(float), 256); }
-    const bool sparse = a.mask && a.mask->kind == ATTN_MASK_BLOCK_SPARSE;
+    const bool sparse = a.mask && mask_is_block(a.mask->kind);
     if (sparse && c.algo != ATTN_ALGO_SIMT) {
         const size_t nb = (a.n + a.mask->block - 1) / a.mask->block, mh = a.mask->mask_heads;
         L->row_ptr = off; off += align_up(mh * 2 * nb * sizeof(int), 256);
@@ -162,7 +162,7 @@ attn_status fill_problem(Problem &p, const Args &a, int backward, float scale, v
     attn_cfg c;
     attn_status st = layout(a, backward, &c, &L);
     if (st != ATTN_OK) return st;
-    if (a.mask && a.mask->kind == ATTN_MASK_BLOCK_SPARSE && !a.mask->block_mask) return ATTN_ERR_NULL;
+    if (a.mask && mask_is_block(a.mask->kind) && !a.mask->block_mask) return ATTN_ERR_NULL;
     if (!workspace || workspace_bytes < L.total) return ATTN_ERR_WORKSPACE;
     if (((uintptr_t)workspace & 255) != 0) return ATTN_ERR_ALIGN;
     if (!(scale >= 0.f) || isinf(scale)) return ATTN_ERR_SHAPE;
@@ -170,10 +170,10 @@ attn_status fill_problem(Problem &p, const Args &a, int backward, float scale, v
     p.BH = (long)a.batch * a.heads;
     p.dt = a.dt;
     p.mask_kind = a.mask ? a.mask->kind : ATTN_MASK_NONE;
-    p.block = p.mask_kind == ATTN_MASK_BLOCK_SPARSE ? a.mask->block : 0;
-    p.mask_heads = p.mask_kind == ATTN_MASK_BLOCK_SPARSE ? a.mask->mask_heads : 1;
+    p.block = mask_is_block(p.mask_kind) ? a.mask->block : 0;
+    p.mask_heads = mask_is_block(p.mask_kind) ? a.mask->mask_heads : 1;
     p.nb = p.block ? (a.n + p.block - 1) / p.block : 0;
-    p.block_mask = p.mask_kind == ATTN_MASK_BLOCK_SPARSE ? a.mask->block_mask : nullptr;
+    p.block_mask = mask_is_block(p.mask_kind) ? a.mask->block_mask : nullptr;
     p.scale = scale == 0.f ? 1.0f / sqrtf((float)a.d) : scale;
     p.cfg = c;
     char *w = (char *)workspace;

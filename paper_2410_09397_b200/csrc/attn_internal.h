@@ -45,6 +45,10 @@ void launch_end(cudaStream_t s);
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// mask kinds: "block" = described by a block mask, "causal" = entries with j > i are dropped
+__host__ __device__ inline bool mask_is_block(int kind) { return kind == ATTN_MASK_BLOCK_SPARSE || kind == ATTN_MASK_BLOCK_SPARSE_CAUSAL; }
+__host__ __device__ inline bool mask_is_causal(int kind) { return kind == ATTN_MASK_CAUSAL || kind == ATTN_MASK_BLOCK_SPARSE_CAUSAL; }
+
 // Streaming multiprocessors of the current device (grid sizing of the grid-stride and persistent kernels).
 int sm_count();
 

@@ -337,7 +337,7 @@ size_t mat_onchip_bytes(int, const attn_cfg &c)
 
 attn_status mat_bwd(const Problem &p)
 {
-    if (p.mask_kind == ATTN_MASK_BLOCK_SPARSE) return ATTN_ERR_MASK;
+    if (mask_is_block(p.mask_kind)) return ATTN_ERR_MASK;
     const size_t rows = (size_t)p.BH * p.n;
     size_t blocks = (rows + 7) / 8;
     if (blocks > (size_t)sm_count() * 8) blocks = (size_t)sm_count() * 8;

@@ -39,6 +39,7 @@ __device__ __forceinline__ bool keep(const MaskDev &m, int i, int j)
 {
     if (m.kind == ATTN_MASK_NONE) return true;
     if (m.kind == ATTN_MASK_CAUSAL) return j <= i;
+    if (m.kind == ATTN_MASK_BLOCK_SPARSE_CAUSAL && j > i) return false;
     return m.bits[(size_t)(i / m.block) * m.nb + j / m.block] != 0;
 }
 
@@ -47,6 +48,7 @@ __device__ __forceinline__ bool tile_any(const MaskDev &m, int i0, int i1, int j
 {
     if (m.kind == ATTN_MASK_NONE) return true;
     if (m.kind == ATTN_MASK_CAUSAL) return j0 <= i1;
+    if (m.kind == ATTN_MASK_BLOCK_SPARSE_CAUSAL && j0 > i1) return false;
     for (int I = i0 / m.block; I <= i1 / m.block; ++I)
         for (int J = j0 / m.block; J <= j1 / m.block; ++J)
             if (m.bits[(size_t)I * m.nb + J]) return true;
@@ -56,7 +58,7 @@ __device__ __forceinline__ bool tile_any(const MaskDev &m, int i0, int i1, int j
 __device__ __forceinline__ MaskDev head_mask(int kind, int block, int nb, const uint8_t *bits, int mask_heads, long bh)
 {
     MaskDev m{kind, block, nb, bits};
-    if (kind == ATTN_MASK_BLOCK_SPARSE && mask_heads != 1) m.bits = bits + (size_t)bh * nb * nb;
+    if (mask_is_block(kind) && mask_heads != 1) m.bits = bits + (size_t)bh * nb * nb;
     return m;
 }
 
@@ -585,7 +587,7 @@ attn_status preprocess_D(const void *O, const void *dO, float *D, size_t rows, i
 
 attn_status build_block_index(const Problem &p)
 {
-    if (p.mask_kind != ATTN_MASK_BLOCK_SPARSE || !p.row_ptr) return ATTN_OK;
+    if (!mask_is_block(p.mask_kind) || !p.row_ptr) return ATTN_OK;
     launch_begin("block_index", p.stream);
     block_index_kernel<<<dim3(p.nb, p.mask_heads), 64, 0, p.stream>>>(p.block_mask, p.nb, p.row_ptr, p.col_idx,
                                                                       p.col_ptr, p.row_idx);

@@ -278,7 +278,7 @@ tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
             const int s2 = k & 1, i0 = it * TQ;
             const float4 *sNL = reinterpret_cast<const float4 *>(smem + L::oLSE + s2 * 512 + h * 256 + qq * 128);
             const float4 *sDs = reinterpret_cast<const float4 *>(smem + L::oD + s2 * 512 + h * 256 + qq * 128);
-            const bool diag = a.mask_kind == ATTN_MASK_CAUSAL && it == jt;
+            const bool diag = mask_is_causal(a.mask_kind) && it == jt;
             const bool masked = diag || i0 + TQ > n || j0 + TK > n;
             const int ig0 = i0 + h * 64 + qq * 32;
             mbar_wait(&bars[KD_S], k & 1, ab);
@@ -671,7 +671,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
             const int s = k & 1, i0 = it * TQ;
             const float4 *sNL = reinterpret_cast<const float4 *>(smem + L::oLSE + s * 512 + h * 256 + qq * 128);
             const float4 *sDs = reinterpret_cast<const float4 *>(smem + L::oD + s * 512 + h * 256 + qq * 128);
-            const bool diag = a.mask_kind == ATTN_MASK_CAUSAL && it == jt;
+            const bool diag = mask_is_causal(a.mask_kind) && it == jt;
             const bool masked = diag || i0 + TQ > n || j0 + TK > n;
             const int ig0 = i0 + h * 64 + qq * 32;
             mbar_wait(&bars[V2_QFULL + s], (k >> 1) & 1, ab);

@@ -287,7 +287,7 @@ tc_bwd_fused64_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_const
             const int s = t % NS, i0 = it * TQ64;
             const float4 *sNL = reinterpret_cast<const float4 *>(smem + L::oLSE + s * 256 + g * 128);
             const float4 *sDs = reinterpret_cast<const float4 *>(smem + L::oD + s * 256 + g * 128);
-            const bool diag = a.mask_kind == ATTN_MASK_CAUSAL && i0 < j0 + TK;   // some (i, j) of the tile pair has j > i
+            const bool diag = mask_is_causal(a.mask_kind) && i0 < j0 + TK;   // some (i, j) of the tile pair has j > i
             const bool masked = diag || i0 + TQ64 > n || j0 + TK > n;
             const int ig0 = i0 + g * 32;
             mbar_wait(&bars[B_QFULL + s], (t / NS) & 1, ab);

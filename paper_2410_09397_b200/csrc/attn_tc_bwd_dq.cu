@@ -58,10 +58,11 @@ enum { DB_Q = 0, DB_KFULL = 1, DB_KEMPTY = 4, DB_VFULL = 7, DB_VEMPTY = 9, DB_S 
        DB_DQ = 17 };
 
 struct KeyIterD {
-    int kind, n, sub, raw;
+    int kind, n, sub, raw, last_i;
     const int *cols;
     __device__ KeyIterD(const DqArgs &a, int it, long bh) : kind(a.mask_kind), n(a.n), sub(1), raw(0), cols(nullptr)
     {
+        last_i = min(it * TQ + TQ, n) - 1;
         const int ntk = (n + TKD - 1) / TKD;
         if (kind == ATTN_MASK_NONE) raw = ntk;
         else if (kind == ATTN_MASK_CAUSAL) raw = (min(it * TQ + TQ, n) - 1) / TKD + 1;
@@ -76,7 +77,9 @@ struct KeyIterD {
     }
     __device__ int tile(int idx) const
     {
-        const int jt = kind == ATTN_MASK_BLOCK_SPARSE ? cols[idx / sub] * sub + idx % sub : idx;
+        const int jt = mask_is_block(kind) ? cols[idx / sub] * sub + idx % sub : idx;
+        // block mask AND causal: a key tile that begins after the last query of the tile keeps nothing
+        if (kind == ATTN_MASK_BLOCK_SPARSE_CAUSAL && jt * TKD > last_i) return -1;
         return jt * TKD < n ? jt : -1;
     }
 };
@@ -239,7 +242,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
             if (jt < 0) continue;
             const int b = k & 1, j0 = jt * TKD + wg * 32;
             const uint32_t T_S = tm + b * 128;
-            const bool masked = (a.mask_kind == ATTN_MASK_CAUSAL && jt * TKD + TKD - 1 > i0) || jt * TKD + TKD > n;
+            const bool masked = (mask_is_causal(a.mask_kind) && jt * TKD + TKD - 1 > i0) || jt * TKD + TKD > n;
             mbar_wait(&bars[DB_S + b], (k >> 1) & 1, ab);
             tcgen05_fence_after();
             float p[32];
@@ -251,7 +254,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
                 for (int e = 0; e < 32; ++e) p[e] = ex2_fast(fmaf(__uint_as_float(sv0[e]), sl2, nl));
             }
             if (masked) {
-                const bool causal = a.mask_kind == ATTN_MASK_CAUSAL;
+                const bool causal = mask_is_causal(a.mask_kind);
 #pragma unroll
                 for (int e = 0; e < 32; ++e) {
                     const int jg = j0 + e;

@@ -70,10 +70,11 @@ enum { FB_Q = 0, FB_KVFULL = 1, FB_KVEMPTY = 4, FB_S = 7, FB_P = 9, FB_O = 11 };
 template <int TKF>
 struct KeyIter {
     // Enumerates the key tiles (of TKF keys) a query tile `it` (128 queries) has to visit.
-    int kind, n, sub, raw;
+    int kind, n, sub, raw, last_i;
     const int *cols;
     __device__ KeyIter(const FwdArgs &a, int it, long bh) : kind(a.mask_kind), n(a.n), sub(1), raw(0), cols(nullptr)
     {
+        last_i = min(it * TQ + TQ, n) - 1;
         const int ntk = (n + TKF - 1) / TKF;
         if (kind == ATTN_MASK_NONE) raw = ntk;
         else if (kind == ATTN_MASK_CAUSAL) {
@@ -91,8 +92,10 @@ struct KeyIter {
     __device__ int tile(int idx) const
     {
         int jt;
-        if (kind == ATTN_MASK_BLOCK_SPARSE) jt = cols[idx / sub] * sub + idx % sub;
+        if (mask_is_block(kind)) jt = cols[idx / sub] * sub + idx % sub;
         else jt = idx;
+        // block mask AND causal: a key tile that begins after the last query of the tile keeps nothing
+        if (kind == ATTN_MASK_BLOCK_SPARSE_CAUSAL && jt * TKF > last_i) return -1;
         return jt * TKF < n ? jt : -1;
     }
 };
@@ -236,10 +239,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
 #pragma unroll
                 for (int e = 0; e < 32; ++e) sv[c + e] = __uint_as_float(v[e]);   // raw scores; scale * log2e enters below
             }
-            const bool need_mask = (a.mask_kind == ATTN_MASK_CAUSAL && j0 + TKF - 1 > i0) || j0 + TKF > n;
+            const bool need_mask = (mask_is_causal(a.mask_kind) && j0 + TKF - 1 > i0) || j0 + TKF > n;
             float mx = -INFINITY;
             if (need_mask) {
-                const bool causal = a.mask_kind == ATTN_MASK_CAUSAL;
+                const bool causal = mask_is_causal(a.mask_kind);
 #pragma unroll
                 for (int e = 0; e < CW; ++e) {
                     const int jg = j0 + wg * CW + e;
@@ -487,7 +490,7 @@ tc_fwd_rows_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
             if (jt < 0) continue;
             if ((k++ & 1) != w) continue;
             const int j0 = jt * TKF;
-            const bool causal = a.mask_kind == ATTN_MASK_CAUSAL;
+            const bool causal = mask_is_causal(a.mask_kind);
             const bool need_mask = (causal && j0 + TKF - 1 > i0) || j0 + TKF > n;
             mbar_wait(&bars[F2_S + w], cnt & 1, ab);
             tcgen05_fence_after();

@@ -51,7 +51,11 @@ struct TileIterT {
         int it;
         if (kind == ATTN_MASK_NONE) it = idx;
         else if (kind == ATTN_MASK_CAUSAL) it = jt * (TK / TQT) + idx;
-        else it = rows[idx / sub] * sub + idx % sub;
+        else {
+            it = rows[idx / sub] * sub + idx % sub;
+            // block mask AND causal: a query tile that ends before the key tile begins keeps nothing
+            if (kind == ATTN_MASK_BLOCK_SPARSE_CAUSAL && (it + 1) * TQT <= jt * TK) return -1;
+        }
         return it * TQT < n ? it : -1;
     }
 };

@@ -34,7 +34,7 @@ _M2 = np.uint64(0x94D049BB133111EB)
 # tensor ids inside one workload seed
 TENSOR_Q, TENSOR_K, TENSOR_V, TENSOR_DO, TENSOR_AUX = 0, 1, 2, 3, 4
 
-MASK_NONE, MASK_CAUSAL, MASK_BLOCK_SPARSE = 0, 1, 2
+MASK_NONE, MASK_CAUSAL, MASK_BLOCK_SPARSE, MASK_BLOCK_SPARSE_CAUSAL = 0, 1, 2, 3
 
 
 def _mix(z: np.ndarray) -> np.ndarray:

@@ -12,6 +12,8 @@ TOL = {"f32": 1e-4, "bf16": 2e-2}   # max|err| <= TOL * max|ref| per output tens
 def oracle_mask_kwargs(mask_kind, block, bmask):
     if mask_kind == inputs.MASK_BLOCK_SPARSE:
         return dict(mask_kind=orc.MASK_BLOCK, block=block, mask_bits=bmask)
+    if mask_kind == inputs.MASK_BLOCK_SPARSE_CAUSAL:
+        return dict(mask_kind=orc.MASK_BLOCK_CAUSAL, block=block, mask_bits=bmask)
     return dict(mask_kind=mask_kind)
 
 
@@ -56,7 +58,7 @@ def run_case(b, h, n, d, dtype, mask_kind, *, seed=7, block=128, bmask=None, cfg
     from paper_2410_09397_b200 import binding as B
 
     x = make_inputs(seed, b, h, n, d, dtype)
-    if mask_kind == inputs.MASK_BLOCK_SPARSE and bmask is None:
+    if mask_kind in (inputs.MASK_BLOCK_SPARSE, inputs.MASK_BLOCK_SPARSE_CAUSAL) and bmask is None:
         bmask = inputs.block_mask(seed + 100, (n + block - 1) // block, keep_prob)
     mk = oracle_mask_kwargs(mask_kind, block, bmask)
     sc = None if scale == 0.0 else scale
