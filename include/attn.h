@@ -68,7 +68,9 @@ typedef enum { ATTN_MASK_NONE = 0, ATTN_MASK_CAUSAL = 1, ATTN_MASK_BLOCK_SPARSE 
  *   BLOCK_SPARSE: keep (i, j) iff block_mask[h][i / block][j / block] != 0, where
  *                 block_mask is DEVICE uint8 [mask_heads][nb][nb], nb = ceil(n / block);
  *                 mask_heads is 1 (shared by every batch and head) or batch * heads.
- *                 The tensor-core algorithms need block to be a multiple of 128.
+ *                 The tensor-core algorithms need block to be a multiple of 128, or 64 or 32:
+ *                 with the two fine sizes they visit every 128 x 128 tile that keeps at
+ *                 least one block and drop the other blocks' entries inside the tile.
  *   BLOCK_SPARSE_CAUSAL: both at once -- keep (i, j) iff its block is kept and j <= i
  *                 (same fields as BLOCK_SPARSE; blocks above the diagonal are never visited).
  * This is the sparse setting of Section 4.1 with Z_QK = the number of kept entries;

@@ -16,6 +16,9 @@ struct Args {
 
 int elem_size(int dt) { return dt == ATTN_F32 ? 4 : 2; }
 
+// block edges the tensor-core kernels take: whole 128 x 128 tiles, or 32 / 64 (several blocks per tile)
+bool tc_block_ok(int block) { return block > 0 && (block % 128 == 0 || block == 64 || block == 32); }
+
 // Resolves algo / tiles; returns ATTN_OK or the validation error.
 attn_status resolve_cfg(const Args &a, int backward, attn_cfg *out)
 {
@@ -27,7 +30,7 @@ attn_status resolve_cfg(const Args &a, int backward, attn_cfg *out)
         attn_cfg probe = c;
         probe.algo = ATTN_ALGO_FUSED;
         const bool tc_ok = a.dt == ATTN_BF16 && (a.n % 8) == 0 && tc_cfg_supported(a.d, probe, backward) &&
-                           !(a.mask && mask_is_block(a.mask->kind) && a.mask->block % 128 != 0);
+                           !(a.mask && mask_is_block(a.mask->kind) && !tc_block_ok(a.mask->block));
         c.algo = tc_ok ? ATTN_ALGO_FUSED : ATTN_ALGO_SIMT;
         // d = 256 backward: the fused tile set does not fit on chip; the small-cache algorithm takes it
         probe.algo = ATTN_ALGO_MATERIALIZED;
@@ -52,7 +55,7 @@ attn_status resolve_cfg(const Args &a, int backward, attn_cfg *out)
         if (a.dt != ATTN_BF16) return ATTN_ERR_DTYPE;
         if (a.d != 64 && a.d != 128 && a.d != 256) return ATTN_ERR_SHAPE;
         if (a.n % 8 != 0) return ATTN_ERR_SHAPE;
-        if (a.mask && mask_is_block(a.mask->kind) && a.mask->block % 128 != 0) return ATTN_ERR_MASK;
+        if (a.mask && mask_is_block(a.mask->kind) && !tc_block_ok(a.mask->block)) return ATTN_ERR_MASK;
         if (c.algo == ATTN_ALGO_MATERIALIZED && a.mask && mask_is_block(a.mask->kind)) return ATTN_ERR_MASK;
         if (!tc_cfg_supported(a.d, c, backward)) return ATTN_ERR_TILE;
         // fill defaults the way the kernels resolve them
@@ -107,7 +110,8 @@ attn_status layout(const Args &a, int backward, attn_cfg *cfg_out, WorkspaceLayo
     if (backward) { L->D = off; off += align_up(BH * a.n * sizeof(float), 256); }
     const bool sparse = a.mask && mask_is_block(a.mask->kind);
     if (sparse && c.algo != ATTN_ALGO_SIMT) {
-        const size_t nb = (a.n + a.mask->block - 1) / a.mask->block, mh = a.mask->mask_heads;
+        const int eff = a.mask->block < 128 ? 128 : a.mask->block;   // fine blocks: lists of 128 x 128 super-blocks
+        const size_t nb = (a.n + eff - 1) / eff, mh = a.mask->mask_heads;
         L->row_ptr = off; off += align_up(mh * 2 * nb * sizeof(int), 256);
         L->col_idx = off; off += align_up(mh * nb * nb * sizeof(int), 256);
         L->col_ptr = off; off += align_up(mh * 2 * nb * sizeof(int), 256);
@@ -174,6 +178,12 @@ attn_status fill_problem(Problem &p, const Args &a, int backward, float scale, v
     p.mask_heads = mask_is_block(p.mask_kind) ? a.mask->mask_heads : 1;
     p.nb = p.block ? (a.n + p.block - 1) / p.block : 0;
     p.block_mask = mask_is_block(p.mask_kind) ? a.mask->block_mask : nullptr;
+    p.fine = FineMask{nullptr, 0, 0};
+    if (p.block && p.block < 128 && c.algo != ATTN_ALGO_SIMT) {
+        p.fine = FineMask{p.block_mask, p.block, p.nb};
+        p.block = 128;
+        p.nb = (a.n + 127) / 128;
+    }
     p.scale = scale == 0.f ? 1.0f / sqrtf((float)a.d) : scale;
     p.cfg = c;
     char *w = (char *)workspace;

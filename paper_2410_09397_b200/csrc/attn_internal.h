@@ -8,6 +8,22 @@
 
 namespace attn {
 
+// A block mask whose blocks are finer than the 128 x 128 tiles of the tensor-core kernels (block edge 32 or
+// 64): the kernels then walk lists of 128 x 128 super-blocks that keep at least one fine block, and drop the
+// entries of the fine blocks that are not kept inside every visited tile.  block == 0: not in use.
+struct FineMask {
+    const uint8_t *bits;   // the caller's mask [mask_heads][nb][nb]
+    int block, nb;
+};
+#ifdef __CUDACC__
+// (i, j) < n; which of the caller's masks: head bh unless one mask serves all
+__device__ __forceinline__ bool fine_keep(const FineMask &f, int mask_heads, long bh, int i, int j)
+{
+    const uint8_t *m = f.bits + (mask_heads == 1 ? 0 : (size_t)bh * f.nb * f.nb);
+    return m[(size_t)(i / f.block) * f.nb + j / f.block] != 0;
+}
+#endif
+
 // One fully validated problem, as handed from the C ABI to the kernel launchers.
 struct Problem {
     const void *Q, *K, *V, *O, *dO;   // inputs (O, dO only for the backward)
@@ -19,6 +35,7 @@ struct Problem {
     long BH;                          // batch * heads
     int mask_kind, block, mask_heads, nb;
     const uint8_t *block_mask;
+    FineMask fine;                    // tensor-core algorithms with a block edge below 128: block / nb then describe the super-blocks
     int dt;
     float scale;
     attn_cfg cfg;                     // resolved: algo and tiles are final

@@ -471,22 +471,31 @@ __global__ void __launch_bounds__(256) preprocess_kernel(const T *__restrict__ O
 // ---------------------------------------------------------------- block-mask index build
 // One CTA per (mask head, block row) for the CSR half and per (mask head, block
 // column) for the CSC half; ordered compaction by a single warp-free scan (nb is small).
-__global__ void block_index_kernel(const uint8_t *bits, int nb, int *row_ptr, int *col_idx, int *col_ptr, int *row_idx)
+// `ratio` > 1: the mask has nbm = about ratio * nb blocks per side, and block (I, J) of the lists is a
+// super-block that is kept if any of its ratio x ratio mask blocks is.
+__global__ void block_index_kernel(const uint8_t *bits, int nb, int nbm, int ratio, int *row_ptr, int *col_idx, int *col_ptr,
+                                   int *row_idx)
 {
     const int h = blockIdx.y, r = blockIdx.x;
-    const uint8_t *m = bits + (size_t)h * nb * nb;
+    const uint8_t *mm = bits + (size_t)h * nbm * nbm;
+    auto kept = [&](int I, int J) {
+        for (int x = I * ratio; x < min((I + 1) * ratio, nbm); ++x)
+            for (int y = J * ratio; y < min((J + 1) * ratio, nbm); ++y)
+                if (mm[(size_t)x * nbm + y]) return true;
+        return false;
+    };
     if (threadIdx.x == 0) {
         int *cidx = col_idx + (size_t)h * nb * nb + (size_t)r * nb;
         int c = 0;
         for (int j = 0; j < nb; ++j)
-            if (m[(size_t)r * nb + j]) cidx[c++] = j;
+            if (kept(r, j)) cidx[c++] = j;
         row_ptr[(size_t)h * 2 * nb + 2 * r] = r * nb;          // start, in col_idx of this head
         row_ptr[(size_t)h * 2 * nb + 2 * r + 1] = r * nb + c;  // end
     } else if (threadIdx.x == 32) {
         int *ridx = row_idx + (size_t)h * nb * nb + (size_t)r * nb;
         int c = 0;
         for (int i = 0; i < nb; ++i)
-            if (m[(size_t)i * nb + r]) ridx[c++] = i;
+            if (kept(i, r)) ridx[c++] = i;
         col_ptr[(size_t)h * 2 * nb + 2 * r] = r * nb;
         col_ptr[(size_t)h * 2 * nb + 2 * r + 1] = r * nb + c;
     }
@@ -589,7 +598,8 @@ attn_status build_block_index(const Problem &p)
 {
     if (!mask_is_block(p.mask_kind) || !p.row_ptr) return ATTN_OK;
     launch_begin("block_index", p.stream);
-    block_index_kernel<<<dim3(p.nb, p.mask_heads), 64, 0, p.stream>>>(p.block_mask, p.nb, p.row_ptr, p.col_idx,
+    const int nbm = p.fine.block ? p.fine.nb : p.nb, ratio = p.fine.block ? 128 / p.fine.block : 1;
+    block_index_kernel<<<dim3(p.nb, p.mask_heads), 64, 0, p.stream>>>(p.block_mask, p.nb, nbm, ratio, p.row_ptr, p.col_idx,
                                                                       p.col_ptr, p.row_idx);
     launch_end(p.stream);
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_LAUNCH;

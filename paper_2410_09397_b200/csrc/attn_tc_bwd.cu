@@ -279,8 +279,10 @@ tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
             const float4 *sNL = reinterpret_cast<const float4 *>(smem + L::oLSE + s2 * 512 + h * 256 + qq * 128);
             const float4 *sDs = reinterpret_cast<const float4 *>(smem + L::oD + s2 * 512 + h * 256 + qq * 128);
             const bool diag = mask_is_causal(a.mask_kind) && it == jt;
-            const bool masked = diag || i0 + TQ > n || j0 + TK > n;
             const int ig0 = i0 + h * 64 + qq * 32;
+            // fine blocks: this thread's 32 query columns and its key row lie in one block of the caller's mask
+            const bool fkeep = !a.fine.block || (ig0 < n && jg < n && fine_keep(a.fine, a.mask_heads, bh, ig0, jg));
+            const bool masked = diag || i0 + TQ > n || j0 + TK > n || a.fine.block != 0;
             mbar_wait(&bars[KD_S], k & 1, ab);
             tcgen05_fence_after();
             uint32_t ppack[16];
@@ -303,7 +305,7 @@ tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const int ig = ig0 + q * 4 + e;
-                            const bool ok = ig < n && jg < n && (!diag || jg <= ig);
+                            const bool ok = ig < n && jg < n && (!diag || jg <= ig) && fkeep;
                             p[e] = ok ? p[e] : 0.f;
                         }
                     }
@@ -422,7 +424,7 @@ constexpr int kThreadsFused = 512 + 256 + 128;  // 16 exp/dS warps, 8 reducer wa
 struct FusedRegs {
     static constexpr int kExp = 88, kReduce = 48, kIssue = 56;
 };
-template <int HD>
+template <int HD, bool FINE>
 __global__ void __launch_bounds__(kThreadsFused, 1)
 tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mK_,
                  const __grid_constant__ CUtensorMap mV, const __grid_constant__ CUtensorMap mdO,
@@ -672,8 +674,11 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
             const float4 *sNL = reinterpret_cast<const float4 *>(smem + L::oLSE + s * 512 + h * 256 + qq * 128);
             const float4 *sDs = reinterpret_cast<const float4 *>(smem + L::oD + s * 512 + h * 256 + qq * 128);
             const bool diag = mask_is_causal(a.mask_kind) && it == jt;
-            const bool masked = diag || i0 + TQ > n || j0 + TK > n;
             const int ig0 = i0 + h * 64 + qq * 32;
+            // fine blocks: this thread's 32 query columns and its key row lie in one block of the caller's mask
+            bool fkeep = true;
+            if constexpr (FINE) fkeep = ig0 < n && jg < n && fine_keep(a.fine, a.mask_heads, bh, ig0, jg);
+            const bool masked = diag || i0 + TQ > n || j0 + TK > n || FINE;
             mbar_wait(&bars[V2_QFULL + s], (k >> 1) & 1, ab);
             // the 32 row statistics of this thread's query columns go into registers before the wait for S^T: while the
             // products stream their operands, a shared-memory load inside the arithmetic below waits a few hundred cycles
@@ -701,7 +706,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const int ig = ig0 + q * 4 + e;
-                            const bool ok = ig < n && jg < n && (!diag || jg <= ig);
+                            const bool ok = ig < n && jg < n && (!diag || jg <= ig) && fkeep;
                             p[e] = ok ? p[e] : 0.f;
                         }
                     }
@@ -839,7 +844,7 @@ attn_status launch_bwd(const Problem &p)
     a.nLSE2 = p.nLSE2; a.Ds = p.D; a.dQ_acc = p.dQ_acc;
     a.dK = (__nv_bfloat16 *)p.dK; a.dV = (__nv_bfloat16 *)p.dV;
     a.n = p.n; a.BH = (int)p.BH;
-    a.mask_kind = p.mask_kind; a.block = p.block; a.nb = p.nb; a.mask_heads = p.mask_heads;
+    a.mask_kind = p.mask_kind; a.block = p.block; a.nb = p.nb; a.mask_heads = p.mask_heads; a.fine = p.fine;
     a.col_ptr = p.col_ptr; a.row_idx = p.row_idx;
     a.scale = p.scale;
     a.status = p.status;
@@ -849,11 +854,12 @@ attn_status launch_bwd(const Problem &p)
     launch_begin(WITH_DQ ? "tc_bwd_fused" : "tc_bwd_dkdv", p.stream);
     if (WITH_DQ) {
         constexpr uint32_t bytes = HD == 64 ? ((L::kBytes + 1023u) & ~1023u) + SLAB : L::kBytes;
-        if (cudaFuncSetAttribute(tc_bwd_fused_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
+        auto kernel = p.fine.block ? tc_bwd_fused_kernel<HD, true> : tc_bwd_fused_kernel<HD, false>;
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
             return ATTN_ERR_LAUNCH;
         CUtensorMap mdK, mdV;
         if (!make_tmap_bf16_3d(&mdK, p.dK, HD, p.n, BH, 128) || !make_tmap_bf16_3d(&mdV, p.dV, HD, p.n, BH, 128)) return ATTN_ERR_LAUNCH;
-        tc_bwd_fused_kernel<HD><<<grid, kThreadsFused, bytes, p.stream>>>(mQ, mK, mV, mdO, mdK, mdV, a);
+        kernel<<<grid, kThreadsFused, bytes, p.stream>>>(mQ, mK, mV, mdO, mdK, mdV, a);
     } else {
         if (cudaFuncSetAttribute(tc_bwd_dkdv_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DkdvSmem<HD>::kBytes) != cudaSuccess)
             return ATTN_ERR_LAUNCH;

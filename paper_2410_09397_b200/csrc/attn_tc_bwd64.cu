@@ -288,8 +288,10 @@ tc_bwd_fused64_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_const
             const float4 *sNL = reinterpret_cast<const float4 *>(smem + L::oLSE + s * 256 + g * 128);
             const float4 *sDs = reinterpret_cast<const float4 *>(smem + L::oD + s * 256 + g * 128);
             const bool diag = mask_is_causal(a.mask_kind) && i0 < j0 + TK;   // some (i, j) of the tile pair has j > i
-            const bool masked = diag || i0 + TQ64 > n || j0 + TK > n;
             const int ig0 = i0 + g * 32;
+            // fine blocks: this thread's 32 query columns and its key row lie in one block of the caller's mask
+            const bool fkeep = !a.fine.block || (ig0 < n && jg < n && fine_keep(a.fine, a.mask_heads, bh, ig0, jg));
+            const bool masked = diag || i0 + TQ64 > n || j0 + TK > n || a.fine.block != 0;
             mbar_wait(&bars[B_QFULL + s], (t / NS) & 1, ab);
             float4 nlr[8];
 #pragma unroll
@@ -313,7 +315,7 @@ tc_bwd_fused64_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_const
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const int ig = ig0 + q * 4 + e;
-                            const bool ok = ig < n && jg < n && (!diag || jg <= ig);
+                            const bool ok = ig < n && jg < n && (!diag || jg <= ig) && fkeep;
                             p[e] = ok ? p[e] : 0.f;
                         }
                     }
@@ -422,7 +424,7 @@ attn_status launch_bwd64(const Problem &p)
     a.nLSE2 = p.nLSE2; a.Ds = p.D; a.dQ_acc = p.dQ_acc;
     a.dK = (__nv_bfloat16 *)p.dK; a.dV = (__nv_bfloat16 *)p.dV;
     a.n = p.n; a.BH = (int)p.BH;
-    a.mask_kind = p.mask_kind; a.block = p.block; a.nb = p.nb; a.mask_heads = p.mask_heads;
+    a.mask_kind = p.mask_kind; a.block = p.block; a.nb = p.nb; a.mask_heads = p.mask_heads; a.fine = p.fine;
     a.col_ptr = p.col_ptr; a.row_idx = p.row_idx;
     a.scale = p.scale;
     a.status = p.status;

@@ -34,6 +34,7 @@ struct DqArgs {
     int n, BH;
     int mask_kind, block, nb, mask_heads;
     const int *row_ptr, *col_idx;
+    FineMask fine;
     float scale;
     uint32_t *status;
 };
@@ -242,7 +243,9 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
             if (jt < 0) continue;
             const int b = k & 1, j0 = jt * TKD + wg * 32;
             const uint32_t T_S = tm + b * 128;
-            const bool masked = (mask_is_causal(a.mask_kind) && jt * TKD + TKD - 1 > i0) || jt * TKD + TKD > n;
+            // fine blocks: this thread's query row and its 32 key columns lie in one block of the caller's mask
+            const bool fkeep = !a.fine.block || (ig < n && j0 < n && fine_keep(a.fine, a.mask_heads, bh, ig, j0));
+            const bool masked = (mask_is_causal(a.mask_kind) && jt * TKD + TKD - 1 > i0) || jt * TKD + TKD > n || a.fine.block != 0;
             mbar_wait(&bars[DB_S + b], (k >> 1) & 1, ab);
             tcgen05_fence_after();
             float p[32];
@@ -258,7 +261,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
 #pragma unroll
                 for (int e = 0; e < 32; ++e) {
                     const int jg = j0 + e;
-                    if (jg >= n || (causal && jg > ig)) p[e] = 0.f;
+                    if (jg >= n || (causal && jg > ig) || !fkeep) p[e] = 0.f;
                 }
             }
             mbar_wait(&bars[DB_DP], k & 1, ab);
@@ -332,7 +335,7 @@ attn_status launch_dq(const Problem &p)
     a.dQ = (__nv_bfloat16 *)p.dQ;
     a.nLSE2 = p.nLSE2; a.Ds = p.D;
     a.n = p.n; a.BH = (int)p.BH;
-    a.mask_kind = p.mask_kind; a.block = p.block; a.nb = p.nb; a.mask_heads = p.mask_heads;
+    a.mask_kind = p.mask_kind; a.block = p.block; a.nb = p.nb; a.mask_heads = p.mask_heads; a.fine = p.fine;
     a.row_ptr = p.row_ptr; a.col_idx = p.col_idx;
     a.scale = p.scale;
     a.status = p.status;

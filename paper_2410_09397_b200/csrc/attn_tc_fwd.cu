@@ -40,6 +40,7 @@ struct FwdArgs {
     int n, BH;
     int mask_kind, block, nb, mask_heads;
     const int *row_ptr, *col_idx;   // block-CSR of the mask
+    FineMask fine;                  // block edge below 128
     float scale;
     uint32_t *status;
 };
@@ -65,7 +66,7 @@ struct FwdCfg {
     static constexpr uint32_t kBytes = kUsed < 117 * 1024 ? 117 * 1024 : kUsed;
 };
 
-enum { FB_Q = 0, FB_KVFULL = 1, FB_KVEMPTY = 4, FB_S = 7, FB_P = 9, FB_O = 11 };
+enum { FB_Q = 0, FB_KVFULL = 1, FB_KVEMPTY = 4, FB_S = 7, FB_P = 9, FB_O = 11, FB_OLAST = 12 };
 
 template <int TKF>
 struct KeyIter {
@@ -143,6 +144,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
         for (int s = 0; s < NST; ++s) { mbar_init(&bars[FB_KVFULL + s], 1); mbar_init(&bars[FB_KVEMPTY + s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&bars[FB_S + b], 1); mbar_init(&bars[FB_P + b], kSoftmaxThreads); }
         mbar_init(&bars[FB_O], 1);
+        mbar_init(&bars[FB_OLAST], 1);
         fence_barrier_init();
         prefetch_tensormap(&mQ); prefetch_tensormap(&mK); prefetch_tensormap(&mV);
     }
@@ -212,6 +214,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
                     mma_ts_lo(T_O, tm + b * 128 + kk * 8, mV_ + kk * 128, idesc_o, (k > 0) || (kk > 0));
                 mma_commit(&bars[FB_KVEMPTY + s]);
                 mma_commit(&bars[FB_O]);
+                if (k + 1 == niter) mma_commit(&bars[FB_OLAST]);
             }
         }
     } else {
@@ -239,14 +242,17 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
 #pragma unroll
                 for (int e = 0; e < 32; ++e) sv[c + e] = __uint_as_float(v[e]);   // raw scores; scale * log2e enters below
             }
-            const bool need_mask = (mask_is_causal(a.mask_kind) && j0 + TKF - 1 > i0) || j0 + TKF > n;
+            const bool need_mask = (mask_is_causal(a.mask_kind) && j0 + TKF - 1 > i0) || j0 + TKF > n || a.fine.block != 0;
             float mx = -INFINITY;
             if (need_mask) {
                 const bool causal = mask_is_causal(a.mask_kind);
 #pragma unroll
                 for (int e = 0; e < CW; ++e) {
                     const int jg = j0 + wg * CW + e;
-                    if (jg >= n || (causal && jg > ig)) sv[e] = -INFINITY;
+                    bool drop = jg >= n || (causal && jg > ig);
+                    // fine blocks: the block of the caller's mask changes at most every 32 columns
+                    if (a.fine.block && !drop && ig < n) drop = !fine_keep(a.fine, a.mask_heads, bh, ig, jg);
+                    if (drop) sv[e] = -INFINITY;
                 }
             }
 #pragma unroll
@@ -303,7 +309,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
         named_bar_sync_f(1, kSoftmaxThreads);
         const float l_tot = xsum[row] + xsum[128 + row];
         if (k > 0) {
-            mbar_wait(&bars[FB_O], (k - 1) & 1, ab);
+            // FB_O completes once per tile and a parity wait tells two phases apart, not three: the last completion
+            // this thread knows of is S(k-1), queued before O += P V of tile k-2, so FB_O may be two completions
+            // behind the one needed here and a wait on it could pass at once.  The last product has a barrier of its own.
+            mbar_wait(&bars[FB_OLAST], 0, ab);
             tcgen05_fence_after();
         }
         const float inv = l_tot > 0.f ? 1.f / l_tot : 0.f;
@@ -353,7 +362,7 @@ enum { F2_Q = 0, F2_KFULL = 1, F2_KEMPTY = 4, F2_VFULL = 7, F2_VEMPTY = 10, F2_S
 // the softmax warpgroups take them (256 x 224 + 128 x 40 = 62,464 of the 384 x 168 = 64,512 the block holds), so
 // that a thread can keep its whole row of 128 scores.
 constexpr int kThreadsRows = kSoftmaxThreads + 128;
-template <int HD>
+template <int HD, bool FINE>
 __global__ void __launch_bounds__(kThreadsRows, 1)
 tc_fwd_rows_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CUtensorMap mK,
                    const __grid_constant__ CUtensorMap mV, const FwdArgs a)
@@ -491,7 +500,7 @@ tc_fwd_rows_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
             if ((k++ & 1) != w) continue;
             const int j0 = jt * TKF;
             const bool causal = mask_is_causal(a.mask_kind);
-            const bool need_mask = (causal && j0 + TKF - 1 > i0) || j0 + TKF > n;
+            const bool need_mask = (causal && j0 + TKF - 1 > i0) || j0 + TKF > n || FINE;
             mbar_wait(&bars[F2_S + w], cnt & 1, ab);
             tcgen05_fence_after();
             // the whole row of raw scores in registers: four loads in flight, one wait
@@ -500,10 +509,17 @@ tc_fwd_rows_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
             for (int c = 0; c < TKF; c += 32) tmem_ld32(T_S + lane_addr + c, *reinterpret_cast<uint32_t(*)[32]>(&v[c]));
             tmem_wait_ld();
             if (need_mask) {
+                // fine blocks: one flag per 32 key columns (the block of the caller's mask is 32 or 64 wide)
+                bool fk[TKF / 32];
+#pragma unroll
+                for (int q = 0; q < TKF / 32; ++q) {
+                    fk[q] = true;
+                    if constexpr (FINE) fk[q] = ig < n && j0 + q * 32 < n && fine_keep(a.fine, a.mask_heads, bh, ig, j0 + q * 32);
+                }
 #pragma unroll
                 for (int e = 0; e < TKF; ++e) {
                     const int jg = j0 + e;
-                    if (jg >= n || (causal && jg > ig)) v[e] = 0xff800000u;   // -inf
+                    if (jg >= n || (causal && jg > ig) || !fk[e / 32]) v[e] = 0xff800000u;   // -inf
                 }
             }
             float mx8[8];   // eight independent chains instead of one of 128 dependent maxima
@@ -611,13 +627,13 @@ attn_status launch_fwd(const Problem &p)
     FwdArgs a{};
     a.O = (__nv_bfloat16 *)p.Oout; a.LSE = p.LSEout;
     a.n = p.n; a.BH = (int)p.BH;
-    a.mask_kind = p.mask_kind; a.block = p.block; a.nb = p.nb; a.mask_heads = p.mask_heads;
+    a.mask_kind = p.mask_kind; a.block = p.block; a.nb = p.nb; a.mask_heads = p.mask_heads; a.fine = p.fine;
     a.row_ptr = p.row_ptr; a.col_idx = p.col_idx;
     a.scale = p.scale;
     a.status = p.status;
     void (*kernel)(CUtensorMap, CUtensorMap, CUtensorMap, FwdArgs);
     if constexpr (HD == 256) kernel = tc_fwd_kernel<HD>;
-    else kernel = tc_fwd_rows_kernel<HD>;
+    else kernel = p.fine.block ? tc_fwd_rows_kernel<HD, true> : tc_fwd_rows_kernel<HD, false>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kBytes) != cudaSuccess)
         return ATTN_ERR_LAUNCH;
     const dim3 grid((p.n + TQ - 1) / TQ, (unsigned)p.BH);
