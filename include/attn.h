@@ -85,8 +85,9 @@ typedef struct {
 /* Which algorithm runs.  The tile sizes play the role of the paper's cache size M.
  *   FUSED        large-cache regime (Appendix D): score tiles never leave the SM.
  *   MATERIALIZED small-cache regime (Appendix C): P, dP and dS are written to and
- *                re-read from device memory in tile_q x tile_k blocks, the head
- *                dimension walked in tile_d chunks (backward only; its forward is FUSED).
+ *                re-read from device memory in tile_q x tile_k blocks (tile_q 256 or 128,
+ *                tile_k 128, 64 or 32; default 256 x 128), the head dimension walked in
+ *                tile_d = 64 chunks (backward only; its forward is FUSED).
  *   SIMT         fp32 FMA kernels without tensor cores; the only choice for ATTN_F32.
  *   AUTO         ATTN_F32 -> SIMT; ATTN_BF16 -> FUSED.                              */
 typedef enum { ATTN_ALGO_AUTO = 0, ATTN_ALGO_FUSED = 1, ATTN_ALGO_MATERIALIZED = 2, ATTN_ALGO_SIMT = 3 } attn_algo;

@@ -331,6 +331,9 @@ int attn_supported_cfgs(int d, int dt, attn_cfg *out, int max_out)
             {128, 128, 0, ATTN_ALGO_FUSED},
             {128, 64, 0, ATTN_ALGO_FUSED},
             {64, 128, 0, ATTN_ALGO_FUSED},
+            {256, 128, 64, ATTN_ALGO_MATERIALIZED},   // the first entry of an algorithm is its default
+            {256, 64, 64, ATTN_ALGO_MATERIALIZED},
+            {256, 32, 64, ATTN_ALGO_MATERIALIZED},
             {128, 128, 64, ATTN_ALGO_MATERIALIZED},
             {128, 64, 64, ATTN_ALGO_MATERIALIZED},
             {128, 32, 64, ATTN_ALGO_MATERIALIZED},

@@ -69,14 +69,14 @@ Count prepass(int n, int d, int with_acc)
     return c;
 }
 
-// blocked GEMM of the materialised path: C (m x nn) in 128 x bn tiles, contraction of length k
-Count gemm(double m, double nn, double k, int bn)
+// blocked GEMM of the materialised path: C (m x nn) in bm x bn tiles, contraction of length k
+Count gemm(double m, double nn, double k, int bm, int bn)
 {
     Count c;
-    const int tm = (int)((m + 127) / 128), tn = (int)((nn + bn - 1) / bn);
+    const int tm = (int)((m + bm - 1) / bm), tn = (int)((nn + bn - 1) / bn);
     for (int i = 0; i < tm; ++i)
         for (int j = 0; j < tn; ++j) {
-            const double rm = m - i * 128 < 128 ? m - i * 128 : 128, rn = nn - j * bn < bn ? nn - j * bn : bn;
+            const double rm = m - i * bm < bm ? m - i * bm : bm, rn = nn - j * bn < bn ? nn - j * bn : bn;
             c.loads += (rm + rn) * k;
             c.stores += rm * rn;
         }
@@ -108,12 +108,12 @@ extern "C" attn_status attn_io_replay(int n, int d, int mask_kind, int dt, const
     if (!backward) {
         r = query_stationary(n, d, causal, d == 256 ? 64 : 128, 0);
     } else if (c.algo == ATTN_ALGO_MATERIALIZED) {
-        const int tk = c.tile_k ? c.tile_k : 128;
+        const int tk = c.tile_k ? c.tile_k : 128, tq = c.tile_q ? c.tile_q : 128;
         r = prepass(n, d, 0);
-        r.add(gemm(n, n, d, tk));                                    // phase 1: P
-        r.add(gemm(n, n, d, tk));                                    // phase 2: dP
+        r.add(gemm(n, n, d, tq, tk));                                // phase 1: P
+        r.add(gemm(n, n, d, tq, tk));                                // phase 2: dP
         r.loads += 2.0 * n * n; r.stores += (double)n * n;           // phase 3: dS from P, dP
-        for (int i = 0; i < 3; ++i) r.add(gemm(n, d, n, d));         // phase 4: dV, dK, dQ
+        for (int i = 0; i < 3; ++i) r.add(gemm(n, d, n, 256, d));    // phase 4: dV, dK, dQ in 256 x d tiles
     } else if (c.deterministic) {
         r = prepass(n, d, 0);
         r.add(key_stationary(n, d, causal, 128, 1, 0));

@@ -11,12 +11,19 @@
 //   phase 3  dS = scale P o (dP - D)          streaming pass: reads P, dP, writes dS
 //   phase 4  dV = P^T dO, dK = dS^T Q, dQ = dS K     blocked GEMMs over n reading P / dS
 //
-// One GEMM kernel serves all products: a CTA computes a 128 x BN tile of C with fp32
-// accumulators in tensor memory; a TMA producer warp and an MMA issuer warp run a
-// 4-stage ring of 64-deep operand chunks; four warps run the epilogue.  Operands are
-// taken K-major or MN-major straight from their row-major arrays (no transposes).
+// One persistent GEMM kernel serves all products.  A CTA walks a strided list of 128 x BN
+// tiles of C (tile t = blockIdx.x + i gridDim.x; the column tile runs fastest, so the CTAs
+// that run together share their A rows in L2).  Per tile: a TMA producer thread and an MMA
+// issuing thread run a ring of 64-deep operand chunks into one of TWO fp32 accumulators in
+// tensor memory; eight epilogue warps turn the other accumulator into bf16 (exp / plain),
+// write it into a swizzled staging tile in shared memory and hand it to a TMA store, so
+// that the epilogue of tile i and its store run under the products of tile i + 1.  Operands
+// are taken K-major or MN-major straight from their row-major arrays (no transposes).
 #include "attn_internal.h"
+#include "tc_bwd_common.cuh"
 #include "tc_common.cuh"
+
+#include <type_traits>
 
 namespace attn {
 namespace {
@@ -24,29 +31,38 @@ namespace {
 using namespace tc;
 
 enum { EPI_EXP = 0, EPI_PLAIN = 1, EPI_OUT = 2 };
-constexpr int kStages = 4;
-constexpr int kGemmThreads = 192;
+constexpr int kEpiWarps = 8;
+constexpr int kGemmThreads = kEpiWarps * 32 + 64;   // epilogue warps, TMA producer warp, MMA issuer warp
 
 struct GemmArgs {
-    __nv_bfloat16 *C;        // output base (head 0 of this launch)
-    size_t c_head_stride;    // elements between heads of C
-    int ldc;                 // row pitch of C in elements
+    int heads;               // of this launch
     int m_total, n_total;    // valid rows / cols of C per head
     int k_total;             // contraction length
     const float *nlse2;      // EPI_EXP: -LSE log2e per row [heads][m_total]
     float sl2;               // EPI_EXP: scale * log2e
-    int causal;              // EPI_EXP: zero entries with col > row
+    int causal;              // EPI_EXP: entries with col > row are zero; tiles wholly above the diagonal skip the product
     uint32_t *status;
 };
 
-template <int BN>
+// BN: columns of a tile; MT: 128-row sub-tiles of a tile (1 or 2).  MT = 2 forms a 256 x BN tile in two accumulators
+// that share every B chunk (less operand traffic than two separate 128-row tiles).  Tensor memory holds two sets of
+// MT accumulators that alternate between tiles where 2 MT BN <= 512 columns, else one set.
+template <int BN, int MT>
 struct GemmSmem {
-    static constexpr uint32_t kA = 128 * 128;           // 128 x 64 bf16 (either major)
-    static constexpr uint32_t kB = BN * 128;            // BN x 64 bf16
+    static constexpr int OUTW = BN < 128 ? BN : 128;     // columns of one staging step
+    static constexpr int kOutBufs = MT * BN >= 512 ? 1 : 2;
+    static constexpr int NBUF = 2 * MT * BN <= 512 ? 2 : 1;   // accumulator sets
+    static constexpr uint32_t kA = MT * 128 * 128;       // MT x 128 x 64 bf16 (either major)
+    static constexpr uint32_t kB = BN * 128;             // BN x 64 bf16
     static constexpr uint32_t kStage = kA + kB;
-    static constexpr uint32_t oBar = kStages * kStage;
+    static constexpr uint32_t kOut = 128 * OUTW * 2;     // staging: [128][64] slabs, 128-byte swizzle (OUTW = 32: [128][32], 64-byte swizzle)
+    static constexpr int kStages = (227 * 1024 - 1024 - kOutBufs * (int)kOut) / (int)kStage < 4 ? (227 * 1024 - 1024 - kOutBufs * (int)kOut) / (int)kStage : 4;
+    static constexpr uint32_t oOut = kStages * kStage;
+    static constexpr uint32_t oBar = oOut + kOutBufs * kOut;
     static constexpr uint32_t oMisc = oBar + 16 * 8;
     static constexpr uint32_t kBytes = oMisc + 64;
+    static_assert(kStages >= 3 && kBytes <= 227 * 1024 && kStage % 1024 == 0 && kOut % 1024 == 0, "shared memory layout");
+    static_assert(NBUF * MT * BN <= 512, "tensor memory");
 };
 
 __device__ __forceinline__ float ex2a(float x)
@@ -56,24 +72,40 @@ __device__ __forceinline__ float ex2a(float x)
     return y;
 }
 
-// A_MN: A is stored [k][m] (m contiguous); otherwise [m][k].  B_MN: B stored [k][n]; otherwise [n][k].
-template <int BN, bool A_MN, bool B_MN, int EPI>
-__global__ void __launch_bounds__(kGemmThreads)
-mat_gemm_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ CUtensorMap mB, const GemmArgs g)
+// byte offset of (row, col) in a staging tile of W columns, as the TMA store reads it
+template <int W>
+__device__ __forceinline__ uint32_t stage_offset(uint32_t row, uint32_t col)
 {
-    using L = GemmSmem<BN>;
+    if constexpr (W >= 64) return (col / 64) * (128u * 128u) + sw128_offset(row, col % 64);
+    else return row * 64u + ((((col >> 3) ^ ((row >> 1) & 3u)) << 4) | ((col & 7u) << 1));   // 64-byte swizzle
+}
+
+// A_MN: A is stored [k][m] (m contiguous); otherwise [m][k].  B_MN: B stored [k][n]; otherwise [n][k].
+template <int BN, int MT, bool A_MN, bool B_MN, int EPI>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+mat_gemm_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ CUtensorMap mB,
+                const __grid_constant__ CUtensorMap mC, const GemmArgs g)
+{
+    using L = GemmSmem<BN, MT>;
+    constexpr int kStages = L::kStages, kOutBufs = L::kOutBufs, OUTW = L::OUTW;
+    constexpr int NBUF = L::NBUF;            // accumulator sets that alternate between tiles
+    constexpr int TM = 128 * MT;
     extern __shared__ __align__(1024) uint8_t smem[];
     uint64_t *full = reinterpret_cast<uint64_t *>(smem + L::oBar);
     uint64_t *empty = full + kStages;
-    uint64_t *done = empty + kStages;
+    uint64_t *accfull = empty + kStages;
+    uint64_t *accempty = accfull + 2;
     uint32_t *tmem_base_s = reinterpret_cast<uint32_t *>(smem + L::oMisc);
     volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(smem + L::oMisc + 4);
     const Abort ab{abort_flag, g.status};
-    constexpr uint32_t kTmemCols = BN < 32 ? 32 : BN;
+    constexpr uint32_t kTmemCols = NBUF * MT * BN < 32 ? 32 : NBUF * MT * BN;
 
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
-    const int n0 = blockIdx.x * BN, m0 = blockIdx.y * 128, head = blockIdx.z;
+    const int tiles_n = (g.n_total + BN - 1) / BN, tiles_m = (g.m_total + TM - 1) / TM;
+    const long total = (long)tiles_n * tiles_m * g.heads;
     const int nk = (g.k_total + 63) / 64;
+    // the product of a tile that lies wholly above the diagonal is not formed (its entries are exact zeros)
+    auto skipped = [&](int m0, int n0) { return EPI == EPI_EXP && g.causal && n0 > m0 + TM - 1; };
 
     if ((smem_u32(smem) & 1023u) != 0) {
         if (tid == 0) atomicExch(g.status, 9u);
@@ -82,9 +114,9 @@ mat_gemm_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ 
     if (tid == 0) {
         *abort_flag = 0;
         for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        mbar_init(done, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(&accfull[b], 1); mbar_init(&accempty[b], kEpiWarps); }
         fence_barrier_init();
-        prefetch_tensormap(&mA); prefetch_tensormap(&mB);
+        prefetch_tensormap(&mA); prefetch_tensormap(&mB); prefetch_tensormap(&mC);
     }
     if (warp == 0) tmem_alloc(tmem_base_s, kTmemCols);
     tcgen05_fence_before();
@@ -92,80 +124,148 @@ mat_gemm_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ 
     tcgen05_fence_after();
     const uint32_t tm = *tmem_base_s;
 
-    if (warp == 4) {
+    if (warp == kEpiWarps) {
+        // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            for (int kt = 0; kt < nk; ++kt) {
-                const int s = kt % kStages;
-                if (kt >= kStages) mbar_wait(&empty[s], ((kt / kStages) - 1) & 1, ab);
-                uint8_t *sA = smem + s * L::kStage, *sB = sA + L::kA;
-                mbar_expect_tx(&full[s], L::kStage);
-                if (A_MN) {
-                    tma_load_3d(sA, &mA, &full[s], m0, kt * 64, head);
-                    tma_load_3d(sA + 8192, &mA, &full[s], m0 + 64, kt * 64, head);
-                } else {
-                    tma_load_3d(sA, &mA, &full[s], kt * 64, m0, head);
-                }
-                if (B_MN) {
+            int kc = 0;   // chunks loaded so far, over all tiles
+            for (long t = blockIdx.x; t < total; t += gridDim.x) {
+                const int head = (int)(t / ((long)tiles_n * tiles_m));
+                const int m0 = (int)(t / tiles_n % tiles_m) * TM, n0 = (int)(t % tiles_n) * BN;
+                if (skipped(m0, n0)) continue;
+                for (int kt = 0; kt < nk; ++kt, ++kc) {
+                    const int s = kc % kStages;
+                    if (kc >= kStages) mbar_wait(&empty[s], ((kc / kStages) - 1) & 1, ab);
+                    uint8_t *sA = smem + s * L::kStage, *sB = sA + L::kA;
+                    mbar_expect_tx(&full[s], L::kStage);
+                    if (A_MN) {
 #pragma unroll
-                    for (int sl = 0; sl < BN / 64; ++sl) tma_load_3d(sB + sl * 8192, &mB, &full[s], n0 + sl * 64, kt * 64, head);
-                } else {
-                    tma_load_3d(sB, &mB, &full[s], kt * 64, n0, head);
-                }
-            }
-        }
-    } else if (warp == 5) {
-        if (lane == 0) {
-            constexpr uint32_t idesc = idesc_bf16(128, BN, A_MN ? 1 : 0, B_MN ? 1 : 0);
-            for (int kt = 0; kt < nk; ++kt) {
-                const int s = kt % kStages;
-                mbar_wait(&full[s], (kt / kStages) & 1, ab);
-                tcgen05_fence_after();
-                const uint32_t sA = smem_u32(smem + s * L::kStage), sB = sA + L::kA;
+                        for (int q = 0; q < 2 * MT; ++q) tma_load_3d(sA + q * 8192, &mA, &full[s], m0 + q * 64, kt * 64, head);
+                    } else {
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks) {
-                    const uint64_t da = A_MN ? smem_desc_mnmajor(sA + ks * 2048, 8192) : smem_desc_kmajor(sA + ks * 32);
-                    const uint64_t db = B_MN ? smem_desc_mnmajor(sB + ks * 2048, 8192) : smem_desc_kmajor(sB + ks * 32);
-                    mma_ss(tm, da, db, idesc, (kt > 0) || (ks > 0));
-                }
-                mma_commit(&empty[s]);
-            }
-            mma_commit(done);
-        }
-    } else {
-        // ------------------------------------------------------------ epilogue (warps 0-3)
-        const int row = warp * 32 + lane, gi = m0 + row;
-        const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
-        mbar_wait(done, 0, ab);
-        tcgen05_fence_after();
-        const bool row_ok = gi < g.m_total;
-        __nv_bfloat16 *crow = g.C + (size_t)head * g.c_head_stride + (size_t)(row_ok ? gi : 0) * g.ldc + n0;
-        float nl = 0.f;
-        if (EPI == EPI_EXP && row_ok) nl = g.nlse2[(size_t)head * g.m_total + gi];
-        constexpr int CH = BN < 32 ? BN : 32;
-#pragma unroll 1
-        for (int c = 0; c < BN; c += CH) {
-            uint32_t v[32];
-            if (CH == 32) tmem_ld32(tm + lane_addr + c, v);
-            else tmem_ld16(tm + lane_addr + c, *reinterpret_cast<uint32_t(*)[16]>(v));
-            tmem_wait_ld();
-            if (!row_ok) continue;
+                        for (int q = 0; q < MT; ++q) tma_load_3d(sA + q * 16384, &mA, &full[s], kt * 64, m0 + q * 128, head);
+                    }
+                    if (B_MN) {
 #pragma unroll
-            for (int e = 0; e < CH; e += 8) {
-                const int gj = n0 + c + e;
-                if (gj >= g.n_total) break;
-                float x[8];
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    x[u] = __uint_as_float(v[e + u]);
-                    if (EPI == EPI_EXP) {
-                        x[u] = ex2a(fmaf(x[u], g.sl2, nl));
-                        if (g.causal && gj + u > gi) x[u] = 0.f;
+                        for (int sl = 0; sl < BN / 64; ++sl) tma_load_3d(sB + sl * 8192, &mB, &full[s], n0 + sl * 64, kt * 64, head);
+                    } else {
+                        tma_load_3d(sB, &mB, &full[s], kt * 64, n0, head);
                     }
                 }
-                *reinterpret_cast<uint4 *>(crow + c + e) =
-                    make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]), pack_bf16(x[4], x[5]), pack_bf16(x[6], x[7]));
             }
         }
+    } else if (warp == kEpiWarps + 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = idesc_bf16(128, BN, A_MN ? 1 : 0, B_MN ? 1 : 0);
+            int kc = 0, ai = 0;   // chunks consumed; accumulator sets filled
+            for (long t = blockIdx.x; t < total; t += gridDim.x) {
+                const int m0 = (int)(t / tiles_n % tiles_m) * TM, n0 = (int)(t % tiles_n) * BN;
+                if (skipped(m0, n0)) continue;
+                const int b = ai % NBUF;
+                if (ai >= NBUF) {   // the epilogue has read the tile that used this accumulator set before
+                    mbar_wait(&accempty[b], ((ai / NBUF) - 1) & 1, ab);
+                    tcgen05_fence_after();
+                }
+                for (int kt = 0; kt < nk; ++kt, ++kc) {
+                    const int s = kc % kStages;
+                    mbar_wait(&full[s], (kc / kStages) & 1, ab);
+                    tcgen05_fence_after();
+                    const uint32_t sA = smem_u32(smem + s * L::kStage), sB = sA + L::kA;
+                    const uint32_t db = B_MN ? desc_lo_mnmajor(sB, 8192) : desc_lo_kmajor(sB);
+#pragma unroll
+                    for (int q = 0; q < MT; ++q) {
+                        const uint32_t da = A_MN ? desc_lo_mnmajor(sA + q * 16384, 8192) : desc_lo_kmajor(sA + q * 16384);
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks)
+                            mma_ss_lo(tm + (b * MT + q) * BN, da + ks * (A_MN ? 128 : 2), db + ks * (B_MN ? 128 : 2), idesc,
+                                      (kt > 0) || (ks > 0));
+                    }
+                    mma_commit(&empty[s]);
+                }
+                mma_commit(&accfull[b]);
+                ++ai;
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 0-7): a tile leaves in steps of
+        // 128 rows x OUTW columns; in every step warp w takes the lane quarter w % 4 (its rows) and the column half w / 4
+        constexpr int CW = OUTW / 2, CH = CW < 32 ? CW : 32;
+        const int row = (warp % 4) * 32 + lane, c_first = (warp / 4) * CW;
+        const uint32_t lane_addr = (uint32_t)((warp % 4) * 32) << 16;
+        int ai = 0, oi = 0;   // accumulator sets read; staging tiles written
+        for (long t = blockIdx.x; t < total; t += gridDim.x) {
+            const int head = (int)(t / ((long)tiles_n * tiles_m));
+            const int m0 = (int)(t / tiles_n % tiles_m) * TM, n0 = (int)(t % tiles_n) * BN;
+            const bool skip = skipped(m0, n0);
+            const int b = ai % NBUF;
+            // the row statistics of this thread's rows are fetched before the wait for the products, which hides the load
+            float nlq[MT];
+#pragma unroll
+            for (int q = 0; q < MT; ++q) {
+                nlq[q] = 0.f;
+                if (EPI == EPI_EXP && m0 + q * 128 + row < g.m_total) nlq[q] = g.nlse2[(size_t)head * g.m_total + m0 + q * 128 + row];
+            }
+            if (!skip) {
+                mbar_wait(&accfull[b], (ai / NBUF) & 1, ab);
+                tcgen05_fence_after();
+            }
+#pragma unroll 1
+            for (int step = 0; step < MT * (BN / OUTW); ++step, ++oi) {
+                const int q = step / (BN / OUTW), cb = (step % (BN / OUTW)) * OUTW;   // row sub-tile, first column
+                const int gi = m0 + q * 128 + row;
+                const uint32_t acc = tm + lane_addr + (b * MT + q) * BN + cb + c_first;
+                uint8_t *stage = smem + L::oOut + (oi % kOutBufs) * L::kOut;
+                const float nl = MT == 1 ? nlq[0] : (q == 0 ? nlq[0] : nlq[MT - 1]);
+                // the store that last read this staging tile is done with it
+                if (tid == 0) {
+                    if (kOutBufs == 1) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                    else asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                }
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+#pragma unroll
+                for (int c = 0; c < CW; c += CH) {
+                    uint32_t v[32];
+                    if (!skip) {
+                        if constexpr (CH == 32) tmem_ld32(acc + c, v);
+                        else tmem_ld16(acc + c, *reinterpret_cast<uint32_t(*)[16]>(v));
+                        tmem_wait_ld();
+                    }
+#pragma unroll
+                    for (int e = 0; e < CH; e += 8) {
+                        const int gj = n0 + cb + c_first + c + e;
+                        float x[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            x[u] = skip ? 0.f : __uint_as_float(v[e + u]);
+                            if (EPI == EPI_EXP) {
+                                x[u] = ex2a(fmaf(x[u], g.sl2, nl));
+                                if (skip || (g.causal && gj + u > gi)) x[u] = 0.f;
+                            }
+                        }
+                        *reinterpret_cast<uint4 *>(stage + stage_offset<OUTW>(row, c_first + c + e)) =
+                            make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]), pack_bf16(x[4], x[5]), pack_bf16(x[6], x[7]));
+                    }
+                }
+                if (!skip && step + 1 == MT * (BN / OUTW)) {   // the accumulator set may take its next tile
+                    tcgen05_fence_before();
+                    bwdk::warp_arrive(&accempty[b], lane);
+                }
+                fence_proxy_async_smem();
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                if (tid == 0 && !*abort_flag) {
+                    // rows beyond m_total and columns beyond n_total are clipped by the store
+                    if constexpr (OUTW >= 64) {
+#pragma unroll
+                        for (int sl = 0; sl < OUTW / 64; ++sl) tma_store_3d(&mC, stage + sl * 16384, n0 + cb + sl * 64, m0 + q * 128, head);
+                    } else {
+                        tma_store_3d(&mC, stage, n0 + cb, m0 + q * 128, head);
+                    }
+                    tma_store_commit();
+                }
+            }
+            if (!skip) ++ai;
+        }
+        if (tid == 0) tma_store_wait_all();
     }
     tcgen05_fence_before();
     __syncthreads();
@@ -193,56 +293,34 @@ __global__ void __launch_bounds__(256) mat_ds_kernel(const uint4 *__restrict__ P
     }
 }
 
-// D pre-pass for d = 256: Ds = scale * rowsum(dO o O), nlse2 = -LSE log2e (one warp per row)
-__global__ void __launch_bounds__(256) mat_preprocess_kernel(const __nv_bfloat16 *__restrict__ O,
-                                                             const __nv_bfloat16 *__restrict__ dO,
-                                                             const float *__restrict__ LSE, float *__restrict__ Ds,
-                                                             float *__restrict__ nlse2, size_t rows, int d, float scale)
-{
-    const int lane = threadIdx.x % 32;
-    const size_t warp = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) / 32;
-    const size_t nwarps = (size_t)gridDim.x * blockDim.x / 32;
-    const int vec = d / 8;
-    for (size_t row = warp; row < rows; row += nwarps) {
-        float acc = 0.f;
-        for (int v = lane; v < vec; v += 32) {
-            const uint4 xo = __ldg(reinterpret_cast<const uint4 *>(O + row * d) + v);
-            const uint4 xg = __ldg(reinterpret_cast<const uint4 *>(dO + row * d) + v);
-            const __nv_bfloat162 *eo = reinterpret_cast<const __nv_bfloat162 *>(&xo);
-            const __nv_bfloat162 *eg = reinterpret_cast<const __nv_bfloat162 *>(&xg);
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float2 fo = __bfloat1622float2(eo[e]), fg = __bfloat1622float2(eg[e]);
-                acc = fmaf(fo.x, fg.x, acc);
-                acc = fmaf(fo.y, fg.y, acc);
-            }
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-        if (lane == 0) {
-            Ds[row] = acc * scale;
-            const float l = LSE[row];
-            nlse2[row] = l == -INFINITY ? -INFINITY : -l * 1.4426950408889634f;
-        }
-    }
-}
-
-template <int BN, bool A_MN, bool B_MN, int EPI>
-attn_status launch_gemm(const char *name, const CUtensorMap &mA, const CUtensorMap &mB, const GemmArgs &g, int heads,
+// C: [heads][m_total][n_total] bf16, rows `ldc` elements apart, heads m_total * ldc elements apart
+template <int BN, int MT, bool A_MN, bool B_MN, int EPI>
+attn_status launch_gemm(const char *name, const CUtensorMap &mA, const CUtensorMap &mB, void *C, int ldc, GemmArgs g, int heads,
                         cudaStream_t s)
 {
-    using L = GemmSmem<BN>;
-    auto kernel = mat_gemm_kernel<BN, A_MN, B_MN, EPI>;
+    using L = GemmSmem<BN, MT>;
+    auto kernel = mat_gemm_kernel<BN, MT, A_MN, B_MN, EPI>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::kBytes) != cudaSuccess)
         return ATTN_ERR_LAUNCH;
-    const dim3 grid((g.n_total + BN - 1) / BN, (g.m_total + 127) / 128, heads);
+    CUtensorMap mC;
+    if (!make_tmap_bf16_3d_box(&mC, C, (uint64_t)g.n_total, (uint64_t)g.m_total, (uint64_t)heads, (uint64_t)ldc, BN < 64 ? BN : 64, 128,
+                               BN < 64 ? 64 : 128))
+        return ATTN_ERR_LAUNCH;
+    g.heads = heads;
+    const long total = (long)((g.n_total + BN - 1) / BN) * ((g.m_total + 128 * MT - 1) / (128 * MT)) * heads;
+    // as many CTAs per SM as fit (registers, shared memory; 2 BN tensor-memory columns each): every CTA is resident
+    int per_sm = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kGemmThreads, L::kBytes) != cudaSuccess || per_sm < 1) per_sm = 1;
+    if (per_sm > 512 / (L::NBUF * MT * BN)) per_sm = 512 / (L::NBUF * MT * BN);
+    if (per_sm > 2) per_sm = 2;
+    const long ctas = (long)sm_count() * per_sm;
     launch_begin(name, s);
-    kernel<<<grid, kGemmThreads, L::kBytes, s>>>(mA, mB, g);
+    kernel<<<(unsigned)(total < ctas ? total : ctas), kGemmThreads, L::kBytes, s>>>(mA, mB, mC, g);
     launch_end(s);
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_LAUNCH;
 }
 
-template <int TK>
+template <int TK, int MT>
 attn_status run_scores(const Problem &p, size_t h0, int mh)
 {
     const int n = p.n, d = p.d;
@@ -253,25 +331,30 @@ attn_status run_scores(const Problem &p, size_t h0, int mh)
         !make_tmap_bf16_3d(&mK, K, d, n, mh, TK) || !make_tmap_bf16_3d(&mV, V, d, n, mh, TK))
         return ATTN_ERR_LAUNCH;
     GemmArgs g{};
-    g.c_head_stride = (size_t)n * n; g.ldc = n; g.m_total = n; g.n_total = n; g.k_total = d;
+    g.m_total = n; g.n_total = n; g.k_total = d;
     g.status = p.status;
     // phase 1: P = exp(scale Q K^T - LSE)
-    g.C = (__nv_bfloat16 *)p.matP;
     g.nlse2 = p.nLSE2 + h0 * n; g.sl2 = p.scale * 1.4426950408889634f; g.causal = p.mask_kind == ATTN_MASK_CAUSAL;
-    attn_status st = launch_gemm<TK, false, false, EPI_EXP>("mat_phase1_P", mQ, mK, g, mh, p.stream);
+    attn_status st = launch_gemm<TK, MT, false, false, EPI_EXP>("mat_phase1_P", mQ, mK, p.matP, n, g, mh, p.stream);
     if (st != ATTN_OK) return st;
     // phase 2: dP = dO V^T
-    g.C = (__nv_bfloat16 *)p.matdP; g.causal = 0;
-    return launch_gemm<TK, false, false, EPI_PLAIN>("mat_phase2_dP", mdO, mV, g, mh, p.stream);
+    g.causal = 0;
+    return launch_gemm<TK, MT, false, false, EPI_PLAIN>("mat_phase2_dP", mdO, mV, p.matdP, n, g, mh, p.stream);
 }
 
 attn_status run_chunk(const Problem &p, size_t h0, int mh)
 {
     const int n = p.n, d = p.d;
     attn_status st;
-    if (p.cfg.tile_k == 128) st = run_scores<128>(p, h0, mh);
-    else if (p.cfg.tile_k == 64) st = run_scores<64>(p, h0, mh);
-    else st = run_scores<32>(p, h0, mh);
+    if (p.cfg.tile_q == 256) {
+        if (p.cfg.tile_k == 128) st = run_scores<128, 2>(p, h0, mh);
+        else if (p.cfg.tile_k == 64) st = run_scores<64, 2>(p, h0, mh);
+        else st = run_scores<32, 2>(p, h0, mh);
+    } else {
+        if (p.cfg.tile_k == 128) st = run_scores<128, 1>(p, h0, mh);
+        else if (p.cfg.tile_k == 64) st = run_scores<64, 1>(p, h0, mh);
+        else st = run_scores<32, 1>(p, h0, mh);
+    }
     if (st != ATTN_OK) return st;
     // phase 3: dS = scale P o (dP - D)
     {
@@ -293,59 +376,51 @@ attn_status run_chunk(const Problem &p, size_t h0, int mh)
         !make_tmap_bf16_3d(&mK, K, d, n, mh, 64) || !make_tmap_bf16_3d(&mdO, dO, d, n, mh, 64))
         return ATTN_ERR_LAUNCH;
     GemmArgs g{};
-    g.c_head_stride = (size_t)n * d; g.ldc = d; g.m_total = n; g.n_total = d; g.k_total = n;
+    g.m_total = n; g.n_total = d; g.k_total = n;
     g.status = p.status;
-    g.C = (__nv_bfloat16 *)p.dV + h0 * n * d;
-    if (d == 256) {
-        if ((st = launch_gemm<256, true, true, EPI_OUT>("mat_phase4_dV", mPt, mdO, g, mh, p.stream)) != ATTN_OK) return st;
-        g.C = (__nv_bfloat16 *)p.dK + h0 * n * d;
-        if ((st = launch_gemm<256, true, true, EPI_OUT>("mat_phase4_dK", mdSt, mQ, g, mh, p.stream)) != ATTN_OK) return st;
-        g.C = (__nv_bfloat16 *)p.dQ + h0 * n * d;
-        return launch_gemm<256, false, true, EPI_OUT>("mat_phase4_dQ", mdS, mK, g, mh, p.stream);
-    } else if (d == 128) {
-        if ((st = launch_gemm<128, true, true, EPI_OUT>("mat_phase4_dV", mPt, mdO, g, mh, p.stream)) != ATTN_OK) return st;
-        g.C = (__nv_bfloat16 *)p.dK + h0 * n * d;
-        if ((st = launch_gemm<128, true, true, EPI_OUT>("mat_phase4_dK", mdSt, mQ, g, mh, p.stream)) != ATTN_OK) return st;
-        g.C = (__nv_bfloat16 *)p.dQ + h0 * n * d;
-        return launch_gemm<128, false, true, EPI_OUT>("mat_phase4_dQ", mdS, mK, g, mh, p.stream);
-    }
-    if ((st = launch_gemm<64, true, true, EPI_OUT>("mat_phase4_dV", mPt, mdO, g, mh, p.stream)) != ATTN_OK) return st;
-    g.C = (__nv_bfloat16 *)p.dK + h0 * n * d;
-    if ((st = launch_gemm<64, true, true, EPI_OUT>("mat_phase4_dK", mdSt, mQ, g, mh, p.stream)) != ATTN_OK) return st;
-    g.C = (__nv_bfloat16 *)p.dQ + h0 * n * d;
-    return launch_gemm<64, false, true, EPI_OUT>("mat_phase4_dQ", mdS, mK, g, mh, p.stream);
+    __nv_bfloat16 *dV = (__nv_bfloat16 *)p.dV + h0 * n * d, *dK = (__nv_bfloat16 *)p.dK + h0 * n * d,
+                  *dQ = (__nv_bfloat16 *)p.dQ + h0 * n * d;
+    auto phase4 = [&](auto bn) -> attn_status {
+        constexpr int BN = decltype(bn)::value;
+        attn_status r;
+        if ((r = launch_gemm<BN, 2, true, true, EPI_OUT>("mat_phase4_dV", mPt, mdO, dV, d, g, mh, p.stream)) != ATTN_OK) return r;
+        if ((r = launch_gemm<BN, 2, true, true, EPI_OUT>("mat_phase4_dK", mdSt, mQ, dK, d, g, mh, p.stream)) != ATTN_OK) return r;
+        return launch_gemm<BN, 2, false, true, EPI_OUT>("mat_phase4_dQ", mdS, mK, dQ, d, g, mh, p.stream);
+    };
+    if (d == 256) return phase4(std::integral_constant<int, 256>{});
+    if (d == 128) return phase4(std::integral_constant<int, 128>{});
+    return phase4(std::integral_constant<int, 64>{});
 }
 
 }  // namespace
 
-// tile_q = 128; tile_k in {128, 64, 32} is the block edge of the n x n matrices in phases
-// 1 and 2; tile_d = 64 is the chunk in which every contraction is walked.
+// tile_q in {128, 256} x tile_k in {128, 64, 32} is the block of the n x n matrices in phases 1 and 2;
+// tile_d = 64 is the chunk in which every contraction is walked.  Phase 4 always forms 256 x d tiles.
 bool mat_cfg_supported(int d, const attn_cfg &c)
 {
     if (d != 64 && d != 128 && d != 256) return false;
-    if (c.tile_q != 0 && c.tile_q != 128) return false;
+    if (c.tile_q != 0 && c.tile_q != 128 && c.tile_q != 256) return false;
     if (c.tile_k != 0 && c.tile_k != 128 && c.tile_k != 64 && c.tile_k != 32) return false;
     return c.tile_d == 0 || c.tile_d == 64;
 }
 
-// On-chip bytes of a phase-1/2 CTA: operand ring + fp32 accumulator tile in tensor memory.
+// On-chip bytes of a phase-1/2 CTA: operand ring + fp32 accumulator tiles in tensor memory + staging tiles of C.
+template <int BN, int MT> constexpr size_t gemm_onchip()
+{
+    using L = GemmSmem<BN, MT>;
+    return (size_t)L::kStages * L::kStage + (size_t)L::kOutBufs * L::kOut + (size_t)L::NBUF * MT * BN * 128 * 4;
+}
 size_t mat_onchip_bytes(int, const attn_cfg &c)
 {
     const int tk = c.tile_k ? c.tile_k : 128;
-    return (size_t)kStages * (128 * 128 + tk * 128) + (size_t)128 * tk * 4;
+    if (c.tile_q == 256) return tk == 128 ? gemm_onchip<128, 2>() : tk == 64 ? gemm_onchip<64, 2>() : gemm_onchip<32, 2>();
+    return tk == 128 ? gemm_onchip<128, 1>() : tk == 64 ? gemm_onchip<64, 1>() : gemm_onchip<32, 1>();
 }
 
 attn_status mat_bwd(const Problem &p)
 {
     if (mask_is_block(p.mask_kind)) return ATTN_ERR_MASK;
-    const size_t rows = (size_t)p.BH * p.n;
-    size_t blocks = (rows + 7) / 8;
-    if (blocks > (size_t)sm_count() * 8) blocks = (size_t)sm_count() * 8;
-    launch_begin("mat_preprocess", p.stream);
-    mat_preprocess_kernel<<<(unsigned)blocks, 256, 0, p.stream>>>((const __nv_bfloat16 *)p.O, (const __nv_bfloat16 *)p.dO,
-                                                                  p.LSE, p.D, p.nLSE2, rows, p.d, p.scale);
-    launch_end(p.stream);
-    if (cudaGetLastError() != cudaSuccess) return ATTN_ERR_LAUNCH;
+    if (bwd_preprocess_launch(p, false) != ATTN_OK) return ATTN_ERR_LAUNCH;   // Ds = scale D, -LSE log2e
     for (size_t h0 = 0; h0 < (size_t)p.BH; h0 += p.mat_heads) {
         const int mh = (int)((size_t)p.BH - h0 < (size_t)p.mat_heads ? (size_t)p.BH - h0 : (size_t)p.mat_heads);
         const attn_status st = run_chunk(p, h0, mh);

@@ -100,11 +100,12 @@ def test_config3_every_head_fused_against_the_path_without_atomics():
         assert float(per_head.max()) <= (H.TOL["bf16"] if name == "dQ" else 2 ** -7), (name, per_head)
 
 
-@pytest.mark.parametrize("tile_k", [128, 64, 32])
-def test_config4_full_small_cache_regime_tile_sweep(tile_k):
-    """d = 256: fused forward, materialised (small-cache) backward, block edge swept over three values."""
+@pytest.mark.parametrize("tile_q,tile_k", [(128, 128), (128, 64), (128, 32), (256, 128), (256, 32)])
+def test_config4_full_small_cache_regime_tile_sweep(tile_q, tile_k):
+    """d = 256: fused forward, materialised (small-cache) backward, block edges swept."""
     import paper_2410_09397_b200 as attn
-    run_full("C4", [0, 7] if tile_k == 128 else [5], cfg=attn.Cfg(tile_k=tile_k, algo=attn.ATTN_ALGO_MATERIALIZED))
+    run_full("C4", [0, 7] if tile_k == 128 else [5],
+             cfg=attn.Cfg(tile_q=tile_q, tile_k=tile_k, algo=attn.ATTN_ALGO_MATERIALIZED))
 
 
 def test_config4_full_default_cfg():

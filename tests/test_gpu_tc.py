@@ -126,17 +126,26 @@ def test_forward_merges_partial_softmaxes_with_unequal_maxima(n, d, mask_kind, b
     H.assert_within({"O": H.rel_err(H.to_np(O), O_ref), "LSE": H.rel_err(H.to_np(LSE), LSE_ref)}, "bf16")
 
 
-def materialized(tile_k=0):
+def materialized(tile_k=0, tile_q=0):
     from paper_2410_09397_b200 import binding as B
-    return B.Cfg(tile_k=tile_k, algo=B.ATTN_ALGO_MATERIALIZED)
+    return B.Cfg(tile_q=tile_q, tile_k=tile_k, algo=B.ATTN_ALGO_MATERIALIZED)
 
 
+@pytest.mark.parametrize("tile_q", [128, 256])
 @pytest.mark.parametrize("tile_k", [128, 64, 32])
 @pytest.mark.parametrize("n,d", [(256, 256), (1000, 256), (384, 128), (200, 64)])
 @pytest.mark.parametrize("mask_kind", [inputs.MASK_NONE, inputs.MASK_CAUSAL])
-def test_materialized_backward(n, d, tile_k, mask_kind):
-    """Small-cache algorithm: P, dP, dS go through device memory; three tile sizes."""
-    errs = H.run_case(1, 2, n, d, "bf16", mask_kind, seed=38, cfg=materialized(tile_k))
+def test_materialized_backward(n, d, tile_k, tile_q, mask_kind):
+    """Small-cache algorithm: P, dP, dS go through device memory; blocks of 128 or 256 rows by 128, 64 or 32 columns
+    (sizes with a ragged last block in either direction, and more tiles than one CTA's two accumulator sets)."""
+    errs = H.run_case(1, 2, n, d, "bf16", mask_kind, seed=38, cfg=materialized(tile_k, tile_q))
+    H.assert_within(errs, "bf16")
+
+
+def test_materialized_backward_many_tiles_per_cta():
+    """More tiles than resident CTAs: every CTA of the persistent products walks several tiles, so that the operand
+    ring, both accumulator sets and both staging tiles wrap (n = 2432: 19 x 19 blocks x 10 heads = 3610 tiles)."""
+    errs = H.run_case(2, 5, 2432, 64, "bf16", inputs.MASK_CAUSAL, seed=40, cfg=materialized(128, 128), check_bwd_only=False)
     H.assert_within(errs, "bf16")
 
 
