@@ -61,7 +61,7 @@ typedef enum {
 typedef enum { ATTN_F32 = 0, ATTN_BF16 = 1 } attn_dtype;
 
 typedef enum { ATTN_MASK_NONE = 0, ATTN_MASK_CAUSAL = 1, ATTN_MASK_BLOCK_SPARSE = 2,
-               ATTN_MASK_BLOCK_SPARSE_CAUSAL = 3 } attn_mask_kind;
+               ATTN_MASK_BLOCK_SPARSE_CAUSAL = 3, ATTN_MASK_ELEMENT = 4 } attn_mask_kind;
 
 /* Which (i, j) score entries are kept.  NULL means ATTN_MASK_NONE.
  *   CAUSAL:       keep j <= i (one n for queries and keys).
@@ -73,6 +73,12 @@ typedef enum { ATTN_MASK_NONE = 0, ATTN_MASK_CAUSAL = 1, ATTN_MASK_BLOCK_SPARSE 
  *                 least one block and drop the other blocks' entries inside the tile.
  *   BLOCK_SPARSE_CAUSAL: both at once -- keep (i, j) iff its block is kept and j <= i
  *                 (same fields as BLOCK_SPARSE; blocks above the diagonal are never visited).
+ *   ELEMENT:      any set of kept entries, one bit each: block_mask points to a DEVICE bitmap of
+ *                 32-bit words [mask_heads][n][ceil(n / 32)], bit (j % 32) of word j / 32 of row i
+ *                 set iff (i, j) is kept; `block` is ignored.  attn_mask_from_coo() builds the
+ *                 bitmap from a coordinate list, the form in which Section 4.1 stores a sparse
+ *                 matrix.  FUSED and SIMT algorithms only; the tensor-core kernels visit the
+ *                 128 x 128 tiles that keep at least one entry.
  * This is the sparse setting of Section 4.1 with Z_QK = the number of kept entries;
  * a masked score is minus infinity, not a stored zero. */
 typedef struct {
@@ -234,6 +240,15 @@ double attn_io_bound_sparse_elems(double z_input, double z_qk, double M);
 typedef struct { double loads, stores, reductions; } attn_io_count; /* elements, per head */
 attn_status attn_io_replay(int n, int d, int mask_kind, int dt, const attn_cfg *cfg, int backward,
                            attn_io_count *out /* host */);
+
+/* Builds the bitmap of an ATTN_MASK_ELEMENT mask from a coordinate list (Section 4.1 stores a sparse
+ * matrix as the coordinates of its entries): clears `bitmap` (DEVICE, mask_heads * n * ceil(n / 32)
+ * 32-bit words, 4-byte aligned) and sets the bit of every (rows[e], cols[e]) of mask heads[e], e < nnz.
+ * rows, cols, heads: DEVICE int32 arrays of nnz entries; heads == NULL puts every entry into mask 0.
+ * An entry whose row, column or head is out of range is ignored; duplicates are harmless.
+ * Enqueued on cuda_stream; returns after validating the arguments. */
+attn_status attn_mask_from_coo(const int *rows, const int *cols, const int *heads, size_t nnz, int n,
+                               int mask_heads, uint32_t *bitmap, void *cuda_stream);
 
 const char *attn_status_str(int status);
 

@@ -19,7 +19,7 @@ ATTN_OK = 0
 (ATTN_ERR_NULL, ATTN_ERR_SHAPE, ATTN_ERR_DTYPE, ATTN_ERR_ALIGN, ATTN_ERR_TILE, ATTN_ERR_MASK, ATTN_ERR_WORKSPACE,
  ATTN_ERR_ARCH, ATTN_ERR_LAUNCH, ATTN_ERR_DEVICE_TIMEOUT) = range(1, 11)
 ATTN_F32, ATTN_BF16 = 0, 1
-ATTN_MASK_NONE, ATTN_MASK_CAUSAL, ATTN_MASK_BLOCK_SPARSE, ATTN_MASK_BLOCK_SPARSE_CAUSAL = 0, 1, 2, 3
+ATTN_MASK_NONE, ATTN_MASK_CAUSAL, ATTN_MASK_BLOCK_SPARSE, ATTN_MASK_BLOCK_SPARSE_CAUSAL, ATTN_MASK_ELEMENT = 0, 1, 2, 3, 4
 ATTN_ALGO_AUTO, ATTN_ALGO_FUSED, ATTN_ALGO_MATERIALIZED, ATTN_ALGO_SIMT = 0, 1, 2, 3
 
 # every symbol include/attn.h declares
@@ -28,7 +28,7 @@ EXPORTS = (
     "attn_workspace_status", "attn_supported_cfgs", "attn_cfg_onchip_elems", "attn_io_bound_elems",
     "attn_io_bound_sparse_elems", "attn_io_replay", "attn_status_str", "attn_kernel_launches", "attn_timing_enable",
     "attn_timing_collect", "attn_bwd_noalloc", "attn_noalloc_scratch_bytes", "attn_noalloc_status",
-    "attn_selftest_wait_timeout",
+    "attn_selftest_wait_timeout", "attn_mask_from_coo",
     "attn_project", "attn_weight_grad", "attn_weights_bwd", "attn_weights_bwd_workspace_bytes",
 )
 
@@ -55,12 +55,16 @@ class CIoCount(ctypes.Structure):
 
 @dataclass
 class Mask:
-    """Which score entries are kept; ``block_mask`` is a CUDA uint8 tensor ``[mask_heads, nb, nb]``."""
+    """Which score entries are kept; ``block_mask`` is a CUDA uint8 tensor ``[mask_heads, nb, nb]``, or, for
+    ATTN_MASK_ELEMENT, a CUDA int32 tensor ``[mask_heads, n, ceil(n / 32)]`` of keep bits."""
     kind: int = ATTN_MASK_NONE
     block: int = 128
     block_mask: object = None
 
     def c(self) -> CMask | None:
+        if self.kind == ATTN_MASK_ELEMENT:
+            bm = self.block_mask
+            return CMask(self.kind, 0, bm.data_ptr() if bm is not None else None, int(bm.shape[0]) if bm is not None else 1)
         if self.kind in (ATTN_MASK_BLOCK_SPARSE, ATTN_MASK_BLOCK_SPARSE_CAUSAL):
             bm = self.block_mask
             return CMask(self.kind, self.block, bm.data_ptr() if bm is not None else None,
@@ -106,6 +110,8 @@ def lib() -> ctypes.CDLL:
     L.attn_noalloc_status.argtypes = [vp]
     L.attn_selftest_wait_timeout.restype = ci
     L.attn_selftest_wait_timeout.argtypes = [vp, sz, ctypes.c_uint, vp]
+    L.attn_mask_from_coo.restype = ci
+    L.attn_mask_from_coo.argtypes = [vp, vp, vp, sz, ci, ci, vp, vp]
     L.attn_bwd_preprocess.restype = ci
     L.attn_bwd_preprocess.argtypes = [vp, vp, vp, sz, ci, ci, vp]
     for f in (L.attn_fwd_workspace_bytes, L.attn_bwd_workspace_bytes):
@@ -323,6 +329,20 @@ def attn_io_replay(n: int, d: int, mask_kind: int, dt: int, cfg: Cfg | None, bac
         raise AttnError(st, "attn_io_replay")
     return {"loads": out.loads, "stores": out.stores, "reductions": out.reductions,
             "total": out.loads + out.stores + out.reductions}
+
+
+def attn_mask_from_coo(rows, cols, heads, n: int, mask_heads: int = 1, bitmap=None):
+    """Bitmap of an ATTN_MASK_ELEMENT mask from CUDA int32 coordinate tensors (``heads`` may be None)."""
+    import torch
+    nnz = int(rows.numel())
+    if bitmap is None:
+        bitmap = torch.empty((mask_heads, n, (n + 31) // 32), dtype=torch.int32, device=rows.device)
+    st = lib().attn_mask_from_coo(rows.data_ptr() if nnz else None, cols.data_ptr() if nnz else None,
+                                  heads.data_ptr() if heads is not None else None, nnz, n, mask_heads, bitmap.data_ptr(),
+                                  _stream())
+    if st != ATTN_OK:
+        raise AttnError(st, "attn_mask_from_coo")
+    return bitmap
 
 
 def attn_io_bound_elems(n, d, M, backward: bool) -> float:

@@ -35,7 +35,7 @@ attn_status resolve_cfg(const Args &a, int backward, attn_cfg *out)
         // d = 256 backward: the fused tile set does not fit on chip; the small-cache algorithm takes it
         probe.algo = ATTN_ALGO_MATERIALIZED;
         if (!tc_ok && backward && a.dt == ATTN_BF16 && a.d == 256 && (a.n % 8) == 0 &&
-            !(a.mask && mask_is_block(a.mask->kind)) && tc_cfg_supported(a.d, probe, backward))
+            !(a.mask && (mask_is_block(a.mask->kind) || mask_is_element(a.mask->kind))) && tc_cfg_supported(a.d, probe, backward))
             c.algo = ATTN_ALGO_MATERIALIZED;
     }
     if (c.algo == ATTN_ALGO_MATERIALIZED && !backward) {   // its forward is the fused one, with that kernel's own tiles
@@ -56,7 +56,8 @@ attn_status resolve_cfg(const Args &a, int backward, attn_cfg *out)
         if (a.d != 64 && a.d != 128 && a.d != 256) return ATTN_ERR_SHAPE;
         if (a.n % 8 != 0) return ATTN_ERR_SHAPE;
         if (a.mask && mask_is_block(a.mask->kind) && !tc_block_ok(a.mask->block)) return ATTN_ERR_MASK;
-        if (c.algo == ATTN_ALGO_MATERIALIZED && a.mask && mask_is_block(a.mask->kind)) return ATTN_ERR_MASK;
+        if (c.algo == ATTN_ALGO_MATERIALIZED && a.mask && (mask_is_block(a.mask->kind) || mask_is_element(a.mask->kind)))
+            return ATTN_ERR_MASK;
         if (!tc_cfg_supported(a.d, c, backward)) return ATTN_ERR_TILE;
         // fill defaults the way the kernels resolve them
         attn_cfg list[32];
@@ -86,9 +87,9 @@ attn_status check_shape(const Args &a)
     if ((double)a.batch * a.heads * a.n * a.d > 1.7e10) return ATTN_ERR_SHAPE;
     if (a.mask) {
         const attn_mask &m = *a.mask;
-        if (m.kind < ATTN_MASK_NONE || m.kind > ATTN_MASK_BLOCK_SPARSE_CAUSAL) return ATTN_ERR_MASK;
-        if (mask_is_block(m.kind)) {
-            if (m.block < 1) return ATTN_ERR_MASK;
+        if (m.kind < ATTN_MASK_NONE || m.kind > ATTN_MASK_ELEMENT) return ATTN_ERR_MASK;
+        if (mask_is_block(m.kind) || mask_is_element(m.kind)) {
+            if (mask_is_block(m.kind) && m.block < 1) return ATTN_ERR_MASK;
             if (m.mask_heads != 1 && m.mask_heads != a.batch * a.heads) return ATTN_ERR_MASK;
         }
     }
@@ -108,14 +109,20 @@ attn_status layout(const Args &a, int backward, attn_cfg *cfg_out, WorkspaceLayo
     L->status = off; off += 256;
     const size_t BH = (size_t)a.batch * a.heads;
     if (backward) { L->D = off; off += align_up(BH * a.n * sizeof(float), 256); }
-    const bool sparse = a.mask && mask_is_block(a.mask->kind);
+    const bool element = a.mask && mask_is_element(a.mask->kind);
+    const bool sparse = a.mask && (mask_is_block(a.mask->kind) || element);
     if (sparse && c.algo != ATTN_ALGO_SIMT) {
-        const int eff = a.mask->block < 128 ? 128 : a.mask->block;   // fine blocks: lists of 128 x 128 super-blocks
+        // fine blocks and element masks: lists of the 128 x 128 tiles that keep anything
+        const int eff = (element || a.mask->block < 128) ? 128 : a.mask->block;
         const size_t nb = (a.n + eff - 1) / eff, mh = a.mask->mask_heads;
         L->row_ptr = off; off += align_up(mh * 2 * nb * sizeof(int), 256);
         L->col_idx = off; off += align_up(mh * nb * nb * sizeof(int), 256);
         L->col_ptr = off; off += align_up(mh * 2 * nb * sizeof(int), 256);
         L->row_idx = off; off += align_up(mh * nb * nb * sizeof(int), 256);
+        if (element) {
+            L->tilemask = off; off += align_up(mh * nb * nb, 256);
+            L->colbits = off; off += align_up(mh * (size_t)a.n * ((a.n + 31) / 32) * sizeof(uint32_t), 256);
+        }
     }
     if (backward && (c.algo == ATTN_ALGO_FUSED || c.algo == ATTN_ALGO_MATERIALIZED)) { L->nLSE2 = off; off += align_up(BH * a.n * sizeof(float), 256); }
     if (backward && c.algo == ATTN_ALGO_FUSED && !c.deterministic) {
@@ -166,7 +173,8 @@ attn_status fill_problem(Problem &p, const Args &a, int backward, float scale, v
     attn_cfg c;
     attn_status st = layout(a, backward, &c, &L);
     if (st != ATTN_OK) return st;
-    if (a.mask && mask_is_block(a.mask->kind) && !a.mask->block_mask) return ATTN_ERR_NULL;
+    if (a.mask && (mask_is_block(a.mask->kind) || mask_is_element(a.mask->kind)) && !a.mask->block_mask) return ATTN_ERR_NULL;
+    if (a.mask && mask_is_element(a.mask->kind) && ((uintptr_t)a.mask->block_mask & 3) != 0) return ATTN_ERR_ALIGN;
     if (!workspace || workspace_bytes < L.total) return ATTN_ERR_WORKSPACE;
     if (((uintptr_t)workspace & 255) != 0) return ATTN_ERR_ALIGN;
     if (!(scale >= 0.f) || isinf(scale)) return ATTN_ERR_SHAPE;
@@ -175,12 +183,12 @@ attn_status fill_problem(Problem &p, const Args &a, int backward, float scale, v
     p.dt = a.dt;
     p.mask_kind = a.mask ? a.mask->kind : ATTN_MASK_NONE;
     p.block = mask_is_block(p.mask_kind) ? a.mask->block : 0;
-    p.mask_heads = mask_is_block(p.mask_kind) ? a.mask->mask_heads : 1;
+    p.mask_heads = (mask_is_block(p.mask_kind) || mask_is_element(p.mask_kind)) ? a.mask->mask_heads : 1;
     p.nb = p.block ? (a.n + p.block - 1) / p.block : 0;
-    p.block_mask = mask_is_block(p.mask_kind) ? a.mask->block_mask : nullptr;
-    p.fine = FineMask{nullptr, 0, 0};
+    p.block_mask = (mask_is_block(p.mask_kind) || mask_is_element(p.mask_kind)) ? a.mask->block_mask : nullptr;
+    p.fine = FineMask{};
     if (p.block && p.block < 128 && c.algo != ATTN_ALGO_SIMT) {
-        p.fine = FineMask{p.block_mask, p.block, p.nb};
+        p.fine.mode = 1; p.fine.bits = p.block_mask; p.fine.block = p.block; p.fine.nb = p.nb;
         p.block = 128;
         p.nb = (a.n + 127) / 128;
     }
@@ -194,6 +202,17 @@ attn_status fill_problem(Problem &p, const Args &a, int backward, float scale, v
     p.col_idx = L.col_idx ? (int *)(w + L.col_idx) : nullptr;
     p.col_ptr = L.col_ptr ? (int *)(w + L.col_ptr) : nullptr;
     p.row_idx = L.row_idx ? (int *)(w + L.row_idx) : nullptr;
+    p.tilemask = L.tilemask ? (uint8_t *)(w + L.tilemask) : nullptr;
+    p.colbits = L.colbits ? (uint32_t *)(w + L.colbits) : nullptr;
+    if (mask_is_element(p.mask_kind) && c.algo != ATTN_ALGO_SIMT) {
+        // the tensor-core kernels see a block mask of 128 x 128 tiles (built from the bitmap) with the bits applied inside the tiles
+        p.fine.mode = 2; p.fine.rowbits = (const uint32_t *)a.mask->block_mask; p.fine.colbits = p.colbits;
+        p.fine.n = a.n; p.fine.words = (a.n + 31) / 32;
+        p.mask_kind = ATTN_MASK_BLOCK_SPARSE;
+        p.block = 128;
+        p.nb = (a.n + 127) / 128;
+        p.block_mask = p.tilemask;
+    }
     p.dQ_acc = L.dQ_acc ? (float *)(w + L.dQ_acc) : nullptr;
     p.matP = L.matP ? w + L.matP : nullptr;
     p.matdP = L.matdP ? w + L.matdP : nullptr;

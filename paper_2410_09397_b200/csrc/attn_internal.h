@@ -8,19 +8,29 @@
 
 namespace attn {
 
-// A block mask whose blocks are finer than the 128 x 128 tiles of the tensor-core kernels (block edge 32 or
-// 64): the kernels then walk lists of 128 x 128 super-blocks that keep at least one fine block, and drop the
-// entries of the fine blocks that are not kept inside every visited tile.  block == 0: not in use.
+// Masks finer than the 128 x 128 tiles of the tensor-core kernels.  The kernels walk lists of the tiles that keep
+// anything and drop the other entries inside every visited tile:
+//   mode 1: a block mask with a block edge of 32 or 64 (`bits`, the caller's mask [mask_heads][nb][nb]);
+//   mode 2: an element mask, one bit per score entry: `rowbits` [mask_heads][n][words] has bit j % 32 of word
+//           j / 32 of row i set iff (i, j) is kept (the caller's bitmap), `colbits` is its transpose (row j, bit i),
+//           built in the workspace for the key-stationary kernels.
 struct FineMask {
-    const uint8_t *bits;   // the caller's mask [mask_heads][nb][nb]
+    int mode;              // 0: not in use
+    const uint8_t *bits;   // mode 1
     int block, nb;
+    const uint32_t *rowbits, *colbits;   // mode 2
+    int n, words;
 };
 #ifdef __CUDACC__
-// (i, j) < n; which of the caller's masks: head bh unless one mask serves all
-__device__ __forceinline__ bool fine_keep(const FineMask &f, int mask_heads, long bh, int i, int j)
+// Keep bits of the 32 entries (r, c0 .. c0 + 31), c0 a multiple of 32, r < n, c0 < n.  by_query: r is a query
+// row and the columns are keys; otherwise r is a key row and the columns are queries.
+__device__ __forceinline__ uint32_t fine_word(const FineMask &f, int mask_heads, long bh, bool by_query, int r, int c0)
 {
-    const uint8_t *m = f.bits + (mask_heads == 1 ? 0 : (size_t)bh * f.nb * f.nb);
-    return m[(size_t)(i / f.block) * f.nb + j / f.block] != 0;
+    const size_t mh = mask_heads == 1 ? 0 : (size_t)bh;
+    if (f.mode == 2) return (by_query ? f.rowbits : f.colbits)[(mh * f.n + r) * f.words + c0 / 32];
+    // mode 1: 32 aligned columns lie in one block (block edge 32 or 64)
+    const int i = by_query ? r : c0, j = by_query ? c0 : r;
+    return f.bits[mh * f.nb * f.nb + (size_t)(i / f.block) * f.nb + j / f.block] != 0 ? 0xffffffffu : 0u;
 }
 #endif
 
@@ -35,7 +45,7 @@ struct Problem {
     long BH;                          // batch * heads
     int mask_kind, block, mask_heads, nb;
     const uint8_t *block_mask;
-    FineMask fine;                    // tensor-core algorithms with a block edge below 128: block / nb then describe the super-blocks
+    FineMask fine;                    // tensor-core algorithms with a mask finer than their tiles: block / nb / block_mask then describe the 128 x 128 tiles
     int dt;
     float scale;
     attn_cfg cfg;                     // resolved: algo and tiles are final
@@ -45,6 +55,8 @@ struct Problem {
     float *nLSE2;                     // [BH * n]: -LSE * log2(e), fused backward only
     int *row_ptr, *col_idx;           // block-CSR of the mask: [mask_heads][nb+1], [mask_heads][nb*nb]
     int *col_ptr, *row_idx;           // block-CSC
+    uint8_t *tilemask;                // element mask: which 128 x 128 tiles keep anything [mask_heads][nb][nb]
+    uint32_t *colbits;                // element mask: the transposed bitmap
     float *dQ_acc;                    // fp32 dQ accumulator [BH * n * d] (fused backward with atomics)
     void *matP, *matdP, *matdS;       // materialised n x n buffers (per head chunk)
     int mat_heads;                    // heads materialised at once
@@ -52,7 +64,7 @@ struct Problem {
 };
 
 struct WorkspaceLayout {
-    size_t status, D, nLSE2, row_ptr, col_idx, col_ptr, row_idx, dQ_acc, matP, matdP, matdS, total;
+    size_t status, D, nLSE2, row_ptr, col_idx, col_ptr, row_idx, tilemask, colbits, dQ_acc, matP, matdP, matdS, total;
     int mat_heads;
 };
 
@@ -64,6 +76,7 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // mask kinds: "block" = described by a block mask, "causal" = entries with j > i are dropped
 __host__ __device__ inline bool mask_is_block(int kind) { return kind == ATTN_MASK_BLOCK_SPARSE || kind == ATTN_MASK_BLOCK_SPARSE_CAUSAL; }
+__host__ __device__ inline bool mask_is_element(int kind) { return kind == ATTN_MASK_ELEMENT; }
 __host__ __device__ inline bool mask_is_causal(int kind) { return kind == ATTN_MASK_CAUSAL || kind == ATTN_MASK_BLOCK_SPARSE_CAUSAL; }
 
 // Streaming multiprocessors of the current device (grid sizing of the grid-stride and persistent kernels).

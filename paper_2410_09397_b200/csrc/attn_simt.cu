@@ -31,8 +31,8 @@ template <> __device__ __forceinline__ float from_f<float>(float v) { return v; 
 template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
 struct MaskDev {
-    int kind, block, nb;
-    const uint8_t *bits;  // already offset to this head's [nb][nb] mask
+    int kind, block, nb;  // element mask: block = n, nb = 32-bit words per row
+    const uint8_t *bits;  // already offset to this head's [nb][nb] mask (element mask: its [n][nb] bitmap)
 };
 
 __device__ __forceinline__ bool keep(const MaskDev &m, int i, int j)
@@ -40,6 +40,8 @@ __device__ __forceinline__ bool keep(const MaskDev &m, int i, int j)
     if (m.kind == ATTN_MASK_NONE) return true;
     if (m.kind == ATTN_MASK_CAUSAL) return j <= i;
     if (m.kind == ATTN_MASK_BLOCK_SPARSE_CAUSAL && j > i) return false;
+    if (m.kind == ATTN_MASK_ELEMENT)
+        return (reinterpret_cast<const uint32_t *>(m.bits)[(size_t)i * m.nb + j / 32] >> (j % 32)) & 1u;
     return m.bits[(size_t)(i / m.block) * m.nb + j / m.block] != 0;
 }
 
@@ -49,6 +51,7 @@ __device__ __forceinline__ bool tile_any(const MaskDev &m, int i0, int i1, int j
     if (m.kind == ATTN_MASK_NONE) return true;
     if (m.kind == ATTN_MASK_CAUSAL) return j0 <= i1;
     if (m.kind == ATTN_MASK_BLOCK_SPARSE_CAUSAL && j0 > i1) return false;
+    if (m.kind == ATTN_MASK_ELEMENT) return true;   // the fp32 kernels visit every tile of an element mask
     for (int I = i0 / m.block; I <= i1 / m.block; ++I)
         for (int J = j0 / m.block; J <= j1 / m.block; ++J)
             if (m.bits[(size_t)I * m.nb + J]) return true;
@@ -59,6 +62,7 @@ __device__ __forceinline__ MaskDev head_mask(int kind, int block, int nb, const 
 {
     MaskDev m{kind, block, nb, bits};
     if (mask_is_block(kind) && mask_heads != 1) m.bits = bits + (size_t)bh * nb * nb;
+    if (mask_is_element(kind) && mask_heads != 1) m.bits = bits + (size_t)bh * block * nb * sizeof(uint32_t);
     return m;
 }
 
@@ -510,6 +514,7 @@ SimtArgs make_args(const Problem &p)
     a.n = p.n; a.d = p.d;
     a.mask_kind = p.mask_kind; a.block = p.block; a.nb = p.nb; a.mask_heads = p.mask_heads;
     a.bits = p.block_mask;
+    if (mask_is_element(p.mask_kind)) { a.block = p.n; a.nb = (p.n + 31) / 32; }
     a.scale = p.scale;
     return a;
 }
@@ -594,11 +599,53 @@ attn_status preprocess_D(const void *O, const void *dO, float *D, size_t rows, i
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_LAUNCH;
 }
 
+// ---------------------------------------------------------------- element masks
+// One warp per 32 x 32 block of the bitmap: writes the transposed block (row j, bit i) for the key-stationary
+// kernels and marks the 128 x 128 tile as kept if the block has a bit set.  Bits beyond n are dropped here, so
+// the kernels never see them.  grid (words, ceil(n / 32), mask_heads), 32 threads.
+__global__ void element_mask_prepare_kernel(const uint32_t *__restrict__ rowbits, uint32_t *__restrict__ colbits,
+                                            uint8_t *__restrict__ tilemask, int n, int words, int nb)
+{
+    const int wj = blockIdx.x, ri = blockIdx.y, h = blockIdx.z, lane = threadIdx.x;
+    const int i = ri * 32 + lane;
+    uint32_t w = i < n ? rowbits[((size_t)h * n + i) * words + wj] : 0u;
+    const int jrem = n - wj * 32;                       // valid columns in this word
+    if (jrem < 32) w &= (1u << jrem) - 1u;
+    uint32_t mine = 0;
+#pragma unroll
+    for (int c = 0; c < 32; ++c) {
+        const uint32_t col = __ballot_sync(0xffffffffu, (w >> c) & 1u);   // bit r = entry (ri * 32 + r, wj * 32 + c)
+        if (lane == c) mine = col;
+    }
+    const int j = wj * 32 + lane;
+    if (j < n) colbits[((size_t)h * n + j) * words + ri] = mine;
+    if (__any_sync(0xffffffffu, w != 0u) && lane == 0) tilemask[((size_t)h * nb + ri / 4) * nb + wj / 4] = 1;
+}
+
+__global__ void coo_scatter_kernel(const int *__restrict__ rows, const int *__restrict__ cols, const int *__restrict__ heads,
+                                   size_t nnz, int n, int mask_heads, int words, uint32_t *__restrict__ bitmap)
+{
+    for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < nnz; e += (size_t)gridDim.x * blockDim.x) {
+        const int i = rows[e], j = cols[e], h = heads ? heads[e] : 0;
+        if (i < 0 || i >= n || j < 0 || j >= n || h < 0 || h >= mask_heads) continue;
+        atomicOr(bitmap + ((size_t)h * n + i) * words + j / 32, 1u << (j % 32));
+    }
+}
+
 attn_status build_block_index(const Problem &p)
 {
     if (!mask_is_block(p.mask_kind) || !p.row_ptr) return ATTN_OK;
+    if (p.fine.mode == 2) {
+        // element mask: transposed bitmap and the mask of 128 x 128 tiles, from which the lists below are built
+        if (cudaMemsetAsync(p.tilemask, 0, (size_t)p.mask_heads * p.nb * p.nb, p.stream) != cudaSuccess) return ATTN_ERR_LAUNCH;
+        launch_begin("element_mask_prepare", p.stream);
+        element_mask_prepare_kernel<<<dim3(p.fine.words, (p.n + 31) / 32, p.mask_heads), 32, 0, p.stream>>>(
+            p.fine.rowbits, p.colbits, p.tilemask, p.n, p.fine.words, p.nb);
+        launch_end(p.stream);
+        if (cudaGetLastError() != cudaSuccess) return ATTN_ERR_LAUNCH;
+    }
     launch_begin("block_index", p.stream);
-    const int nbm = p.fine.block ? p.fine.nb : p.nb, ratio = p.fine.block ? 128 / p.fine.block : 1;
+    const int nbm = p.fine.mode == 1 ? p.fine.nb : p.nb, ratio = p.fine.mode == 1 ? 128 / p.fine.block : 1;
     block_index_kernel<<<dim3(p.nb, p.mask_heads), 64, 0, p.stream>>>(p.block_mask, p.nb, nbm, ratio, p.row_ptr, p.col_idx,
                                                                       p.col_ptr, p.row_idx);
     launch_end(p.stream);
@@ -606,3 +653,21 @@ attn_status build_block_index(const Problem &p)
 }
 
 }  // namespace attn
+
+extern "C" attn_status attn_mask_from_coo(const int *rows, const int *cols, const int *heads, size_t nnz, int n, int mask_heads,
+                                          uint32_t *bitmap, void *cuda_stream)
+{
+    if (!bitmap || (nnz && (!rows || !cols))) return ATTN_ERR_NULL;
+    if (n < 1 || mask_heads < 1) return ATTN_ERR_SHAPE;
+    if (((uintptr_t)bitmap & 3) != 0) return ATTN_ERR_ALIGN;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const int words = (n + 31) / 32;
+    if (cudaMemsetAsync(bitmap, 0, (size_t)mask_heads * n * words * sizeof(uint32_t), s) != cudaSuccess) return ATTN_ERR_LAUNCH;
+    if (nnz == 0) return ATTN_OK;
+    size_t blocks = (nnz + 255) / 256;
+    if (blocks > (size_t)attn::sm_count() * 16) blocks = (size_t)attn::sm_count() * 16;
+    attn::launch_begin("mask_from_coo", s);
+    attn::coo_scatter_kernel<<<(unsigned)blocks, 256, 0, s>>>(rows, cols, heads, nnz, n, mask_heads, words, bitmap);
+    attn::launch_end(s);
+    return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_LAUNCH;
+}

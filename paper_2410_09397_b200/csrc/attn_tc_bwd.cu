@@ -280,9 +280,10 @@ tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
             const float4 *sDs = reinterpret_cast<const float4 *>(smem + L::oD + s2 * 512 + h * 256 + qq * 128);
             const bool diag = mask_is_causal(a.mask_kind) && it == jt;
             const int ig0 = i0 + h * 64 + qq * 32;
-            // fine blocks: this thread's 32 query columns and its key row lie in one block of the caller's mask
-            const bool fkeep = !a.fine.block || (ig0 < n && jg < n && fine_keep(a.fine, a.mask_heads, bh, ig0, jg));
-            const bool masked = diag || i0 + TQ > n || j0 + TK > n || a.fine.block != 0;
+            // a mask finer than the tile: the keep bits of this thread's key row and its 32 query columns
+            uint32_t kw = 0xffffffffu;
+            if (a.fine.mode) kw = (ig0 < n && jg < n) ? fine_word(a.fine, a.mask_heads, bh, false, jg, ig0) : 0u;
+            const bool masked = diag || i0 + TQ > n || j0 + TK > n || a.fine.mode != 0;
             mbar_wait(&bars[KD_S], k & 1, ab);
             tcgen05_fence_after();
             uint32_t ppack[16];
@@ -305,7 +306,7 @@ tc_bwd_dkdv_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const int ig = ig0 + q * 4 + e;
-                            const bool ok = ig < n && jg < n && (!diag || jg <= ig) && fkeep;
+                            const bool ok = ig < n && jg < n && (!diag || jg <= ig) && ((kw >> (q * 4 + e)) & 1u);
                             p[e] = ok ? p[e] : 0.f;
                         }
                     }
@@ -675,9 +676,9 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
             const float4 *sDs = reinterpret_cast<const float4 *>(smem + L::oD + s * 512 + h * 256 + qq * 128);
             const bool diag = mask_is_causal(a.mask_kind) && it == jt;
             const int ig0 = i0 + h * 64 + qq * 32;
-            // fine blocks: this thread's 32 query columns and its key row lie in one block of the caller's mask
-            bool fkeep = true;
-            if constexpr (FINE) fkeep = ig0 < n && jg < n && fine_keep(a.fine, a.mask_heads, bh, ig0, jg);
+            // a mask finer than the tile: the keep bits of this thread's key row and its 32 query columns
+            uint32_t kw = 0xffffffffu;
+            if constexpr (FINE) kw = (ig0 < n && jg < n) ? fine_word(a.fine, a.mask_heads, bh, false, jg, ig0) : 0u;
             const bool masked = diag || i0 + TQ > n || j0 + TK > n || FINE;
             mbar_wait(&bars[V2_QFULL + s], (k >> 1) & 1, ab);
             // the 32 row statistics of this thread's query columns go into registers before the wait for S^T: while the
@@ -706,7 +707,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const int ig = ig0 + q * 4 + e;
-                            const bool ok = ig < n && jg < n && (!diag || jg <= ig) && fkeep;
+                            const bool ok = ig < n && jg < n && (!diag || jg <= ig) && ((kw >> (q * 4 + e)) & 1u);
                             p[e] = ok ? p[e] : 0.f;
                         }
                     }
@@ -854,7 +855,7 @@ attn_status launch_bwd(const Problem &p)
     launch_begin(WITH_DQ ? "tc_bwd_fused" : "tc_bwd_dkdv", p.stream);
     if (WITH_DQ) {
         constexpr uint32_t bytes = HD == 64 ? ((L::kBytes + 1023u) & ~1023u) + SLAB : L::kBytes;
-        auto kernel = p.fine.block ? tc_bwd_fused_kernel<HD, true> : tc_bwd_fused_kernel<HD, false>;
+        auto kernel = p.fine.mode ? tc_bwd_fused_kernel<HD, true> : tc_bwd_fused_kernel<HD, false>;
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
             return ATTN_ERR_LAUNCH;
         CUtensorMap mdK, mdV;

@@ -289,9 +289,10 @@ tc_bwd_fused64_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_const
             const float4 *sDs = reinterpret_cast<const float4 *>(smem + L::oD + s * 256 + g * 128);
             const bool diag = mask_is_causal(a.mask_kind) && i0 < j0 + TK;   // some (i, j) of the tile pair has j > i
             const int ig0 = i0 + g * 32;
-            // fine blocks: this thread's 32 query columns and its key row lie in one block of the caller's mask
-            const bool fkeep = !a.fine.block || (ig0 < n && jg < n && fine_keep(a.fine, a.mask_heads, bh, ig0, jg));
-            const bool masked = diag || i0 + TQ64 > n || j0 + TK > n || a.fine.block != 0;
+            // a mask finer than the tile: the keep bits of this thread's key row and its 32 query columns
+            uint32_t kw = 0xffffffffu;
+            if (a.fine.mode) kw = (ig0 < n && jg < n) ? fine_word(a.fine, a.mask_heads, bh, false, jg, ig0) : 0u;
+            const bool masked = diag || i0 + TQ64 > n || j0 + TK > n || a.fine.mode != 0;
             mbar_wait(&bars[B_QFULL + s], (t / NS) & 1, ab);
             float4 nlr[8];
 #pragma unroll
@@ -315,7 +316,7 @@ tc_bwd_fused64_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_const
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const int ig = ig0 + q * 4 + e;
-                            const bool ok = ig < n && jg < n && (!diag || jg <= ig) && fkeep;
+                            const bool ok = ig < n && jg < n && (!diag || jg <= ig) && ((kw >> (q * 4 + e)) & 1u);
                             p[e] = ok ? p[e] : 0.f;
                         }
                     }

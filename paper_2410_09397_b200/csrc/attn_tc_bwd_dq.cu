@@ -243,9 +243,10 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
             if (jt < 0) continue;
             const int b = k & 1, j0 = jt * TKD + wg * 32;
             const uint32_t T_S = tm + b * 128;
-            // fine blocks: this thread's query row and its 32 key columns lie in one block of the caller's mask
-            const bool fkeep = !a.fine.block || (ig < n && j0 < n && fine_keep(a.fine, a.mask_heads, bh, ig, j0));
-            const bool masked = (mask_is_causal(a.mask_kind) && jt * TKD + TKD - 1 > i0) || jt * TKD + TKD > n || a.fine.block != 0;
+            // a mask finer than the tile: the keep bits of this thread's query row and its 32 key columns
+            uint32_t kw = 0xffffffffu;
+            if (a.fine.mode) kw = (ig < n && j0 < n) ? fine_word(a.fine, a.mask_heads, bh, true, ig, j0) : 0u;
+            const bool masked = (mask_is_causal(a.mask_kind) && jt * TKD + TKD - 1 > i0) || jt * TKD + TKD > n || a.fine.mode != 0;
             mbar_wait(&bars[DB_S + b], (k >> 1) & 1, ab);
             tcgen05_fence_after();
             float p[32];
@@ -261,7 +262,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__
 #pragma unroll
                 for (int e = 0; e < 32; ++e) {
                     const int jg = j0 + e;
-                    if (jg >= n || (causal && jg > ig) || !fkeep) p[e] = 0.f;
+                    if (jg >= n || (causal && jg > ig) || !((kw >> e) & 1u)) p[e] = 0.f;
                 }
             }
             mbar_wait(&bars[DB_DP], k & 1, ab);

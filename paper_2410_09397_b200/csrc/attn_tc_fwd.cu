@@ -40,7 +40,7 @@ struct FwdArgs {
     int n, BH;
     int mask_kind, block, nb, mask_heads;
     const int *row_ptr, *col_idx;   // block-CSR of the mask
-    FineMask fine;                  // block edge below 128
+    FineMask fine;                  // a mask finer than the tiles (32- / 64-wide blocks, element bitmap)
     float scale;
     uint32_t *status;
 };
@@ -242,17 +242,19 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
 #pragma unroll
                 for (int e = 0; e < 32; ++e) sv[c + e] = __uint_as_float(v[e]);   // raw scores; scale * log2e enters below
             }
-            const bool need_mask = (mask_is_causal(a.mask_kind) && j0 + TKF - 1 > i0) || j0 + TKF > n || a.fine.block != 0;
+            const bool need_mask = (mask_is_causal(a.mask_kind) && j0 + TKF - 1 > i0) || j0 + TKF > n || a.fine.mode != 0;
             float mx = -INFINITY;
             if (need_mask) {
                 const bool causal = mask_is_causal(a.mask_kind);
 #pragma unroll
+                static_assert(CW == 32, "one keep word per thread and tile");
+                // a mask finer than the tile: the keep bits of this thread's query row and its 32 key columns
+                uint32_t kw = 0xffffffffu;
+                if (a.fine.mode) kw = (ig < n && j0 + wg * CW < n) ? fine_word(a.fine, a.mask_heads, bh, true, ig, j0 + wg * CW) : 0u;
+#pragma unroll
                 for (int e = 0; e < CW; ++e) {
                     const int jg = j0 + wg * CW + e;
-                    bool drop = jg >= n || (causal && jg > ig);
-                    // fine blocks: the block of the caller's mask changes at most every 32 columns
-                    if (a.fine.block && !drop && ig < n) drop = !fine_keep(a.fine, a.mask_heads, bh, ig, jg);
-                    if (drop) sv[e] = -INFINITY;
+                    if (jg >= n || (causal && jg > ig) || !((kw >> e) & 1u)) sv[e] = -INFINITY;
                 }
             }
 #pragma unroll
@@ -509,17 +511,17 @@ tc_fwd_rows_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
             for (int c = 0; c < TKF; c += 32) tmem_ld32(T_S + lane_addr + c, *reinterpret_cast<uint32_t(*)[32]>(&v[c]));
             tmem_wait_ld();
             if (need_mask) {
-                // fine blocks: one flag per 32 key columns (the block of the caller's mask is 32 or 64 wide)
-                bool fk[TKF / 32];
+                // a mask finer than the tile: the keep bits of this thread's query row, one word per 32 key columns
+                uint32_t kw[TKF / 32];
 #pragma unroll
                 for (int q = 0; q < TKF / 32; ++q) {
-                    fk[q] = true;
-                    if constexpr (FINE) fk[q] = ig < n && j0 + q * 32 < n && fine_keep(a.fine, a.mask_heads, bh, ig, j0 + q * 32);
+                    kw[q] = 0xffffffffu;
+                    if constexpr (FINE) kw[q] = (ig < n && j0 + q * 32 < n) ? fine_word(a.fine, a.mask_heads, bh, true, ig, j0 + q * 32) : 0u;
                 }
 #pragma unroll
                 for (int e = 0; e < TKF; ++e) {
                     const int jg = j0 + e;
-                    if (jg >= n || (causal && jg > ig) || !fk[e / 32]) v[e] = 0xff800000u;   // -inf
+                    if (jg >= n || (causal && jg > ig) || !((kw[e / 32] >> (e % 32)) & 1u)) v[e] = 0xff800000u;   // -inf
                 }
             }
             float mx8[8];   // eight independent chains instead of one of 128 dependent maxima
@@ -633,7 +635,7 @@ attn_status launch_fwd(const Problem &p)
     a.status = p.status;
     void (*kernel)(CUtensorMap, CUtensorMap, CUtensorMap, FwdArgs);
     if constexpr (HD == 256) kernel = tc_fwd_kernel<HD>;
-    else kernel = p.fine.block ? tc_fwd_rows_kernel<HD, true> : tc_fwd_rows_kernel<HD, false>;
+    else kernel = p.fine.mode ? tc_fwd_rows_kernel<HD, true> : tc_fwd_rows_kernel<HD, false>;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kBytes) != cudaSuccess)
         return ATTN_ERR_LAUNCH;
     const dim3 grid((p.n + TQ - 1) / TQ, (unsigned)p.BH);

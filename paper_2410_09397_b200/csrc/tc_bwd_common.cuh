@@ -21,7 +21,7 @@ struct BwdArgs {
     const int *col_ptr, *row_idx;   // block-CSC of the mask
     float scale;
     int group;                 // heads per launch group (divides BH)
-    FineMask fine;             // block edge below 128: entries of dropped fine blocks are masked inside the tiles
+    FineMask fine;             // a mask finer than the tiles: dropped entries are masked inside the visited tiles
     uint32_t *status;
 };
 

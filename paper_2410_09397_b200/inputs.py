@@ -34,7 +34,7 @@ _M2 = np.uint64(0x94D049BB133111EB)
 # tensor ids inside one workload seed
 TENSOR_Q, TENSOR_K, TENSOR_V, TENSOR_DO, TENSOR_AUX = 0, 1, 2, 3, 4
 
-MASK_NONE, MASK_CAUSAL, MASK_BLOCK_SPARSE, MASK_BLOCK_SPARSE_CAUSAL = 0, 1, 2, 3
+MASK_NONE, MASK_CAUSAL, MASK_BLOCK_SPARSE, MASK_BLOCK_SPARSE_CAUSAL, MASK_ELEMENT = 0, 1, 2, 3, 4
 
 
 def _mix(z: np.ndarray) -> np.ndarray:
@@ -115,6 +115,22 @@ def block_mask(seed: int, n_blocks: int, keep_prob: float, heads: int = 1) -> np
     m = (u < keep_prob).reshape(heads, n_blocks, n_blocks)
     eye = np.eye(n_blocks, dtype=bool)[None]
     return (m | eye).astype(np.uint8)
+
+
+def element_mask(seed: int, n: int, keep_prob: float, heads: int = 1) -> np.ndarray:
+    """uint8 ``[heads, n, n]``: every entry kept with probability ``keep_prob`` (row-major draw order)."""
+    u = uniform(stream_id(seed, TENSOR_AUX), 0, heads * n * n)
+    return (u < keep_prob).reshape(heads, n, n).astype(np.uint8)
+
+
+def pack_element_mask(keep: np.ndarray) -> np.ndarray:
+    """Keep matrix ``[heads, n, n]`` -> int32 bitmap ``[heads, n, ceil(n / 32)]``: bit j % 32 of word j / 32."""
+    h, n, _ = keep.shape
+    words = (n + 31) // 32
+    padded = np.zeros((h, n, words * 32), dtype=np.uint8)
+    padded[:, :, :n] = keep != 0
+    bits = np.packbits(padded.reshape(h, n, words, 32), axis=-1, bitorder="little")   # 4 bytes per word, low bits first
+    return np.ascontiguousarray(bits).view("<u4").reshape(h, n, words).astype(np.uint32).view(np.int32)
 
 
 @dataclass(frozen=True)

@@ -14,6 +14,8 @@ def oracle_mask_kwargs(mask_kind, block, bmask):
         return dict(mask_kind=orc.MASK_BLOCK, block=block, mask_bits=bmask)
     if mask_kind == inputs.MASK_BLOCK_SPARSE_CAUSAL:
         return dict(mask_kind=orc.MASK_BLOCK_CAUSAL, block=block, mask_bits=bmask)
+    if mask_kind == inputs.MASK_ELEMENT:
+        return dict(mask_kind=orc.MASK_ELEMENT, mask_bits=bmask)       # the explicit keep matrix [mask_heads, n, n]
     return dict(mask_kind=mask_kind)
 
 
@@ -60,6 +62,8 @@ def run_case(b, h, n, d, dtype, mask_kind, *, seed=7, block=128, bmask=None, cfg
     x = make_inputs(seed, b, h, n, d, dtype)
     if mask_kind in (inputs.MASK_BLOCK_SPARSE, inputs.MASK_BLOCK_SPARSE_CAUSAL) and bmask is None:
         bmask = inputs.block_mask(seed + 100, (n + block - 1) // block, keep_prob)
+    if mask_kind == inputs.MASK_ELEMENT and bmask is None:
+        bmask = inputs.element_mask(seed + 100, n, keep_prob)
     mk = oracle_mask_kwargs(mask_kind, block, bmask)
     sc = None if scale == 0.0 else scale
     O_ref, LSE_ref = orc.attn_fwd(x["Q"], x["K"], x["V"], scale=sc, **mk)
@@ -67,7 +71,10 @@ def run_case(b, h, n, d, dtype, mask_kind, *, seed=7, block=128, bmask=None, cfg
 
     dev = {k: to_dev(v, dtype) for k, v in x.items()}
     mask = None
-    if mask_kind != inputs.MASK_NONE:
+    if mask_kind == inputs.MASK_ELEMENT:
+        # the library takes the keep matrix as a bitmap, one bit per entry
+        mask = B.Mask(kind=mask_kind, block_mask=torch.from_numpy(inputs.pack_element_mask(bmask)).cuda())
+    elif mask_kind != inputs.MASK_NONE:
         mask = B.Mask(kind=mask_kind, block=block,
                       block_mask=torch.from_numpy(bmask).cuda() if bmask is not None else None)
     dt = B.ATTN_BF16 if dtype == "bf16" else B.ATTN_F32

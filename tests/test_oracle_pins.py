@@ -154,6 +154,43 @@ def test_gradients_against_torch_autograd_float64():
             np.testing.assert_allclose(mine, theirs.numpy(), rtol=1e-10, atol=1e-13)
 
 
+def test_element_mask_against_autograd_and_central_differences():
+    """An arbitrary set of kept entries, a different one per head, with a row and a column that keep nothing
+    (the coordinate-list sparsity of Section 4.1 as an explicit keep matrix): the textbook formula with the
+    dropped scores at minus infinity, differentiated by a library in float64, and central differences of
+    L = sum(O o G) (an index swap between rows and columns of the mask, or between the heads' masks, fails)."""
+    torch = pytest.importorskip("torch")
+    n, d = 11, 5
+    Q, K, V, G = make(16, n, d, b=1, h=2)
+    keep = inputs.element_mask(17, n, 0.45, heads=2)
+    keep[0, 3, :] = 0
+    keep[1, :, 6] = 0
+    keep[1, 0, 0] = 1
+    mk = dict(mask_kind=orc.MASK_ELEMENT, mask_bits=keep)
+    O, LSE = orc.attn_fwd(Q, K, V, **mk)
+    dQ, dK, dV = orc.attn_bwd(Q, K, V, O, G, LSE, **mk)
+    q, k, v = (torch.tensor(a, dtype=torch.float64, requires_grad=True) for a in (Q, K, V))
+    s = (q @ k.transpose(-1, -2)) / math.sqrt(d)
+    s = s.masked_fill(~torch.from_numpy(keep.astype(bool))[None], float("-inf"))
+    pr = torch.nan_to_num(torch.softmax(s, dim=-1), nan=0.0)       # a row that keeps nothing: all zeros
+    o = pr @ v
+    (o * torch.from_numpy(G)).sum().backward()
+    np.testing.assert_allclose(O, o.detach().numpy(), rtol=1e-12, atol=1e-14)
+    assert np.all(O[0, 0, 3] == 0) and LSE[0, 0, 3] == -np.inf
+    np.testing.assert_allclose(dV, v.grad.numpy(), rtol=1e-10, atol=1e-13)
+    assert np.all(dV[0, 1, 6] == 0) and np.all(dK[0, 1, 6] == 0)
+    h = 1e-5
+    rng = np.random.default_rng(18)
+    for name, X, g in (("Q", Q, dQ), ("K", K, dK), ("V", V, dV)):
+        for _ in range(12):
+            idx = tuple(int(rng.integers(0, sz)) for sz in X.shape)
+            old = X[idx]
+            X[idx] = old + h; lp = loss(Q, K, V, G, **mk)
+            X[idx] = old - h; lm = loss(Q, K, V, G, **mk)
+            X[idx] = old
+            assert abs((lp - lm) / (2 * h) - g[idx]) <= 1e-7 * max(1.0, abs(g[idx])), (name, idx)
+
+
 def test_dense_intermediates_invariants():
     """Rows of f sum to 1; rows of p sum to 0; (f o q) 1 = (O o dO) 1 (the two matrix
     forms of Definition B.9); p equals the row form (diag(f_i) - f_i f_i^T) q_i;
