@@ -52,6 +52,9 @@ def kept_entries(w: inputs.Workload, bmask) -> float:
         return float(w.n) * w.n
     if w.mask == inputs.MASK_CAUSAL:
         return float(w.n) * w.n / 2
+    if w.mask == inputs.MASK_BLOCK_SPARSE_CAUSAL:   # blocks below the diagonal whole, kept diagonal blocks as one half
+        m = bmask[0].astype(bool)
+        return (float(np.tril(m, -1).sum()) + 0.5 * float(np.diag(m).sum())) * w.block * w.block
     return float(bmask[0].sum()) * w.block * w.block
 
 
@@ -149,7 +152,7 @@ def cpu_baseline(w: inputs.Workload, bmask, budget_s: float = 15.0):
     """Times the float64 oracle's backward on a bounded sample: whole (batch, head) units."""
     from oracle import oracle as orc
     kind = {inputs.MASK_NONE: orc.MASK_NONE, inputs.MASK_CAUSAL: orc.MASK_CAUSAL,
-            inputs.MASK_BLOCK_SPARSE: orc.MASK_BLOCK}[w.mask]
+            inputs.MASK_BLOCK_SPARSE: orc.MASK_BLOCK, inputs.MASK_BLOCK_SPARSE_CAUSAL: orc.MASK_BLOCK_CAUSAL}[w.mask]
     mk = dict(mask_kind=kind, block=w.block, mask_bits=bmask)
 
     def run(units):
@@ -175,25 +178,25 @@ def run_reference(args, w, bmask, rank, world):
         return
     from oracle import oracle as orc
     kind = {inputs.MASK_NONE: orc.MASK_NONE, inputs.MASK_CAUSAL: orc.MASK_CAUSAL,
-            inputs.MASK_BLOCK_SPARSE: orc.MASK_BLOCK}[w.mask]
+            inputs.MASK_BLOCK_SPARSE: orc.MASK_BLOCK, inputs.MASK_BLOCK_SPARSE_CAUSAL: orc.MASK_BLOCK_CAUSAL}[w.mask]
     mk = dict(mask_kind=kind, block=w.block, mask_bits=bmask)
     x = {k: v.astype(np.float64)[None] for k, v in w.tensors(head_slice=(0, 1)).items()}
     # sample: the leading r rows of one (batch, head) unit.  For the causal workload this
     # is a self-contained sub-problem (rows < r only see keys < r); r is sized so that
     # all steps end within about two minutes.
     r = min(w.n, 1024)
-    if w.mask == inputs.MASK_BLOCK_SPARSE:
+    if inputs.is_block_mask(w.mask):
         r = w.n
     xs = {k: np.ascontiguousarray(v[:, :, :r]) for k, v in x.items()}
     mks = dict(mk)
-    if w.mask == inputs.MASK_BLOCK_SPARSE:
+    if inputs.is_block_mask(w.mask):
         mks["mask_bits"] = bmask
     O, LSE = orc.attn_fwd(xs["Q"], xs["K"], xs["V"], **mks)
     t = time.perf_counter()
     orc.attn_bwd(xs["Q"], xs["K"], xs["V"], O, xs["dO"], LSE, **mks)
     t_probe = time.perf_counter() - t
     total_steps = args.steps + args.warmup
-    if w.mask != inputs.MASK_BLOCK_SPARSE:
+    if not inputs.is_block_mask(w.mask):
         while r * 2 <= w.n and t_probe * 4 * total_steps < 120.0:
             r *= 2
             t_probe *= 4
@@ -228,7 +231,8 @@ def run_reference(args, w, bmask, rank, world):
 
 
 def workload_name(w):
-    mask = {0: "no mask", 1: "causal", 2: f"block-sparse {w.block}x{w.block} p={w.keep_prob}"}[w.mask]
+    mask = {0: "no mask", 1: "causal", 2: f"block-sparse {w.block}x{w.block} p={w.keep_prob}",
+            3: f"block-sparse {w.block}x{w.block} p={w.keep_prob} AND causal"}[w.mask]
     return f"{w.name}: batch={w.batch} heads={w.heads} n={w.n} d={w.d} {w.dtype} {mask}"
 
 
@@ -294,6 +298,10 @@ def main():
     ap.add_argument("--heads", type=int, default=0, help="override the workload's heads")
     ap.add_argument("--keep-prob", type=float, default=0.0,
                     help="override the off-diagonal keep probability of a block-sparse workload (density sweep)")
+    ap.add_argument("--mask-block", type=int, default=0,
+                    help="override the block edge of a block-sparse workload (128, 64 or 32; the mask is redrawn at that edge)")
+    ap.add_argument("--block-causal", action="store_true",
+                    help="block-sparse workload: also drop the entries above the diagonal (block mask AND causal)")
     ap.add_argument("--profile", action="store_true",
                     help="for runs under ncu: allow fewer than 3 warm-up steps, skip e2e and the CPU baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -313,8 +321,12 @@ def main():
     if args.batch or args.heads:
         w = inputs.Workload(**{**w.__dict__, "batch": args.batch or w.batch, "heads": args.heads or w.heads,
                                "name": w.name + "-reduced"})
-    if args.keep_prob and w.mask == inputs.MASK_BLOCK_SPARSE:
+    if args.keep_prob and inputs.is_block_mask(w.mask):
         w = inputs.Workload(**{**w.__dict__, "keep_prob": args.keep_prob, "name": w.name + "-density"})
+    if (args.mask_block or args.block_causal) and inputs.is_block_mask(w.mask):
+        w = inputs.Workload(**{**w.__dict__, "block": args.mask_block or w.block,
+                               "mask": inputs.MASK_BLOCK_SPARSE_CAUSAL if args.block_causal else w.mask,
+                               "name": w.name + "-variant"})
     bmask = w.block_mask()
 
     if args.impl == "reference":
@@ -560,14 +572,14 @@ def main():
     # the paper's I/O bound (Theorem 1.1 / 1.2, constant 1, elements -> bytes) at this configuration's on-chip size
     elem = 2 if w.bf16 else 4
     M = attn.attn_cfg_onchip_elems(w.d, dt_code, cfg, True)
-    if w.mask == inputs.MASK_BLOCK_SPARSE:
+    if inputs.is_block_mask(w.mask):
         bound_el = attn.attn_io_bound_sparse_elems(w.n * w.d, kept_entries(w, bmask), M) if M else None
     else:
         bound_el = attn.attn_io_bound_elems(w.n, w.d, M, True) * (0.5 if w.mask == inputs.MASK_CAUSAL else 1.0) if M else None
     comp = (8 * w.n * w.d * elem + 2 * 4 * w.n) * w.batch * w.heads
     io = {"backward_compulsory_bytes": comp, "onchip_elems_M": M,
           # Theorem 1.2: Z_input^2 / Z_QK is the cache size at which the two terms of the sparse bound meet
-          "sparse_dividing_M": (float(w.n * w.d) ** 2 / kept_entries(w, bmask)) if w.mask == inputs.MASK_BLOCK_SPARSE else None,
+          "sparse_dividing_M": (float(w.n * w.d) ** 2 / kept_entries(w, bmask)) if inputs.is_block_mask(w.mask) else None,
           "kept_entries_per_head": kept_entries(w, bmask),
           "paper_bound_bytes_at_M": bound_el * elem * w.batch * w.heads if bound_el else None,
           "dram_bytes_from_profile_dominant_kernel": traffic_of(max(tot, key=tot.get), w.name) if tot else None}
@@ -613,6 +625,22 @@ def main():
 # SHA-1 that file had when the counters were taken: once the file has changed the entry is stale and the
 # bench reports null instead.
 TRAFFIC: dict = {
+    ("tc_bwd_fused", "C3"): {"bytes": 6.07e+08, "src": "attn_tc_bwd.cu", "sha1": "b1f46a636f189e46f6aa28e8a67431c4588b29a8",
+                 "note": "16 of 32 heads captured, x 2"},
+    ("tc_fwd", "C3"): {"bytes": 2.386e+08, "src": "attn_tc_fwd.cu", "sha1": "3e482a01da96fd761afa70217fad46c2f835e4dd",
+                 "note": "16 of 32 heads captured, x 2"},
+    ("tc_bwd_fused64", "C3"): {"bytes": 5.904e+08, "src": "attn_tc_bwd64.cu", "sha1": "a71a96f8af4e8f387830d7fc92c83e7e4968337e",
+                 "note": "16 of 32 heads captured, x 2"},
+    ("tc_bwd_dkdv", "C3"): {"bytes": 3.47e+08, "src": "attn_tc_bwd.cu", "sha1": "b1f46a636f189e46f6aa28e8a67431c4588b29a8",
+                 "note": "16 of 32 heads captured, x 2"},
+    ("tc_bwd_fused64", "C4"): {"bytes": 1.04e+08, "src": "attn_tc_bwd64.cu", "sha1": "a71a96f8af4e8f387830d7fc92c83e7e4968337e",
+                 "note": "4 of 8 heads captured, x 2; the inputs of either case fit in L2"},
+    ("tc_fwd", "C4"): {"bytes": 5.04e+07, "src": "attn_tc_fwd.cu", "sha1": "3e482a01da96fd761afa70217fad46c2f835e4dd",
+                 "note": "4 of 8 heads captured, x 2; the inputs of either case fit in L2"},
+    ("tc_bwd_fused", "C2"): {"bytes": 1.277e+08, "src": "attn_tc_bwd.cu", "sha1": "b1f46a636f189e46f6aa28e8a67431c4588b29a8",
+                 "note": "the whole workload captured"},
+    ("tc_bwd_fused", "C5"): {"bytes": 3.352e+09, "src": "attn_tc_bwd.cu", "sha1": "b1f46a636f189e46f6aa28e8a67431c4588b29a8",
+                 "note": "8 of 32 heads captured, x 4"},
 }
 
 

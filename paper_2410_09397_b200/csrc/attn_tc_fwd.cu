@@ -230,6 +230,10 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
             const int jt = iter.tile(idx);
             if (jt < 0) continue;
             const int b = k & 1, j0 = jt * TKF;
+            // a mask finer than the tile: the keep bits of this thread's query row and its 32 key columns, fetched
+            // before the wait for S
+            uint32_t kw = 0xffffffffu;
+            if (a.fine.mode) kw = (ig < n && j0 + wg * CW < n) ? fine_word(a.fine, a.mask_heads, bh, true, ig, j0 + wg * CW) : 0u;
             mbar_wait(&bars[FB_S + b], (k >> 1) & 1, ab);
             tcgen05_fence_after();
             const uint32_t T_S = tm + b * 128;
@@ -248,9 +252,6 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant__ CU
                 const bool causal = mask_is_causal(a.mask_kind);
 #pragma unroll
                 static_assert(CW == 32, "one keep word per thread and tile");
-                // a mask finer than the tile: the keep bits of this thread's query row and its 32 key columns
-                uint32_t kw = 0xffffffffu;
-                if (a.fine.mode) kw = (ig < n && j0 + wg * CW < n) ? fine_word(a.fine, a.mask_heads, bh, true, ig, j0 + wg * CW) : 0u;
 #pragma unroll
                 for (int e = 0; e < CW; ++e) {
                     const int jg = j0 + wg * CW + e;
@@ -511,17 +512,24 @@ tc_fwd_rows_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
             for (int c = 0; c < TKF; c += 32) tmem_ld32(T_S + lane_addr + c, *reinterpret_cast<uint32_t(*)[32]>(&v[c]));
             tmem_wait_ld();
             if (need_mask) {
-                // a mask finer than the tile: the keep bits of this thread's query row, one word per 32 key columns
-                uint32_t kw[TKF / 32];
+                const bool edge = (causal && j0 + TKF - 1 > i0) || j0 + TKF > n;   // entries dropped by position as well
 #pragma unroll
                 for (int q = 0; q < TKF / 32; ++q) {
-                    kw[q] = 0xffffffffu;
-                    if constexpr (FINE) kw[q] = (ig < n && j0 + q * 32 < n) ? fine_word(a.fine, a.mask_heads, bh, true, ig, j0 + q * 32) : 0u;
-                }
+                    // a mask finer than the tile: the keep bits of this thread's query row and 32 key columns.  A word that
+                    // keeps all or nothing (the rule with 32- and 64-wide blocks) needs no test per entry
+                    uint32_t kw = 0xffffffffu;
+                    if constexpr (FINE) kw = (ig < n && j0 + q * 32 < n) ? fine_word(a.fine, a.mask_heads, bh, true, ig, j0 + q * 32) : 0u;
+                    if (FINE && !edge && kw == 0xffffffffu) continue;
+                    if (FINE && kw == 0u) {
 #pragma unroll
-                for (int e = 0; e < TKF; ++e) {
-                    const int jg = j0 + e;
-                    if (jg >= n || (causal && jg > ig) || !((kw[e / 32] >> (e % 32)) & 1u)) v[e] = 0xff800000u;   // -inf
+                        for (int e = 0; e < 32; ++e) v[q * 32 + e] = 0xff800000u;   // -inf
+                        continue;
+                    }
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) {
+                        const int jg = j0 + q * 32 + e;
+                        if (jg >= n || (causal && jg > ig) || !((kw >> e) & 1u)) v[q * 32 + e] = 0xff800000u;
+                    }
                 }
             }
             float mx8[8];   // eight independent chains instead of one of 128 dependent maxima

@@ -37,6 +37,10 @@ TENSOR_Q, TENSOR_K, TENSOR_V, TENSOR_DO, TENSOR_AUX = 0, 1, 2, 3, 4
 MASK_NONE, MASK_CAUSAL, MASK_BLOCK_SPARSE, MASK_BLOCK_SPARSE_CAUSAL, MASK_ELEMENT = 0, 1, 2, 3, 4
 
 
+def is_block_mask(kind: int) -> bool:
+    return kind in (MASK_BLOCK_SPARSE, MASK_BLOCK_SPARSE_CAUSAL)
+
+
 def _mix(z: np.ndarray) -> np.ndarray:
     z = z ^ (z >> np.uint64(30))
     z = z * _M1
@@ -159,6 +163,9 @@ class Workload:
         if self.mask == MASK_CAUSAL:
             return self.n * (self.n + 1) // 2
         assert bmask is not None
+        if self.mask == MASK_BLOCK_SPARSE_CAUSAL:   # whole blocks below the diagonal, kept diagonal blocks with j <= i
+            m = bmask[0].astype(bool)
+            return int(np.tril(m, -1).sum()) * self.block * self.block + int(np.diag(m).sum()) * (self.block * (self.block + 1) // 2)
         return int(bmask[0].sum()) * self.block * self.block
 
     def tensors(self, head_slice: tuple[int, int] | None = None) -> dict[str, np.ndarray]:
@@ -175,7 +182,7 @@ class Workload:
         return out
 
     def block_mask(self) -> np.ndarray | None:
-        if self.mask != MASK_BLOCK_SPARSE:
+        if not is_block_mask(self.mask):
             return None
         nb = (self.n + self.block - 1) // self.block
         return block_mask(self.mask_seed, nb, self.keep_prob, heads=1)
