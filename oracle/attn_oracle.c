@@ -33,10 +33,10 @@
  * [batch, heads, n].  Functions are independent per (batch, head).
  *
  * attn_oracle_fwd / attn_oracle_bwd stream one row at a time (memory O(n)), so they
- * also serve the long-sequence workloads.  attn_oracle_dense follows the seven dense
- * steps of the paper's no-cache algorithm (Appendix C.1) literally, without the
- * max shift, materialising the n x n matrices; it is a second implementation that
- * the tests compare the first one with on small inputs.
+ * also serve the long-sequence workloads.  attn_oracle_dense forms, row by row and
+ * without the max shift, the n x n matrices that Definitions B.3 - B.9 name (A, f, q, p)
+ * and the vectors l and (f o q) 1; it is a second implementation that the tests compare
+ * the first one with on small inputs.
  *
  * The attention weights (the paper's own gradient target):
  *   attn_oracle_project      S = A1 X and h = A3 Y, the two products of phase 1 of the
@@ -202,51 +202,42 @@ void attn_oracle_bwd(const double *Q, const double *K, const double *V, const do
     free(D);
 }
 
-/* One head, dense n x n intermediates, following the no-cache algorithm of
- * Appendix C.1 step by step and without the max shift:
- *   A <- scale * Q K^T ; A <- exp(A) ; l <- A 1 ; f <- diag(l)^-1 A ; q <- dO V^T ;
- *   p <- f o q - diag((f o q) 1) f.
- * Masked entries get A = 0 after the exponential.  Outputs (any may be NULL):
- *   l [n], f [n*n], q [n*n], p [n*n], v_fq [n] = (f o q) 1.                       */
+/* One head, the dense n x n matrices of the definitions, unshifted, one query row at a time:
+ *   A_ij = exp(scale q_i . k_j) on kept entries, 0 elsewhere     (Definition B.3)
+ *   l_i  = sum_j A_ij                                            (Definition B.4)
+ *   f_ij = A_ij / l_i                                            (Definition B.5, the form with the inverse)
+ *   q_ij = dO_i . V_j                                            (Definition B.8)
+ *   v_i  = sum_j f_ij q_ij
+ *   p_ij = f_ij (q_ij - v_i)                                     (Definition B.9, row form)
+ * Outputs (any may be NULL): l [n], f [n*n], q [n*n], p [n*n], v_fq [n] = (f o q) 1.          */
 void attn_oracle_dense(const double *Q, const double *K, const double *V, const double *dO, int n, int d,
                        int mask_kind, int block, const uint8_t *mask_bits, double scale,
                        double *l_out, double *f_out, double *q_out, double *p_out, double *v_fq_out)
 {
     mask_t mk = { mask_kind, block, mask_bits, 1 };
-    size_t nn = (size_t)n * n;
-    double *A = (double *)calloc(nn, sizeof(double));
-    double *l = (double *)calloc((size_t)n, sizeof(double));
-    double *f = (double *)calloc(nn, sizeof(double));
-    double *q = (double *)calloc(nn, sizeof(double));
-    double *v = (double *)calloc((size_t)n, sizeof(double));
-    for (int i = 0; i < n; ++i)
-        for (int j = 0; j < n; ++j)
-            A[(size_t)i * n + j] = scale * dot(Q + (long)i * d, K + (long)j * d, d);
-    for (int i = 0; i < n; ++i)
+    double *f = (double *)calloc((size_t)n, sizeof(double));
+    double *q = (double *)calloc((size_t)n, sizeof(double));
+    for (int i = 0; i < n; ++i) {
+        double l = 0.0, v = 0.0;
+        for (int j = 0; j < n; ++j) {
+            f[j] = kept(&mk, n, 0, i, j) ? exp(scale * dot(Q + (long)i * d, K + (long)j * d, d)) : 0.0;
+            l += f[j];
+        }
+        for (int j = 0; j < n; ++j) {
+            f[j] = l > 0.0 ? f[j] / l : 0.0;
+            q[j] = dot(dO + (long)i * d, V + (long)j * d, d);
+            v += f[j] * q[j];
+        }
+        if (l_out) l_out[i] = l;
+        if (v_fq_out) v_fq_out[i] = v;
         for (int j = 0; j < n; ++j) {
             size_t e = (size_t)i * n + j;
-            A[e] = kept(&mk, n, 0, i, j) ? exp(A[e]) : 0.0;
-            l[i] += A[e];
+            if (f_out) f_out[e] = f[j];
+            if (q_out) q_out[e] = q[j];
+            if (p_out) p_out[e] = f[j] * (q[j] - v);
         }
-    for (int i = 0; i < n; ++i)
-        for (int j = 0; j < n; ++j)
-            f[(size_t)i * n + j] = l[i] > 0.0 ? A[(size_t)i * n + j] / l[i] : 0.0;
-    for (int i = 0; i < n; ++i)
-        for (int j = 0; j < n; ++j)
-            q[(size_t)i * n + j] = dot(dO + (long)i * d, V + (long)j * d, d);
-    for (int i = 0; i < n; ++i)
-        for (int j = 0; j < n; ++j) v[i] += f[(size_t)i * n + j] * q[(size_t)i * n + j];
-    if (p_out)
-        for (int i = 0; i < n; ++i)
-            for (int j = 0; j < n; ++j) {
-                size_t e = (size_t)i * n + j;
-                p_out[e] = f[e] * q[e] - v[i] * f[e];
-            }
-    if (l_out) memcpy(l_out, l, sizeof(double) * (size_t)n);
-    if (f_out) memcpy(f_out, f, sizeof(double) * nn);
-    if (q_out) memcpy(q_out, q, sizeof(double) * nn);
-    if (v_fq_out) memcpy(v_fq_out, v, sizeof(double) * (size_t)n);
-    free(A); free(l); free(f); free(q); free(v);
+    }
+    free(f); free(q);
 }
 
 /* out_u = A_u W_{u mod weight_units}; A, out: [units][n][d]; W: [weight_units][d][d], row = input

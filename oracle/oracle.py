@@ -6,13 +6,13 @@ CPU-baseline leg may import it.  It shares nothing with the CUDA library.
 All tensors are numpy float64 arrays shaped ``[batch, heads, n, d]`` (LSE
 ``[batch, heads, n]``).  Mask kinds: 0 none, 1 causal (keep j <= i), 2 block mask
 (uint8 ``[mask_heads, nb, nb]``), 3 explicit element mask (uint8 ``[mask_heads, n, n]``,
-used only to cross-check the other kinds by brute force).
+the reference for ATTN_MASK_ELEMENT and the brute-force check of the other kinds).
 
 ``project`` / ``weight_grad`` / ``attn_weights_bwd`` cover the paper's own gradient target,
 the attention weights X and Y (Definition 3.2, Appendix D).
 
 Also here: ``io_bound_*`` -- the paper's closed-form I/O bounds (Theorem 1.1 and the
-sparse lower bound, Theorem 1.2 / 4.5) written out literally, used to check the
+sparse lower bound, Theorem 1.2 / 4.5) as plain expressions, used to check the
 library's bound calculators.
 """
 from __future__ import annotations
