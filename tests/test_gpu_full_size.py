@@ -16,10 +16,12 @@ from tests import helpers as H
 pytestmark = pytest.mark.gpu
 
 
-def run_full(name, sample_heads, cfg=None, backward=True):
+def run_full(name, sample_heads, cfg=None, backward=True, w=None, element_keep=None):
+    """`w`: a variant of the named workload (other head count, block edge or mask kind); `element_keep`: run with the
+    element mask given as a keep matrix [1][n][n] instead of the workload's own mask."""
     import torch
     import paper_2410_09397_b200 as attn
-    w = inputs.WORKLOADS[name]
+    w = w or inputs.WORKLOADS[name]
     BH = w.batch * w.heads
     tdt = torch.bfloat16 if w.bf16 else torch.float32
     gen = torch.Generator(device="cuda").manual_seed(1234 + w.seed)
@@ -34,7 +36,11 @@ def run_full(name, sample_heads, cfg=None, backward=True):
             dev[k][h].copy_(torch.from_numpy(host[h][k][0]).to(tdt))
     bmask = w.block_mask()
     mask = None
-    if w.mask != inputs.MASK_NONE:
+    mask_kind = w.mask
+    if element_keep is not None:
+        mask_kind, bmask = inputs.MASK_ELEMENT, element_keep
+        mask = attn.Mask(kind=attn.ATTN_MASK_ELEMENT, block_mask=torch.from_numpy(inputs.pack_element_mask(element_keep)).cuda())
+    elif w.mask != inputs.MASK_NONE:
         mask = attn.Mask(kind=w.mask, block=w.block, block_mask=torch.from_numpy(bmask).cuda() if bmask is not None else None)
     view = {k: v.view(w.batch, w.heads, w.n, w.d) for k, v in dev.items()}
     O, LSE = attn.attn_fwd(view["Q"], view["K"], view["V"], mask=mask, cfg=cfg)
@@ -42,7 +48,7 @@ def run_full(name, sample_heads, cfg=None, backward=True):
         dQ, dK, dV = attn.attn_bwd(view["Q"], view["K"], view["V"], O, view["dO"], LSE, mask=mask, cfg=cfg)
     torch.cuda.synchronize()
     assert torch.isfinite(O.float()).all()
-    mk = H.oracle_mask_kwargs(w.mask, w.block, bmask)
+    mk = H.oracle_mask_kwargs(mask_kind, w.block, bmask)
     tol = H.TOL[w.dtype]
     for h in sample_heads:
         x = {k: v.astype(np.float64)[None] for k, v in host[h].items()}
@@ -68,6 +74,31 @@ def test_config3_full_headline():
 def test_config5_full_block_sparse():
     # one head from the first, a middle and the last launch group of the backward
     run_full("C5", [0, 17, 31])
+
+
+def test_config5_shape_with_64_wide_blocks_and_with_the_causal_mask_on_top():
+    """C5's sequence length (n = 32768, 8 heads) with the mask redrawn on 64 x 64 blocks, and with the 128 x 128
+    block mask combined with the causal mask: one head each against the oracle."""
+    base = inputs.WORKLOADS["C5"]
+    w64 = inputs.Workload(**{**base.__dict__, "heads": 8, "block": 64})
+    run_full("C5", [3], w=w64)
+    wbc = inputs.Workload(**{**base.__dict__, "heads": 8, "mask": inputs.MASK_BLOCK_SPARSE_CAUSAL})
+    run_full("C5", [6], w=wbc)
+
+
+def test_config3_shape_with_an_element_mask():
+    """The headline shape (n = 8192, d = 128, 4 heads) under an element mask: a causal band of 1000 keys plus 2 %
+    of all other causal entries at random, so that tiles are empty, partly kept and full; one head against the oracle,
+    on the fused path and on the path without atomics."""
+    import paper_2410_09397_b200 as attn
+    base = inputs.WORKLOADS["C3"]
+    w = inputs.Workload(**{**base.__dict__, "batch": 1, "heads": 4, "mask": inputs.MASK_NONE})
+    n = w.n
+    i, j = np.indices((n, n), dtype=np.int32)
+    keep = ((j <= i) & ((i - j < 1000) | (inputs.element_mask(7, n, 0.02)[0] != 0))).astype(np.uint8)[None]
+    del i, j
+    run_full("C3", [2], w=w, element_keep=keep)
+    run_full("C3", [1], w=w, element_keep=keep, cfg=attn.Cfg(deterministic=1))
 
 
 def test_config3_full_without_atomics():
