@@ -236,7 +236,7 @@ def workload_name(w):
     return f"{w.name}: batch={w.batch} heads={w.heads} n={w.n} d={w.d} {w.dtype} {mask}"
 
 
-def weights_leg(attn, torch, w, dev, peaks, steps=20):
+def weights_leg(attn, torch, w, dev, peaks, phase2=None, steps=20):
     """The memory-bound kernels around the attention proper, timed on their own after the main loop: the
     projection out = A W (S = A1 X, h = A3 Y) and the weight gradient g = A^T G, on tensors of the workload's
     shape with one weight matrix per head.  Returns per-kernel HBM rooflines (algorithmic bytes / event time)."""
@@ -279,6 +279,29 @@ def weights_leg(attn, torch, w, dev, peaks, steps=20):
                      "bytes_per_launch": nbytes[key], "launches_timed": len(lst), "peak_source": peaks["source"]}
     res["note"] = ("out = A W and g = A^T G on tensors of the workload's shape, one d x d weight per head; "
                    "timed separately from the step above")
+    if phase2 is not None:
+        # phase 2 of the large-cache algorithm as one call: the attention backward and both weight gradients
+        # (gX = A1^T dQ, gY = A3^T dV), with the workload's tensors standing in for A1 = S = Q, A2 = K, A3 = h = V
+        O, LSE, mask, cfg, dt_code, bwd_flops = phase2
+        gy = torch.empty_like(g)
+        wsb = torch.empty(max(256, attn.attn_weights_bwd_workspace_bytes(w.n, w.d, w.heads, w.batch, mask, dt_code, cfg)),
+                          dtype=torch.uint8, device="cuda")
+        call = lambda: attn.attn_weights_bwd(dev["Q"], dev["K"], dev["V"], dev["Q"], dev["V"], O, dev["dO"], LSE, w.heads,
+                                             g, gy, mask=mask, cfg=cfg, workspace=wsb)
+        for _ in range(3):
+            call()
+        ts = []
+        for _ in range(max(3, steps // 2)):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); call(); e1.record(); torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        if attn.attn_workspace_status(wsb) != attn.ATTN_OK:
+            raise SystemExit("attn_weights_bwd reported a device-side error")
+        avg = sum(ts) / len(ts)
+        fl = bwd_flops + 2 * 2.0 * units * w.n * w.d * w.d
+        res["weights_bwd"] = {"avg_ms": avg, "min_ms": min(ts), "tflops": fl / (avg * 1e-3) / 1e12, "flops": fl,
+                              "hbm_bytes_of_the_two_weight_gradients": 2 * nbytes["wgrad"],
+                              "note": "attn_weights_bwd as a whole: attention backward + gX + gY"}
     return res
 
 
@@ -611,7 +634,7 @@ def main():
                                "calls_per_step > 1: the API is called on that many chunks of (batch, head) units, "
                                "copies and kernels on three streams; serial_ms_per_step: one call, one stream"}
     if world == 1 and not args.no_weights:
-        line["weights"] = weights_leg(attn, torch, w, dev, peaks)
+        line["weights"] = weights_leg(attn, torch, w, dev, peaks, phase2=(O, LSE, mask, cfg, dt_code, fb))
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(w, bmask)
     print(json.dumps(line), flush=True)
