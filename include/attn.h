@@ -236,7 +236,9 @@ double attn_io_bound_sparse_elems(double z_input, double z_qk, double M);
  * belong to the call are included (D pre-pass, accumulator clear and conversion, the materialised
  * path's P, dP, dS round trips).  The sum is what Theorem 1.1 bounds from below at
  * M = attn_cfg_onchip_elems(); comparing the two shows how close a tile shape is to the bound and
- * how the I/O falls as the tile -- the cache -- grows (Figure 1 of the introduction).  Host only. */
+ * how the I/O falls as the tile -- the cache -- grows (Figure 1 of the introduction).  Host only.
+ * The materialised backward can also be replayed at d = 512 and 1024 (multiples of 64), sizes no kernel of
+ * the library runs: its blocks then hold fewer than d^2 elements, the small-cache side of Theorem 1.1. */
 typedef struct { double loads, stores, reductions; } attn_io_count; /* elements, per head */
 attn_status attn_io_replay(int n, int d, int mask_kind, int dt, const attn_cfg *cfg, int backward,
                            attn_io_count *out /* host */);

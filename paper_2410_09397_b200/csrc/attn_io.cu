@@ -99,7 +99,12 @@ extern "C" attn_status attn_io_replay(int n, int d, int mask_kind, int dt, const
     if (c.algo == ATTN_ALGO_AUTO) c.algo = dt == ATTN_BF16 ? ATTN_ALGO_FUSED : ATTN_ALGO_SIMT;
     if (c.algo == ATTN_ALGO_SIMT) return ATTN_ERR_TILE;      // the fp32 FMA kernels are not tiled for a cache size
     if (c.algo == ATTN_ALGO_MATERIALIZED && !backward) { c.algo = ATTN_ALGO_FUSED; c.tile_q = c.tile_k = c.tile_d = 0; }
-    if (!tc_cfg_supported(d, c, backward)) {
+    // the blocked loop nest of the materialised backward is the same for every head dimension: it can be replayed for
+    // d = 512 or 1024 as well (multiples of 64), where its blocks hold fewer than d^2 elements -- the small-cache side
+    // of Theorem 1.1 -- although no kernel of the library runs those sizes
+    const bool replay_only = c.algo == ATTN_ALGO_MATERIALIZED && backward && d > 256 && d <= 1024 && d % 64 == 0 &&
+                             mat_cfg_supported(256, c);
+    if (!replay_only && !tc_cfg_supported(d, c, backward)) {
         if (!(c.algo == ATTN_ALGO_FUSED && !backward && tc_cfg_supported(d, c, 1))) return ATTN_ERR_TILE;
         c.tile_q = c.tile_k = c.tile_d = 0;
     }

@@ -18,8 +18,11 @@ def rows(n: int, causal: bool):
     mk = B.ATTN_MASK_CAUSAL if causal else B.ATTN_MASK_NONE
     half = 0.5 if causal else 1.0
     names = {B.ATTN_ALGO_FUSED: "fused", B.ATTN_ALGO_MATERIALIZED: "materialised"}
-    for d in (64, 128, 256):
-        for cfg in B.attn_supported_cfgs(d, B.ATTN_BF16):
+    for d in (64, 128, 256, 512, 1024):
+        # d = 512, 1024: replay only (no kernel runs them); the materialised blocks are those of d = 256
+        for cfg in B.attn_supported_cfgs(min(d, 256), B.ATTN_BF16):
+            if d > 256 and cfg.algo != B.ATTN_ALGO_MATERIALIZED:
+                continue
             if cfg.algo not in names:
                 continue
             for det in ((0, 1) if cfg.algo == B.ATTN_ALGO_FUSED else (0,)):
@@ -28,7 +31,7 @@ def rows(n: int, causal: bool):
                     r = B.attn_io_replay(n, d, mk, B.ATTN_BF16, c, True)
                 except B.AttnError:
                     continue
-                M = B.attn_cfg_onchip_elems(d, B.ATTN_BF16, c, True)
+                M = B.attn_cfg_onchip_elems(min(d, 256), B.ATTN_BF16, c, True)
                 large = (n * n * d * d + n * d ** 3) / M * half
                 small = (n * n * d + n * d * d) / M ** 0.5 * half
                 yield {"d": d, "algo": names[cfg.algo] + (" (no atomics)" if det else ""), "tile_q": cfg.tile_q,

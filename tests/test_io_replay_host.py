@@ -84,6 +84,24 @@ def test_materialised_replay_counts_the_n_by_n_round_trips():
     assert r["stores"] == 2 * n + 2 * n * n + n * n + 3 * n * d
 
 
+def test_materialised_replay_beyond_the_kernels_head_sizes_reaches_the_small_cache_regime():
+    """d = 512 and 1024 are replayed although no kernel runs them: there a block of 128 x 32 (65,536 elements) is
+    smaller than d^2, the I/O still never undercuts the bound, and the bound's active branch is n^2 d / sqrt(M)."""
+    n = 4096
+    for d in (512, 1024):
+        cfg = B.Cfg(tile_q=128, tile_k=32, algo=B.ATTN_ALGO_MATERIALIZED)
+        r = B.attn_io_replay(n, d, NONE, B.ATTN_BF16, cfg, True)
+        M = B.attn_cfg_onchip_elems(256, B.ATTN_BF16, cfg, True)
+        assert M < d * d
+        small, large = (n * n * d + n * d * d) / M ** 0.5, (n * n * d * d + n * d ** 3) / M
+        assert small < large and B.attn_io_bound_elems(n, d, M, True) == pytest.approx(small)
+        assert r["total"] >= small
+        tiles = (n // 128) * (n // 32)
+        assert r["loads"] == (2 * n * d + n) + 2 * tiles * (128 + 32) * d + 2 * n * n + 3 * (n // 256) * (256 + d) * n
+    with pytest.raises(B.AttnError):
+        B.attn_io_replay(n, 512, NONE, B.ATTN_BF16, fused(), True)       # the fused tilings exist for d <= 256 only
+
+
 def test_replay_rejects_what_it_cannot_replay():
     with pytest.raises(B.AttnError):
         B.attn_io_replay(1024, 128, B.ATTN_MASK_BLOCK_SPARSE, B.ATTN_BF16, fused(), True)
