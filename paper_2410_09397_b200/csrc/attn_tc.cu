@@ -35,7 +35,8 @@ size_t tc_cfg_onchip_bytes(int d, const attn_cfg &c, int backward)
     // tensor memory: 128 lanes x 4 bytes per column
     if (backward && (c.tile_q == 64 || d == 256))   // 64-query tiles: dV, dK (128 columns each), S^T / P^T, dP^T / dQ^T, V_j at d = 256
         return bwd64_smem_bytes(d) + (size_t)(256 + 128 + (d == 256 ? 128 : 0)) * 128 * 4;
-    if (backward) return bwd_smem_bytes(d) + (size_t)(256 + 2 * d) * 128 * 4;
+    // regions A and B, dK_j and dV_j; d = 64: a second region for dP^T in the columns that would otherwise stay free
+    if (backward) return bwd_smem_bytes(d) + (size_t)(256 + 2 * d + (d == 64 ? 128 : 0)) * 128 * 4;
     return fwd_smem_bytes(d) + (size_t)(256 + d) * 128 * 4;
 }
 

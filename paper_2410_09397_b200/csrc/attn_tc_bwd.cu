@@ -483,6 +483,10 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
     tcgen05_fence_after();
     const uint32_t tm = *tmem_base_s;
     const uint32_t T_A = tm, T_B = tm + 128, T_dV = tm + 256, T_dK = tm + 256 + HD;
+    // d = 64 leaves 128 columns free: dP^T gets a region of its own there, so that S^T(k+1) does not wait for dP^T(k)
+    // to be copied out of region A and dP^T(k+1) does not wait for S^T(k+1)
+    constexpr bool kSplitA = HD == 64;
+    const uint32_t T_A2 = kSplitA ? tm + 384 : T_A;
     constexpr uint32_t HALF_ROWS = 64 * 128;   // byte offset of rows 64.. inside a [128][64] slab
 
     const TileIter iter(a, jt, bh);
@@ -538,6 +542,16 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
                 }
                 mma_commit(&bars[V2_S]);
             };
+            // dP^T = V_j dO_i^T for the whole tile in stage s
+            auto issue_dP = [&](int s) {
+                const uint32_t kdO = desc_lo_kmajor(smem_u32(smem + L::odO + s * L::kTile));
+#pragma unroll
+                for (int kk = 0; kk < HD / 16; ++kk) {
+                    const uint32_t off = (kk / 4) * kSlab + (kk % 4) * 2;
+                    mma_ss_lo(T_A2, kV + off, kdO + off, idesc_s, kk > 0);
+                }
+                mma_commit(&bars[V2_DP]);
+            };
             int idx = 0, it = -1;
             while (idx < iter.raw && (it = iter.tile(idx)) < 0) ++idx;
             if (it >= 0) {
@@ -545,28 +559,36 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
                 mbar_wait(&bars[V2_KV], 0, ab);
                 tcgen05_fence_after();
                 issue_S(0);
+                if (kSplitA) issue_dP(0);
             }
             int k = 0;
             while (idx < iter.raw) {
                 const int s = k & 1;
                 int nidx = idx + 1, nit = -1;
                 while (nidx < iter.raw && (nit = iter.tile(nidx)) < 0) ++nidx;
-                const uint32_t kdO = desc_lo_kmajor(smem_u32(smem + L::odO + s * L::kTile));
-                // dP^T = V_j dO_i^T into region A once every exp / dS warp holds its part of S^T in registers
-                mbar_wait(&bars[V2_SLD], k & 1, ab);
-                tcgen05_fence_after();
-#pragma unroll
-                for (int kk = 0; kk < HD / 16; ++kk) {
-                    const uint32_t off = (kk / 4) * kSlab + (kk % 4) * 2;
-                    mma_ss_lo(T_A, kV + off, kdO + off, idesc_s, kk > 0);
-                }
-                mma_commit(&bars[V2_DP]);
-                // S^T of the next tile into region A as soon as dP^T has been read out of it
-                if (nit >= 0) {
-                    mbar_wait(&bars[V2_DPLD], k & 1, ab);
-                    mbar_wait(&bars[V2_QFULL + (s ^ 1)], ((k + 1) >> 1) & 1, ab);
+                if constexpr (kSplitA) {
+                    // two regions: S^T(k+1) as soon as S^T(k) has been copied out, dP^T(k+1) as soon as dP^T(k) has been
+                    if (nit >= 0) {
+                        mbar_wait(&bars[V2_SLD], k & 1, ab);
+                        mbar_wait(&bars[V2_QFULL + (s ^ 1)], ((k + 1) >> 1) & 1, ab);
+                        tcgen05_fence_after();
+                        issue_S(s ^ 1);
+                        mbar_wait(&bars[V2_DPLD], k & 1, ab);
+                        tcgen05_fence_after();
+                        issue_dP(s ^ 1);
+                    }
+                } else {
+                    // dP^T = V_j dO_i^T into region A once every exp / dS warp holds its part of S^T in registers
+                    mbar_wait(&bars[V2_SLD], k & 1, ab);
                     tcgen05_fence_after();
-                    issue_S(s ^ 1);
+                    issue_dP(s);
+                    // S^T of the next tile into region A as soon as dP^T has been read out of it
+                    if (nit >= 0) {
+                        mbar_wait(&bars[V2_DPLD], k & 1, ab);
+                        mbar_wait(&bars[V2_QFULL + (s ^ 1)], ((k + 1) >> 1) & 1, ab);
+                        tcgen05_fence_after();
+                        issue_S(s ^ 1);
+                    }
                 }
                 ++k;
                 idx = nidx;
@@ -731,7 +753,7 @@ tc_bwd_fused_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constan
             {
                 uint8_t *slab = smem + L::odS + h * SLAB;
                 uint32_t dv[32];
-                tmem_ld32(T_A + lane_addr + c0, dv);
+                tmem_ld32(T_A2 + lane_addr + c0, dv);
                 tmem_wait_ld();
                 tcgen05_fence_before();
                 warp_arrive(&bars[V2_DPLD], lane);   // region A may take the next S^T
