@@ -87,21 +87,23 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
+            self.rows.append((time.perf_counter(), [c.strip() for c in line.split(",")]))
 
-    def stop(self):
+    def stop(self, since: float | None = None, until: float | None = None):
+        """Ends the sampling (first call); only samples taken in [since, until] (perf_counter values) are used."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
-        self.thread.join(timeout=5)
+        if self.proc.poll() is None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+            self.thread.join(timeout=5)
         sm, mx, reasons = [], [], set()
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
-        for r in self.rows:
-            if len(r) < 6:
+        for t, r in self.rows:
+            if len(r) < 6 or (since is not None and t < since) or (until is not None and t > until):
                 continue
             try:
                 sm.append(float(r[0]))
@@ -433,9 +435,19 @@ def main():
                 kernel_ms.setdefault(name, []).append(ms)
     barrier()
     wall_ms = (time.perf_counter() - t_wall) * 1e3
-    clocks = sampler.stop() if rank == 0 else None
     launches = attn.attn_kernel_launches() - launches0
     attn.attn_timing_enable(False)
+    # nvidia-smi samples every 100 ms.  The clock record is of the samples that fell into the timed region; a region too
+    # short to catch one is reported with the samples of the whole run (warm-up included) and says so
+    t_end = time.perf_counter()
+    clocks = None
+    if rank == 0:
+        clocks = sampler.stop(since=t_wall, until=t_end)
+        clocks["window"] = "timed region"
+        if not clocks.get("samples"):
+            clocks = sampler.stop()
+            clocks["window"] = "whole run, warm-up included (no sample fell into the timed region of %.0f ms)" % wall_ms
+            clocks["in_region_samples"] = 0
     fwd_ms = sum(ev[s][0].elapsed_time(ev[s][1]) for s in range(args.steps))
     bwd_ms = sum(ev[s][1].elapsed_time(ev[s][2]) for s in range(args.steps))
     step_ms = sum(ev[s][0].elapsed_time(ev[s][2]) for s in range(args.steps))
@@ -568,7 +580,9 @@ def main():
         # region is shorter than a second and the sampled SM clock stayed within 3 % of its maximum, else the
         # sustained peak (a seconds-long GEMM loop under the power cap)
         sm, smx = (clocks or {}).get("sm_mhz"), (clocks or {}).get("sm_max_mhz")
-        burst = wall_ms < 1000.0 and sm is not None and smx and sm >= 0.97 * smx
+        # a sub-second region without a sample of its own is taken as a burst, the stricter denominator
+        in_region = (clocks or {}).get("in_region_samples", 1) != 0
+        burst = wall_ms < 1000.0 and (not in_region or sm is None or (smx and sm >= 0.97 * smx))
         pk = peaks["bf16_tflops"] if burst else peaks["bf16_tflops_sustained"]
         roofline = {"bound": "tensor", "kernel": top, "achieved": ach, "peak": pk,
                     "unit": "TFLOP/s", "frac": ach / pk, "peak_kind": "burst" if burst else "sustained",
