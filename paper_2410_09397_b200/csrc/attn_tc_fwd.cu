@@ -433,7 +433,12 @@ tc_fwd_rows_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
 #pragma unroll
                 for (uint32_t sl = 0; sl < C::kSlabs; ++sl)
                     tma_load_3d(smem + C::oK + s * C::kKTile + sl * C::kKSlab, &mK, &bars[F2_KFULL + s], sl * 64, jt * TKF, (int)bh);
-                if (k >= NST) mbar_wait(&bars[F2_VEMPTY + s], ((k / NST) - 1) & 1, ab);
+                // The release of a V stage has no barrier of its own (a commit costs the issuing thread about a hundred
+                // cycles per tile): the V stage of tile k - 3 is free when S(k-1) has completed, which the issuing thread
+                // queues right after O += P V of tile k - 3 (products complete in issue order).  S(k-1) is the newest
+                // completion its barrier can have here -- S(k+1) needs the K tile that this thread loads next -- so the
+                // parity wait cannot be a phase behind
+                if (k >= NST) mbar_wait(&bars[F2_S + ((k - 1) & 1)], ((k - 1) >> 1) & 1, ab);
                 mbar_expect_tx(&bars[F2_VFULL + s], C::kKTile);
 #pragma unroll
                 for (uint32_t sl = 0; sl < C::kSlabs; ++sl)
@@ -482,7 +487,6 @@ tc_fwd_rows_kernel(const __grid_constant__ CUtensorMap mQ, const __grid_constant
                 // its completion tells warpgroup b that O_b holds the product of tile k as well
                 if (k + 2 < niter) issue_S(k + 2);
                 else mma_commit(&bars[F2_O + b]);   // the last product of each warpgroup, for the epilogue
-                mma_commit(&bars[F2_VEMPTY + s]);
             }
         }
       }
