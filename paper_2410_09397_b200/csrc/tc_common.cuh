@@ -99,7 +99,7 @@ __device__ __forceinline__ void tcgen05_fence_after()
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
 
-// ------------------------------------------------------------------ TMA (tiled, no multicast)
+// ------------------------------------------------------------------ TMA (tiled; every load is issued by one CTA for itself)
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *m)
 {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
