@@ -301,8 +301,13 @@ def weights_leg(attn, torch, w, dev, peaks, phase2=None, steps=20):
             raise SystemExit("attn_weights_bwd reported a device-side error")
         avg = sum(ts) / len(ts)
         fl = bwd_flops + 2 * 2.0 * units * w.n * w.d * w.d
+        # gX reads A1 (2 B) and the fp32 dQ accumulator (4 B) per element where the backward keeps one
+        # (bf16, d = 64 or 128, fused, with atomics); otherwise the stored dQ, like gY
+        acc = w.bf16 and w.d in (64, 128) and not (cfg and (cfg.deterministic or cfg.algo == attn.ATTN_ALGO_MATERIALIZED))
+        gx_bytes = units * w.n * w.d * (elem + 4) + w.heads * w.d * w.d * 4 if acc else nbytes["wgrad"]
         res["weights_bwd"] = {"avg_ms": avg, "min_ms": min(ts), "tflops": fl / (avg * 1e-3) / 1e12, "flops": fl,
-                              "hbm_bytes_of_the_two_weight_gradients": 2 * nbytes["wgrad"],
+                              "hbm_bytes_of_the_two_weight_gradients": gx_bytes + nbytes["wgrad"],
+                              "gX_from_fp32_accumulator": bool(acc),
                               "note": "attn_weights_bwd as a whole: attention backward + gX + gY"}
     return res
 
@@ -662,21 +667,21 @@ def main():
 # SHA-1 that file had when the counters were taken: once the file has changed the entry is stale and the
 # bench reports null instead.
 TRAFFIC: dict = {
-    ("tc_bwd_fused", "C3"): {"bytes": 6.044e+08, "src": "attn_tc_bwd.cu", "sha1": "a9592ca62197ac7e2e16a7185aa63cfa824166f5",
+    ("tc_bwd_fused", "C3"): {"bytes": 5.916e+08, "src": "attn_tc_bwd.cu", "sha1": "1b0a4a390dd829f7fafd8c47cd68eea024361713",
                  "note": "16 of 32 heads captured, x 2"},
     ("tc_fwd", "C3"): {"bytes": 2.362e+08, "src": "attn_tc_fwd.cu", "sha1": "d8be6effe28394a321c2d3d45e60bf375c4da969",
                  "note": "16 of 32 heads captured, x 2"},
     ("tc_bwd_fused64", "C3"): {"bytes": 5.862e+08, "src": "attn_tc_bwd64.cu", "sha1": "a71a96f8af4e8f387830d7fc92c83e7e4968337e",
                  "note": "16 of 32 heads captured, x 2"},
-    ("tc_bwd_dkdv", "C3"): {"bytes": 3.458e+08, "src": "attn_tc_bwd.cu", "sha1": "a9592ca62197ac7e2e16a7185aa63cfa824166f5",
+    ("tc_bwd_dkdv", "C3"): {"bytes": 3.385e+08, "src": "attn_tc_bwd.cu", "sha1": "1b0a4a390dd829f7fafd8c47cd68eea024361713",
                  "note": "16 of 32 heads captured, x 2"},
     ("tc_bwd_fused64", "C4"): {"bytes": 1.038e+08, "src": "attn_tc_bwd64.cu", "sha1": "a71a96f8af4e8f387830d7fc92c83e7e4968337e",
                  "note": "4 of 8 heads captured, x 2; the inputs of either case fit in L2"},
     ("tc_fwd", "C4"): {"bytes": 5.04e+07, "src": "attn_tc_fwd.cu", "sha1": "d8be6effe28394a321c2d3d45e60bf375c4da969",
                  "note": "4 of 8 heads captured, x 2; the inputs of either case fit in L2"},
-    ("tc_bwd_fused", "C2"): {"bytes": 1.284e+08, "src": "attn_tc_bwd.cu", "sha1": "a9592ca62197ac7e2e16a7185aa63cfa824166f5",
+    ("tc_bwd_fused", "C2"): {"bytes": 1.250e+08, "src": "attn_tc_bwd.cu", "sha1": "1b0a4a390dd829f7fafd8c47cd68eea024361713",
                  "note": "the whole workload captured"},
-    ("tc_bwd_fused", "C5"): {"bytes": 3.333e+09, "src": "attn_tc_bwd.cu", "sha1": "a9592ca62197ac7e2e16a7185aa63cfa824166f5",
+    ("tc_bwd_fused", "C5"): {"bytes": 3.249e+09, "src": "attn_tc_bwd.cu", "sha1": "1b0a4a390dd829f7fafd8c47cd68eea024361713",
                  "note": "8 of 32 heads captured, x 4"},
 }
 

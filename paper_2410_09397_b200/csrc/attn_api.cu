@@ -257,6 +257,34 @@ void launch_end(cudaStream_t s)
         g_timing.open = false;
     }
 }
+
+attn_status bwd_internal(const void *Q, const void *K, const void *V, const void *O, const void *dO, const float *LSE,
+                         void *dQ, void *dK, void *dV, int n, int d, int heads, int batch, const attn_mask *mask, int dt,
+                         float scale, const attn_cfg *cfg, void *workspace, size_t workspace_bytes, void *cuda_stream,
+                         bool keep_acc, const float **dQ_acc)
+{
+    if (dQ_acc) *dQ_acc = nullptr;
+    if (!Q || !K || !V || !O || !dO || !LSE || !dQ || !dK || !dV) return ATTN_ERR_NULL;
+    Problem p{};
+    const Args a{n, d, heads, batch, dt, mask, cfg};
+    attn_status st = fill_problem(p, a, 1, scale, workspace, workspace_bytes, cuda_stream);
+    if (st != ATTN_OK) return st;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) || !aligned16(dQ) ||
+        !aligned16(dK) || !aligned16(dV) || ((uintptr_t)LSE & 3))
+        return ATTN_ERR_ALIGN;
+    if ((st = check_arch()) != ATTN_OK) return st;
+    p.Q = Q; p.K = K; p.V = V; p.O = O; p.dO = dO; p.LSE = LSE; p.dQ = dQ; p.dK = dK; p.dV = dV;
+    if (cudaMemsetAsync(p.status, 0, 4, p.stream) != cudaSuccess) return ATTN_ERR_LAUNCH;
+    if (p.cfg.algo == ATTN_ALGO_SIMT) return simt_bwd(p);
+    if ((st = build_block_index(p)) != ATTN_OK) return st;
+    if (p.cfg.algo == ATTN_ALGO_MATERIALIZED) return mat_bwd(p);
+    if (keep_acc && dQ_acc && p.dQ_acc) {
+        // the fused kernels leave the final dQ in the fp32 accumulator; without a destination the conversion is skipped
+        p.dQ = nullptr;
+        *dQ_acc = p.dQ_acc;
+    }
+    return tc_bwd(p);
+}
 }  // namespace attn
 
 using namespace attn;
@@ -285,21 +313,8 @@ attn_status attn_bwd(const void *Q, const void *K, const void *V, const void *O,
                      void *dQ, void *dK, void *dV, int n, int d, int heads, int batch, const attn_mask *mask, int dt,
                      float scale, const attn_cfg *cfg, void *workspace, size_t workspace_bytes, void *cuda_stream)
 {
-    if (!Q || !K || !V || !O || !dO || !LSE || !dQ || !dK || !dV) return ATTN_ERR_NULL;
-    Problem p{};
-    const Args a{n, d, heads, batch, dt, mask, cfg};
-    attn_status st = fill_problem(p, a, 1, scale, workspace, workspace_bytes, cuda_stream);
-    if (st != ATTN_OK) return st;
-    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) || !aligned16(dQ) ||
-        !aligned16(dK) || !aligned16(dV) || ((uintptr_t)LSE & 3))
-        return ATTN_ERR_ALIGN;
-    if ((st = check_arch()) != ATTN_OK) return st;
-    p.Q = Q; p.K = K; p.V = V; p.O = O; p.dO = dO; p.LSE = LSE; p.dQ = dQ; p.dK = dK; p.dV = dV;
-    if (cudaMemsetAsync(p.status, 0, 4, p.stream) != cudaSuccess) return ATTN_ERR_LAUNCH;
-    if (p.cfg.algo == ATTN_ALGO_SIMT) return simt_bwd(p);
-    if ((st = build_block_index(p)) != ATTN_OK) return st;
-    if (p.cfg.algo == ATTN_ALGO_MATERIALIZED) return mat_bwd(p);
-    return tc_bwd(p);
+    return attn::bwd_internal(Q, K, V, O, dO, LSE, dQ, dK, dV, n, d, heads, batch, mask, dt, scale, cfg, workspace,
+                              workspace_bytes, cuda_stream, false, nullptr);
 }
 
 attn_status attn_bwd_preprocess(const void *O, const void *dO, float *D, size_t rows, int d, int dt, void *cuda_stream)

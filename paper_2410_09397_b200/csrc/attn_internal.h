@@ -88,6 +88,15 @@ attn_status simt_bwd(const Problem &p);
 attn_status preprocess_D(const void *O, const void *dO, float *D, size_t rows, int d, int dt, cudaStream_t s);
 attn_status build_block_index(const Problem &p);
 
+// attn_bwd for a caller inside the library that consumes dQ itself (the weight gradients).  With `keep_acc` set and an
+// algorithm that accumulates dQ in fp32 in the workspace, the conversion to the storage type is skipped, dQ is left
+// untouched and *dQ_acc receives the accumulator's address ([batch * heads][n][d], final values); in every other case
+// dQ is written as attn_bwd writes it and *dQ_acc is nullptr.
+attn_status bwd_internal(const void *Q, const void *K, const void *V, const void *O, const void *dO, const float *LSE,
+                         void *dQ, void *dK, void *dV, int n, int d, int heads, int batch, const attn_mask *mask, int dt,
+                         float scale, const attn_cfg *cfg, void *workspace, size_t workspace_bytes, void *cuda_stream,
+                         bool keep_acc, const float **dQ_acc);
+
 // Tensor-core path (attn_tc_*.cu)
 attn_status tc_fwd(const Problem &p);
 attn_status tc_bwd(const Problem &p);

@@ -936,6 +936,7 @@ attn_status bwd_preprocess_launch(const Problem &p, bool clear_acc)
 
 attn_status bwd_dq_convert_launch(const Problem &p)
 {
+    if (!p.dQ) return ATTN_OK;   // the caller reads the fp32 accumulator itself
     const size_t n4 = (size_t)p.BH * p.n * p.d / 4;
     const size_t cap = (size_t)sm_count() * 16;
     const unsigned blocks = (unsigned)((n4 + 255) / 256 < cap ? (n4 + 255) / 256 : cap);

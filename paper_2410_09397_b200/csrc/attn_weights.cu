@@ -4,7 +4,8 @@
 //   attn_project       out = A W per (batch, head) unit        (Appendix D, phase 1)
 //   attn_weight_grad   g  += A^T G over the units of a weight  (closing product of phase 2)
 //   attn_weights_bwd   phase 2 as a whole: attn_bwd for p A2 and f^T dO, then the two
-//                      weight-gradient products
+//                      weight-gradient products (the first one straight from the fp32
+//                      dQ accumulator where the backward has one)
 //
 // Both products stream n x d operands once and produce (or consume) a d x d matrix, so
 // they are bound by HBM bandwidth; the bf16 kernels use tcgen05 only so that the
@@ -474,6 +475,187 @@ wgrad_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ CUt
     if (warp == 0) tmem_dealloc(tm, kTmemCols);
 }
 
+// ===================================================================== g += A^T G with G in fp32 (d = 64, 128)
+// The same product for a G that sits in device memory as fp32 -- the dQ accumulator of the fused backward, so that
+// the closing product of phase 2 (Appendix D) reads it directly: no bf16 copy of dQ is written and read back, and dQ
+// is rounded once, on its way into the product.  Per stage the loading thread brings a bf16 tile of A and the fp32
+// tile of G; warps 0-3 turn the latter into the bf16 MN-major operand (two buffers) and later add finished d x d
+// blocks to g; the issuing thread runs the products.  A stage is free again when its product has completed and all
+// four converting warps have read it (five arrivals).
+template <int HD> struct GradAccSmem {
+    static constexpr int TR = HD == 64 ? 128 : 64;           // rows per stage
+    static constexpr int kStages = 3;
+    static constexpr uint32_t kSlab = TR * 128;              // [TR rows][128 bytes]: 64 bf16 or 32 fp32 a row
+    static constexpr uint32_t kATile = (HD / 64) * kSlab;    // bf16 tile (A, and G after conversion)
+    static constexpr uint32_t kGfTile = (HD / 32) * kSlab;   // fp32 tile of G
+    static constexpr uint32_t kStage = kATile + kGfTile;
+    static constexpr uint32_t oGb = kStages * kStage;        // two converted tiles
+    static constexpr uint32_t oZero = oGb + 2 * kATile;      // d = 64: an all-zero slab, the upper half of M = 128
+    static constexpr uint32_t oBar = oZero + (HD == 64 ? kSlab : 0);
+    static constexpr uint32_t oMisc = oBar + 128;
+    static constexpr uint32_t kBytes = oMisc + 64;
+    static_assert(kBytes <= 227 * 1024, "shared memory budget");
+};
+
+template <int HD>
+__global__ void __launch_bounds__(kGradThreads)
+wgrad_acc_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ CUtensorMap mG, const GradArgs g)
+{
+    static_assert(HD == 64 || HD == 128, "head sizes of the fp32-source weight gradient");
+    using L = GradAccSmem<HD>;
+    constexpr int TR = L::TR, kStages = L::kStages;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem + L::oBar);
+    uint64_t *empty = full + kStages;       // 1 (the product) + 4 (the converting warps)
+    uint64_t *gbfull = empty + kStages;     // [2] converted tile written, 4 arrivals
+    uint64_t *gbfree = gbfull + 2;          // [2] its product has completed
+    uint64_t *done = gbfree + 2;
+    uint64_t *tfree = done + 1;
+    uint32_t *tmem_base_s = reinterpret_cast<uint32_t *>(smem + L::oMisc);
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(smem + L::oMisc + 4);
+    const Abort ab{abort_flag, g.status};
+    constexpr uint32_t kTmemCols = HD;
+
+    const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
+    const long t0 = g.total_tiles * blockIdx.x / gridDim.x, t1 = g.total_tiles * (blockIdx.x + 1) / gridDim.x;
+
+    if ((smem_u32(smem) & 1023u) != 0) {
+        if (tid == 0) atomicExch(g.status, 9u);
+        return;
+    }
+    auto load_stage = [&](int kt, long t) {
+        const int s = kt % kStages;
+        const int unit = (int)(t / g.tiles_per_unit), r0 = (int)(t % g.tiles_per_unit) * TR;
+        uint8_t *sA = smem + s * L::kStage, *sGf = sA + L::kATile;
+        mbar_expect_tx(&full[s], L::kStage);
+#pragma unroll
+        for (int sl = 0; sl < HD / 64; ++sl) tma_load_3d(sA + sl * L::kSlab, &mA, &full[s], sl * 64, r0, unit);
+#pragma unroll
+        for (int sl = 0; sl < HD / 32; ++sl) tma_load_3d(sGf + sl * L::kSlab, &mG, &full[s], sl * 32, r0, unit);
+    };
+    const int early = (int)((t1 - t0) < kStages ? (t1 - t0) : kStages);
+    if (tid == 0) {
+        *abort_flag = 0;
+        for (int b = 0; b < 2; ++b) { mbar_init(&gbfull[b], 4); mbar_init(&gbfree[b], 1); }
+        mbar_init(done, 1);
+        mbar_init(tfree, 128);
+        fence_barrier_init();
+    }
+    if (tid == 4 * 32) {
+        // the loading thread sets up its own ring and fills it before the CTA-wide setup is over
+        for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 5); }
+        fence_barrier_init();
+        for (int kt = 0; kt < early; ++kt) load_stage(kt, t0 + kt);
+    }
+    if (HD == 64) {
+        for (uint32_t i = tid; i < L::kSlab / 16; i += kGradThreads)
+            reinterpret_cast<uint4 *>(smem + L::oZero)[i] = make_uint4(0, 0, 0, 0);
+        fence_proxy_async_smem();
+    }
+    if (warp == 0) tmem_alloc(tmem_base_s, kTmemCols);
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tm = *tmem_base_s;
+
+    if (warp == 4) {
+        if (lane == 0) {
+            int kt = early;
+            for (long t = t0 + early; t < t1; ++t, ++kt) {
+                mbar_wait(&empty[kt % kStages], ((kt / kStages) - 1) & 1, ab);
+                load_stage(kt, t);
+            }
+        }
+    } else if (warp == 5) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = idesc_bf16(128, HD, 1, 1);
+            int kt = 0, flushes = 0;
+            bool fresh = true;
+            for (long t = t0; t < t1; ++t, ++kt) {
+                const int s = kt % kStages, cb = kt & 1;
+                if (fresh && flushes > 0) {            // the previous block must have left tensor memory
+                    mbar_wait(tfree, (flushes - 1) & 1, ab);
+                    tcgen05_fence_after();
+                }
+                mbar_wait(&full[s], (kt / kStages) & 1, ab);
+                mbar_wait(&gbfull[cb], (kt >> 1) & 1, ab);
+                tcgen05_fence_after();
+                const uint32_t sA = smem_u32(smem + s * L::kStage), sG = smem_u32(smem + L::oGb + cb * L::kATile);
+                const uint32_t lboA = HD == 64 ? smem_u32(smem + L::oZero) - sA : L::kSlab;
+                const uint32_t bG = desc_lo_mnmajor(sG, L::kSlab);
+#pragma unroll
+                for (int ks = 0; ks < TR / 16; ++ks)
+                    mma_ss_lo(tm, desc_lo_mnmajor(sA + ks * 2048, lboA), bG + ks * (2048 >> 4), idesc,
+                              (!fresh || ks > 0) ? 1u : 0u);
+                mma_commit(&empty[s]);
+                mma_commit(&gbfree[cb]);
+                fresh = false;
+                const long w = (t / g.tiles_per_unit) % g.weight_units;
+                if (t + 1 == t1 || ((t + 1) / g.tiles_per_unit) % g.weight_units != w) {
+                    mma_commit(done);
+                    ++flushes;
+                    fresh = true;
+                }
+            }
+        }
+    } else {
+        // converting warps: thread -> (row, column range) of the stage's tile; a 16-byte chunk of the swizzled fp32 slab
+        // holds 4 columns, of the bf16 slab 8
+        constexpr int kColsPerThread = HD * TR / 128;
+        const int row = tid % TR, col0 = (tid / TR) * kColsPerThread;
+        const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+        const int grow = warp * 32 + lane;    // row of the d x d block this thread adds to g
+        int flushes = 0, kt = 0;
+        for (long t = t0; t < t1; ++t, ++kt) {
+            const int s = kt % kStages, cb = kt & 1;
+            mbar_wait(&full[s], (kt / kStages) & 1, ab);
+            if (kt >= 2) mbar_wait(&gbfree[cb], ((kt >> 1) - 1) & 1, ab);
+            const uint8_t *sGf = smem + s * L::kStage + L::kATile;
+            uint8_t *sGb = smem + L::oGb + cb * L::kATile;
+#pragma unroll
+            for (int j = 0; j < kColsPerThread; j += 8) {
+                const uint32_t c = col0 + j, cc = c % 32;
+                const uint8_t *src = sGf + (c / 32) * L::kSlab + row * 128;
+                const float4 lo = *reinterpret_cast<const float4 *>(src + ((((cc >> 2)) ^ (row & 7)) << 4));
+                const float4 hi = *reinterpret_cast<const float4 *>(src + ((((cc >> 2) + 1) ^ (row & 7)) << 4));
+                *reinterpret_cast<uint4 *>(sGb + (c / 64) * L::kSlab + sw128_offset(row, c % 64)) =
+                    make_uint4(pack_bf16(lo.x, lo.y), pack_bf16(lo.z, lo.w), pack_bf16(hi.x, hi.y), pack_bf16(hi.z, hi.w));
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(&gbfull[cb]);
+                mbar_arrive(&empty[s]);
+            }
+            const long w = (t / g.tiles_per_unit) % g.weight_units;
+            if (!(t + 1 == t1 || ((t + 1) / g.tiles_per_unit) % g.weight_units != w)) continue;
+            // the last tile of a weight's block: add the block to g
+            mbar_wait(done, flushes & 1, ab);
+            tcgen05_fence_after();
+            float *grow_p = g.g + (size_t)w * HD * HD + (size_t)grow * HD;
+            if (HD != 64 || warp < 2) {
+#pragma unroll 1
+                for (int c = 0; c < HD; c += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(tm + lane_addr + c, v);
+                    tmem_wait_ld();
+                    if (*abort_flag) continue;
+#pragma unroll
+                    for (int e = 0; e < 32; e += 4)
+                        red_add_v4(grow_p + c + e, __uint_as_float(v[e]), __uint_as_float(v[e + 1]), __uint_as_float(v[e + 2]),
+                                   __uint_as_float(v[e + 3]));
+                }
+            }
+            tcgen05_fence_before();
+            mbar_arrive(tfree);
+            ++flushes;
+        }
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tm, kTmemCols);
+}
+
 // ===================================================================== fp32 FMA kernels (any dtype, d % 8 == 0)
 template <typename T> __device__ __forceinline__ float to_f(T v);
 template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
@@ -606,6 +788,30 @@ attn_status launch_grad(const void *A, const void *G, float *g, int n, long BH, 
     return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_LAUNCH;
 }
 
+template <int HD>
+attn_status launch_grad_acc(const void *A, const float *G, float *g, int n, long BH, long wu, uint32_t *status, cudaStream_t s)
+{
+    using L = GradAccSmem<HD>;
+    CUtensorMap mA, mG;
+    if (!make_tmap_bf16_3d(&mA, A, HD, (uint64_t)n, (uint64_t)BH, L::TR) ||
+        !make_tmap_f32_3d(&mG, G, HD, (uint64_t)n, (uint64_t)BH, L::TR))
+        return ATTN_ERR_LAUNCH;
+    if (cudaFuncSetAttribute(wgrad_acc_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::kBytes) != cudaSuccess)
+        return ATTN_ERR_LAUNCH;
+    if (cudaMemsetAsync(g, 0, (size_t)wu * HD * HD * sizeof(float), s) != cudaSuccess) return ATTN_ERR_LAUNCH;
+    GradArgs a{};
+    a.g = g; a.status = status; a.n = n;
+    a.tiles_per_unit = (n + L::TR - 1) / L::TR;
+    a.total_tiles = (long)a.tiles_per_unit * BH;
+    a.weight_units = wu;
+    const long sms = sm_count();
+    const unsigned grid = (unsigned)(a.total_tiles < sms ? a.total_tiles : sms);
+    launch_begin("wgrad_acc", s);
+    wgrad_acc_kernel<HD><<<grid, kGradThreads, L::kBytes, s>>>(mA, mG, a);
+    launch_end(s);
+    return cudaGetLastError() == cudaSuccess ? ATTN_OK : ATTN_ERR_LAUNCH;
+}
+
 template <typename T>
 attn_status launch_simt_project(const void *A, const void *W, void *out, int n, int d, long BH, long wu, cudaStream_t s)
 {
@@ -714,11 +920,19 @@ attn_status attn_weights_bwd(const void *A1, const void *A2, const void *A3, con
     uint8_t *base = (uint8_t *)workspace;
     void *dS = base + align_up(inner, 256), *dK = (uint8_t *)dS + tensor, *dh = (uint8_t *)dK + tensor;
     // gradients of S = A1 X (p A2, times the scale), of A2 and of h = A3 Y (f^T dO)
-    st = attn_bwd(S, A2, h, O, dO, LSE, dS, dK, dh, n, d, heads, batch, mask, dt, scale, cfg, workspace, inner, cuda_stream);
+    // where the backward leaves dS (the gradient of S = A1 X) in its fp32 accumulator, gX is formed from that
+    const float *acc = nullptr;
+    const bool from_acc = dt == ATTN_BF16 && (d == 64 || d == 128);
+    st = bwd_internal(S, A2, h, O, dO, LSE, dS, dK, dh, n, d, heads, batch, mask, dt, scale, cfg, workspace, inner,
+                      cuda_stream, from_acc, &acc);
     if (st != ATTN_OK) return st;
     cudaStream_t s = (cudaStream_t)cuda_stream;
     const long BH = (long)heads * batch;
-    st = grad_impl(A1, dS, gX, n, d, BH, weight_units, dt, (uint32_t *)workspace, s);
+    if (acc)
+        st = d == 64 ? launch_grad_acc<64>(A1, acc, gX, n, BH, weight_units, (uint32_t *)workspace, s)
+                     : launch_grad_acc<128>(A1, acc, gX, n, BH, weight_units, (uint32_t *)workspace, s);
+    else
+        st = grad_impl(A1, dS, gX, n, d, BH, weight_units, dt, (uint32_t *)workspace, s);
     if (st != ATTN_OK) return st;
     if (gY) st = grad_impl(A3, dh, gY, n, d, BH, weight_units, dt, (uint32_t *)workspace, s);
     return st;

@@ -299,7 +299,9 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 // rank-3 bf16 tensor [dim2][dim1][dim0] (dim0 contiguous), box [1][box1][64], 128-byte swizzle,
 // out-of-range elements read as zero.  Returns false if the driver refuses.
 bool make_tmap_bf16_3d(CUtensorMap *out, const void *base, uint64_t dim0, uint64_t dim1, uint64_t dim2, uint32_t box1);
-// the same with the row pitch (elements), the box [1][box1][box0] and the swizzle span (64 or 128 bytes;
+// rank-3 fp32 tensor [dim2][dim1][dim0], box [1][box1][32] (128 bytes a row), 128-byte swizzle
+bool make_tmap_f32_3d(CUtensorMap *out, const void *base, uint64_t dim0, uint64_t dim1, uint64_t dim2, uint32_t box1);
+// the same as the first with the row pitch (elements), the box [1][box1][box0] and the swizzle span (64 or 128 bytes;
 // box0 * 2 bytes must not exceed it) given: the maps of the tiles that TMA stores write
 bool make_tmap_bf16_3d_box(CUtensorMap *out, const void *base, uint64_t dim0, uint64_t dim1, uint64_t dim2, uint64_t pitch_elems,
                            uint32_t box0, uint32_t box1, int swizzle_bytes);

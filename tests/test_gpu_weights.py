@@ -86,7 +86,7 @@ E2E_CASES = [
     (2, 2, 300, 64, "bf16", "heads", inputs.MASK_CAUSAL),
     (2, 2, 392, 128, "bf16", "heads", inputs.MASK_NONE),
     (1, 2, 392, 128, "bf16", "all", inputs.MASK_CAUSAL),
-    (1, 2, 264, 256, "bf16", "one", inputs.MASK_NONE),     # backward through the materialised algorithm
+    (1, 2, 264, 256, "bf16", "one", inputs.MASK_NONE),     # backward with 64-query tiles, gX from the stored dQ
 ]
 
 
@@ -172,3 +172,50 @@ def test_weight_gradients_through_a_block_sparse_mask():
     torch.cuda.synchronize()
     assert attn.attn_workspace_status(ws) == attn.ATTN_OK
     assert rel_err(to_np(gX), ref["gX"]) <= TOL["bf16"] and rel_err(to_np(gY), ref["gY"]) <= TOL["bf16"]
+
+
+ALGO_CASES = [
+    # d, n, configuration of the attention backward inside attn_weights_bwd
+    (128, 392, dict()),                                   # fused, 128-query tiles: gX read from the fp32 dQ accumulator
+    (64, 300, dict()),
+    (128, 392, dict(algo="fused", tile_q=64)),            # fused, 64-query tiles: the accumulator as well
+    (128, 392, dict(deterministic=1)),                    # no accumulator: gX from the stored dQ
+    (64, 300, dict(deterministic=1)),
+    (128, 264, dict(algo="materialized")),
+    (256, 264, dict()),                                   # accumulator, but a head size the fp32-source kernel lacks
+]
+
+
+@pytest.mark.parametrize("d,n,cfg_kw", ALGO_CASES)
+def test_weight_gradients_for_every_backward_algorithm(d, n, cfg_kw):
+    """gX and gY through attn_weights_bwd with each algorithm of the attention backward (causal mask, one weight
+    per head, a ragged last tile), against the oracle; where dQ is accumulated in fp32 the result must also agree
+    with the product formed from the stored bf16 dQ of attn_bwd to within the storage rounding."""
+    import torch
+    import paper_2410_09397_b200 as attn
+    from paper_2410_09397_b200 import binding as B
+    b, h = 2, 2
+    A1, A2, A3, dO = (inputs.normal_tensor(41, t, (b, h, n, d), bf16=True) for t in range(4))
+    X, Y = weights(41, 4, h, d, "bf16"), weights(41, 5, h, d, "bf16")
+    ref = orc.attn_weights_bwd(A1, A2, A3, X, Y, dO, mask_kind=inputs.MASK_CAUSAL)
+    dev = {k: to_dev(v, "bf16") for k, v in dict(A1=A1, A2=A2, A3=A3, dO=dO, X=X, Y=Y).items()}
+    mask = B.Mask(kind=inputs.MASK_CAUSAL)
+    kw = dict(cfg_kw)
+    if "algo" in kw:
+        kw["algo"] = {"fused": B.ATTN_ALGO_FUSED, "materialized": B.ATTN_ALGO_MATERIALIZED}[kw["algo"]]
+    cfg = B.Cfg(**kw) if kw else None
+    S, hh = attn.attn_project(dev["A1"], dev["X"]), attn.attn_project(dev["A3"], dev["Y"])
+    O, LSE = attn.attn_fwd(S, dev["A2"], hh, mask=mask)
+    ws = torch.zeros(B.attn_weights_bwd_workspace_bytes(n, d, h, b, mask, B.ATTN_BF16, cfg), dtype=torch.uint8,
+                     device="cuda")
+    for _ in range(2):      # the second call finds the workspace as the first left it
+        gX, gY = attn.attn_weights_bwd(dev["A1"], dev["A2"], dev["A3"], S, hh, O, dev["dO"], LSE, h, mask=mask, cfg=cfg,
+                                       workspace=ws)
+        torch.cuda.synchronize()
+        assert attn.attn_workspace_status(ws) == attn.ATTN_OK
+        errs = {"gX": rel_err(to_np(gX), ref["gX"]), "gY": rel_err(to_np(gY), ref["gY"])}
+        assert all(v <= TOL["bf16"] for v in errs.values()), errs
+    dQ, dK, dV = attn.attn_bwd(S, dev["A2"], hh, O, dev["dO"], LSE, mask=mask, cfg=cfg)
+    g2 = attn.attn_weight_grad(dev["A1"], dQ, h)
+    torch.cuda.synchronize()
+    assert rel_err(to_np(gX), to_np(g2)) <= 1e-2
