@@ -302,8 +302,8 @@ def weights_leg(attn, torch, w, dev, peaks, phase2=None, steps=20):
         avg = sum(ts) / len(ts)
         fl = bwd_flops + 2 * 2.0 * units * w.n * w.d * w.d
         # gX reads A1 (2 B) and the fp32 dQ accumulator (4 B) per element where the backward keeps one
-        # (bf16, d = 64 or 128, fused, with atomics); otherwise the stored dQ, like gY
-        acc = w.bf16 and w.d in (64, 128) and not (cfg and (cfg.deterministic or cfg.algo == attn.ATTN_ALGO_MATERIALIZED))
+        # (bf16, fused, with atomics); otherwise the stored dQ, like gY
+        acc = w.bf16 and w.d in (64, 128, 256) and not (cfg and (cfg.deterministic or cfg.algo == attn.ATTN_ALGO_MATERIALIZED))
         gx_bytes = units * w.n * w.d * (elem + 4) + w.heads * w.d * w.d * 4 if acc else nbytes["wgrad"]
         res["weights_bwd"] = {"avg_ms": avg, "min_ms": min(ts), "tflops": fl / (avg * 1e-3) / 1e12, "flops": fl,
                               "hbm_bytes_of_the_two_weight_gradients": gx_bytes + nbytes["wgrad"],

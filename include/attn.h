@@ -163,7 +163,7 @@ attn_status attn_weight_grad(const void *A, const void *G, float *g, int n, int 
  * gX = dL/dX = A1^T p A2 (times `scale` when the scores carry one) and, unless gY is NULL
  * (the paper treats Y as fixed), gY = dL/dY = A3^T f^T dO.  Runs attn_bwd with Q = S,
  * K = A2, V = h into workspace buffers, then the two weight-gradient products; where the
- * backward accumulates dQ in fp32 (fused algorithm, bf16, d = 64 or 128) gX is formed
+ * backward accumulates dQ in fp32 (fused algorithm with atomics, bf16) gX is formed
  * from that accumulator and no bf16 copy of dQ is written.  mask, scale, cfg as in
  * attn_bwd; workspace of attn_weights_bwd_workspace_bytes() bytes. */
 attn_status attn_weights_bwd(const void *A1, const void *A2, const void *A3, const void *S, const void *h,

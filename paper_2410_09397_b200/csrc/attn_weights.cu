@@ -475,7 +475,7 @@ wgrad_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ CUt
     if (warp == 0) tmem_dealloc(tm, kTmemCols);
 }
 
-// ===================================================================== g += A^T G with G in fp32 (d = 64, 128)
+// ===================================================================== g += A^T G with G in fp32
 // The same product for a G that sits in device memory as fp32 -- the dQ accumulator of the fused backward, so that
 // the closing product of phase 2 (Appendix D) reads it directly: no bf16 copy of dQ is written and read back, and dQ
 // is rounded once, on its way into the product.  Per stage the loading thread brings a bf16 tile of A and the fp32
@@ -483,7 +483,7 @@ wgrad_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ CUt
 // blocks to g; the issuing thread runs the products.  A stage is free again when its product has completed and all
 // four converting warps have read it (five arrivals).
 template <int HD> struct GradAccSmem {
-    static constexpr int TR = HD == 64 ? 128 : 64;           // rows per stage
+    static constexpr int TR = 8192 / HD;                     // rows per stage: 48 KB a stage at every head size
     static constexpr int kStages = 3;
     static constexpr uint32_t kSlab = TR * 128;              // [TR rows][128 bytes]: 64 bf16 or 32 fp32 a row
     static constexpr uint32_t kATile = (HD / 64) * kSlab;    // bf16 tile (A, and G after conversion)
@@ -501,7 +501,6 @@ template <int HD>
 __global__ void __launch_bounds__(kGradThreads)
 wgrad_acc_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__ CUtensorMap mG, const GradArgs g)
 {
-    static_assert(HD == 64 || HD == 128, "head sizes of the fp32-source weight gradient");
     using L = GradAccSmem<HD>;
     constexpr int TR = L::TR, kStages = L::kStages;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -514,7 +513,7 @@ wgrad_acc_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__
     uint32_t *tmem_base_s = reinterpret_cast<uint32_t *>(smem + L::oMisc);
     volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(smem + L::oMisc + 4);
     const Abort ab{abort_flag, g.status};
-    constexpr uint32_t kTmemCols = HD;
+    constexpr uint32_t kTmemCols = HD == 256 ? 512 : HD;   // d = 256: two accumulators of 128 rows x 256 columns
 
     const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
     const long t0 = g.total_tiles * blockIdx.x / gridDim.x, t1 = g.total_tiles * (blockIdx.x + 1) / gridDim.x;
@@ -584,9 +583,13 @@ wgrad_acc_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__
                 const uint32_t lboA = HD == 64 ? smem_u32(smem + L::oZero) - sA : L::kSlab;
                 const uint32_t bG = desc_lo_mnmajor(sG, L::kSlab);
 #pragma unroll
-                for (int ks = 0; ks < TR / 16; ++ks)
-                    mma_ss_lo(tm, desc_lo_mnmajor(sA + ks * 2048, lboA), bG + ks * (2048 >> 4), idesc,
-                              (!fresh || ks > 0) ? 1u : 0u);
+                for (int ks = 0; ks < TR / 16; ++ks) {
+                    const uint32_t acc = (!fresh || ks > 0) ? 1u : 0u;
+                    mma_ss_lo(tm, desc_lo_mnmajor(sA + ks * 2048, lboA), bG + ks * (2048 >> 4), idesc, acc);
+                    if (HD == 256)
+                        mma_ss_lo(tm + 256, desc_lo_mnmajor(sA + 2 * L::kSlab + ks * 2048, lboA), bG + ks * (2048 >> 4),
+                                  idesc, acc);
+                }
                 mma_commit(&empty[s]);
                 mma_commit(&gbfree[cb]);
                 fresh = false;
@@ -632,18 +635,21 @@ wgrad_acc_kernel(const __grid_constant__ CUtensorMap mA, const __grid_constant__
             // the last tile of a weight's block: add the block to g
             mbar_wait(done, flushes & 1, ab);
             tcgen05_fence_after();
-            float *grow_p = g.g + (size_t)w * HD * HD + (size_t)grow * HD;
             if (HD != 64 || warp < 2) {
 #pragma unroll 1
-                for (int c = 0; c < HD; c += 32) {
-                    uint32_t v[32];
-                    tmem_ld32(tm + lane_addr + c, v);
-                    tmem_wait_ld();
-                    if (*abort_flag) continue;
+                for (int half = 0; half < (HD == 256 ? 2 : 1); ++half) {
+                    float *grow_p = g.g + (size_t)w * HD * HD + (size_t)(half * 128 + grow) * HD;
+#pragma unroll 1
+                    for (int c = 0; c < HD; c += 32) {
+                        uint32_t v[32];
+                        tmem_ld32(tm + lane_addr + half * 256 + c, v);
+                        tmem_wait_ld();
+                        if (*abort_flag) continue;
 #pragma unroll
-                    for (int e = 0; e < 32; e += 4)
-                        red_add_v4(grow_p + c + e, __uint_as_float(v[e]), __uint_as_float(v[e + 1]), __uint_as_float(v[e + 2]),
-                                   __uint_as_float(v[e + 3]));
+                        for (int e = 0; e < 32; e += 4)
+                            red_add_v4(grow_p + c + e, __uint_as_float(v[e]), __uint_as_float(v[e + 1]),
+                                       __uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
+                    }
                 }
             }
             tcgen05_fence_before();
@@ -922,15 +928,16 @@ attn_status attn_weights_bwd(const void *A1, const void *A2, const void *A3, con
     // gradients of S = A1 X (p A2, times the scale), of A2 and of h = A3 Y (f^T dO)
     // where the backward leaves dS (the gradient of S = A1 X) in its fp32 accumulator, gX is formed from that
     const float *acc = nullptr;
-    const bool from_acc = dt == ATTN_BF16 && (d == 64 || d == 128);
+    const bool from_acc = use_tc(d, dt);
     st = bwd_internal(S, A2, h, O, dO, LSE, dS, dK, dh, n, d, heads, batch, mask, dt, scale, cfg, workspace, inner,
                       cuda_stream, from_acc, &acc);
     if (st != ATTN_OK) return st;
     cudaStream_t s = (cudaStream_t)cuda_stream;
     const long BH = (long)heads * batch;
     if (acc)
-        st = d == 64 ? launch_grad_acc<64>(A1, acc, gX, n, BH, weight_units, (uint32_t *)workspace, s)
-                     : launch_grad_acc<128>(A1, acc, gX, n, BH, weight_units, (uint32_t *)workspace, s);
+        st = d == 64    ? launch_grad_acc<64>(A1, acc, gX, n, BH, weight_units, (uint32_t *)workspace, s)
+             : d == 128 ? launch_grad_acc<128>(A1, acc, gX, n, BH, weight_units, (uint32_t *)workspace, s)
+                        : launch_grad_acc<256>(A1, acc, gX, n, BH, weight_units, (uint32_t *)workspace, s);
     else
         st = grad_impl(A1, dS, gX, n, d, BH, weight_units, dt, (uint32_t *)workspace, s);
     if (st != ATTN_OK) return st;

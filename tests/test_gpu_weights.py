@@ -86,7 +86,7 @@ E2E_CASES = [
     (2, 2, 300, 64, "bf16", "heads", inputs.MASK_CAUSAL),
     (2, 2, 392, 128, "bf16", "heads", inputs.MASK_NONE),
     (1, 2, 392, 128, "bf16", "all", inputs.MASK_CAUSAL),
-    (1, 2, 264, 256, "bf16", "one", inputs.MASK_NONE),     # backward with 64-query tiles, gX from the stored dQ
+    (1, 2, 264, 256, "bf16", "one", inputs.MASK_NONE),     # backward with 64-query tiles
 ]
 
 
@@ -182,7 +182,7 @@ ALGO_CASES = [
     (128, 392, dict(deterministic=1)),                    # no accumulator: gX from the stored dQ
     (64, 300, dict(deterministic=1)),
     (128, 264, dict(algo="materialized")),
-    (256, 264, dict()),                                   # accumulator, but a head size the fp32-source kernel lacks
+    (256, 264, dict()),                                   # 64-query tiles with the head dimension split: accumulator too
 ]
 
 
