@@ -219,3 +219,38 @@ def test_weight_gradients_for_every_backward_algorithm(d, n, cfg_kw):
     g2 = attn.attn_weight_grad(dev["A1"], dQ, h)
     torch.cuda.synchronize()
     assert rel_err(to_np(gX), to_np(g2)) <= 1e-2
+
+
+def test_weights_bwd_at_headline_size_on_sampled_units():
+    """attn_weights_bwd on the launch shape the benchmark times (batch 2 x 16 heads, n = 8192, d = 128, causal, one
+    weight per unit so that every unit's gradient can be read on its own, S = A1 and h = A3 as in the benchmark):
+    for two sampled units the oracle's attention backward followed by its weight-gradient product gives gX and gY."""
+    import torch
+    import paper_2410_09397_b200 as attn
+    from paper_2410_09397_b200 import binding as B
+    w = inputs.WORKLOADS["C3"]
+    b, h, n, d = w.batch, w.heads, w.n, w.d
+    sample = [5, 30]
+    gen = torch.Generator(device="cuda").manual_seed(77)
+    dev = {k: torch.randn((b * h, n, d), generator=gen, device="cuda").to(torch.bfloat16) for k in ("Q", "K", "V", "dO")}
+    host = {}
+    for u in sample:
+        host[u] = w.tensors(head_slice=(u, u + 1))
+        for k in dev:
+            dev[k][u].copy_(torch.from_numpy(host[u][k][0]).to(torch.bfloat16))
+    view = {k: v.view(b, h, n, d) for k, v in dev.items()}
+    mask = B.Mask(kind=inputs.MASK_CAUSAL)
+    O, LSE = attn.attn_fwd(view["Q"], view["K"], view["V"], mask=mask)
+    ws = torch.zeros(B.attn_weights_bwd_workspace_bytes(n, d, h, b, mask, B.ATTN_BF16, None), dtype=torch.uint8,
+                     device="cuda")
+    gX, gY = attn.attn_weights_bwd(view["Q"], view["K"], view["V"], view["Q"], view["V"], O, view["dO"], LSE, b * h,
+                                   mask=mask, workspace=ws)
+    torch.cuda.synchronize()
+    assert attn.attn_workspace_status(ws) == attn.ATTN_OK
+    for u in sample:
+        x = {k: v.astype(np.float64)[None] for k, v in host[u].items()}
+        O_ref, LSE_ref = orc.attn_fwd(x["Q"], x["K"], x["V"], mask_kind=orc.MASK_CAUSAL)
+        dQ, dK, dV = orc.attn_bwd(x["Q"], x["K"], x["V"], O_ref, x["dO"], LSE_ref, mask_kind=orc.MASK_CAUSAL)
+        errs = {"gX": rel_err(to_np(gX[u]), orc.weight_grad(x["Q"], dQ, 1)[0]),
+                "gY": rel_err(to_np(gY[u]), orc.weight_grad(x["V"], dV, 1)[0])}
+        assert all(v <= TOL["bf16"] for v in errs.values()), (u, errs)
